@@ -1,0 +1,157 @@
+/*
+ * w2a8.h -- C ABI of the B200 (sm_100a) W2A8 library: 2-bit weights x int8
+ * activations -> int32 per-group sums -> fp32 outputs.
+ *
+ * Naming (GEMM convention, not the paper's): M = tokens, N = output channels,
+ * K = contraction length, group = number of consecutive k that share one fp32
+ * weight scale.  (The paper calls the weights A [its M x K], the activations
+ * B [its N x K] and the result C.)
+ *
+ * General rules for every entry point
+ *   - Returns a w2a8_status (0 = OK, negative = error).  Never throws, never
+ *     exits, never allocates or frees device memory.
+ *   - Unless a parameter says HOST, every pointer is a DEVICE pointer owned by
+ *     the caller, 16-byte aligned, valid until the enqueued work has run.
+ *     Nothing is retained after the call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
+ *     work is enqueued on it; the calls do not synchronise.
+ *   - Argument errors are detected on the host before anything is launched.
+ *     Launch failures are reported as W2A8_ERR_CUDA.
+ *   - Kernels are launched with programmatic dependent launch: they may start
+ *     while the previous kernel of the stream drains, but touch nothing except
+ *     the frozen weights and scales until that kernel has completed.  Set the
+ *     environment variable W2A8_PDL=0 to launch them plainly.
+ *
+ * Shape rules: K % 64 == 0, N % 16 == 0, M >= 1, K % group == 0 and group is
+ * 64, 128, a multiple of 256, or K itself (one scale per output channel).
+ */
+#ifndef W2A8_H_
+#define W2A8_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    W2A8_OK = 0,
+    W2A8_ERR_NULL = -1,      /* a required pointer is NULL */
+    W2A8_ERR_SHAPE = -2,     /* M, N, K or group violates the shape rules */
+    W2A8_ERR_ALIGN = -3,     /* a pointer is not 16-byte aligned */
+    W2A8_ERR_WORKSPACE = -4, /* workspace missing or too small */
+    W2A8_ERR_CUDA = -5,      /* a CUDA runtime call or launch failed */
+    W2A8_ERR_ARCH = -6       /* the current device is not sm_100 */
+} w2a8_status;
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int w2a8_version(void);
+
+/* Static, human-readable text for a status code. */
+const char *w2a8_status_string(int status);
+
+/*
+ * Size in bytes of the packed form of an N x K code matrix: N * K / 4
+ * (16 two-bit codes per 32-bit word; Sec. II-B: a 256-bit load carries 128
+ * codes).  Returns 0 for shapes that violate the shape rules.
+ */
+size_t w2_packed_bytes(int N, int K);
+
+/*
+ * w2_pack -- re-lay frozen 2-bit codes into the streaming format, once, ahead
+ * of time (Sec. II-B / II-C: weights are frozen at inference, so they are
+ * packed off-line into a layout from which one shift+mask yields int8 lanes in
+ * dot-product order).
+ *   codes  [N][K] uint8, row-major, one code per byte; only the low two bits
+ *          are used (value = code - 2, i.e. {0,1,2,3} -> {-2,-1,0,1}).
+ *   packed [N][K/16] uint32, fully overwritten.  Layout ("W2P"):
+ *          a row is cut into blocks of up to four 64-k slices; inside block b
+ *          with R slices (R = 4 except possibly the last), the word holding
+ *          k = 256 b + 64 s + 16 t + l (s < R, t < 4, l < 16) is word
+ *          16 b + t R + s of the row, and code l sits at bit
+ *          8 (l mod 4) + 2 (l div 4) of that word.
+ */
+int w2_pack(const uint8_t *codes, int N, int K, uint32_t *packed, void *stream);
+
+/*
+ * a8_quantize -- per-token symmetric abs-max quantisation of bf16 activations
+ * to int8 (Sec. II-D: multiply by the inverse of the scale, convert to int8;
+ * the scale comes from the abs-max of the quantisation granule, here one
+ * token).  For token m, all in fp32 with round-to-nearest-even operations:
+ *   amax = max_k |x[m][k]|, a_scale[m] = amax / 127, inv = 1 / a_scale[m],
+ *   a[m][k] = clamp(rne(x[m][k] * inv), -127, 127).
+ * A row with amax == 0, or with a non-finite inv, gives a[m][:] = 0 and
+ * a_scale[m] = 0.  NaN / Inf inputs are outside the contract.
+ *   x_bf16  [M][K] bf16 bit patterns, row-major
+ *   a       [M][K] int8, fully overwritten
+ *   a_scale [M] fp32, fully overwritten (4-byte alignment suffices)
+ */
+int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, void *stream);
+
+/*
+ * Workspace size in bytes that w2a8_gemm / w2a8_gemm_partials need for this
+ * problem (split-K partial outputs and their arrival counters).  Returns 0 for
+ * shapes that violate the shape rules.  The workspace must be zero-filled once
+ * (w2a8_workspace_init) before its first use; the kernels leave it reusable.
+ * One workspace serves any sequence of calls on one stream as long as it is at
+ * least as large as each call needs; calls that may overlap on the device
+ * (different streams) need separate workspaces.
+ */
+size_t w2a8_workspace_bytes(int M, int N, int K, int group);
+
+/* Zero-fill a workspace (asynchronous, on `stream`). */
+int w2a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * w2a8_gemm -- y[m][n] = a_scale[m] * sum_gi w_scale[n][gi] * P[m][n][gi] with
+ * P[m][n][gi] = sum_{k in group gi} a[m][k] * (code[n][k] - 2), the int32
+ * sums being exact (Sec. II-C microkernel: int2 weights up-converted to int8,
+ * int8 multiply-accumulate into int32; Sec. II-D: int32 -> float times the
+ * product of activation and weight scales; K-splitting for small shapes).
+ * fp32 summation order is unspecified but fixed for a given problem shape:
+ * repeated calls give bitwise-equal outputs.
+ *   a       [M][K] int8 (from a8_quantize)         a_scale [M] fp32
+ *   packed  [N][K/16] uint32 (from w2_pack)        w_scale [N][K/group] fp32
+ *   y       [M][N] fp32, row-major, fully overwritten
+ *   workspace / workspace_bytes: see w2a8_workspace_bytes.
+ * M <= 32 takes the memory-bound decode kernel (weights streamed once); larger
+ * M takes the tensor-core prefill path.
+ */
+int w2a8_gemm(const int8_t *a, const float *a_scale, const uint32_t *packed,
+              const float *w_scale, float *y, int M, int N, int K, int group,
+              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * w2a8_gemm_partials -- parity/debug export of the exact int32 per-group sums
+ * P[m][n][gi] computed by the same inner-product code as w2a8_gemm.
+ *   partials [M][N][K/group] int32, fully overwritten.
+ */
+int w2a8_gemm_partials(const int8_t *a, const uint32_t *packed, int32_t *partials,
+                       int M, int N, int K, int group,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Workspace size for w2a8_linear_host: staging for x, a, a_scale and y plus
+ * the GEMM workspace.  Zero-fill once with w2a8_workspace_init.
+ */
+size_t w2a8_linear_host_workspace_bytes(int M, int N, int K, int group);
+
+/*
+ * w2a8_linear_host -- the whole path for callers whose activations live in
+ * HOST memory: copy x to the device, a8_quantize, w2a8_gemm, copy y back
+ * (the fused "bf16 in, scaled output" use of Sec. II-D, with weights resident).
+ *   x_host [M][K] bf16 bit patterns, HOST (pinned memory makes the copies
+ *          asynchronous);  y_host [M][N] fp32, HOST, fully overwritten once the
+ *          stream has run.  packed, w_scale, workspace: DEVICE.
+ * The call itself does not synchronise; synchronise the stream before reading
+ * y_host.
+ */
+int w2a8_linear_host(const void *x_host, int M, int K, const uint32_t *packed,
+                     const float *w_scale, int N, int group, float *y_host,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* W2A8_H_ */

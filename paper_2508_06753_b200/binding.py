@@ -1,0 +1,168 @@
+"""Thin ctypes binding of the C-ABI library ``libw2a8.so`` (see include/w2a8.h).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of
+the library.  torch supplies device memory and the current stream, nothing
+else.  There is no CPU fallback: if the library is missing, ``lib()`` raises.
+Function names match the C entry points.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libw2a8.so")
+
+EXPORTS = [
+    "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
+    "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_gemm", "w2a8_gemm_partials",
+    "w2a8_linear_host_workspace_bytes", "w2a8_linear_host",
+]
+
+_lib = None
+
+
+class W2A8Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load the library once; raise if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2508_06753_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.w2a8_version.restype = i
+        L.w2a8_status_string.restype = ctypes.c_char_p
+        L.w2a8_status_string.argtypes = [i]
+        L.w2_packed_bytes.restype = sz
+        L.w2_packed_bytes.argtypes = [i, i]
+        L.w2_pack.argtypes = [vp, i, i, vp, vp]
+        L.a8_quantize.argtypes = [vp, i, i, vp, vp, vp]
+        L.w2a8_workspace_bytes.restype = sz
+        L.w2a8_workspace_bytes.argtypes = [i, i, i, i]
+        L.w2a8_workspace_init.argtypes = [vp, sz, vp]
+        L.w2a8_gemm.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+        L.w2a8_gemm_partials.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
+        L.w2a8_linear_host_workspace_bytes.restype = sz
+        L.w2a8_linear_host_workspace_bytes.argtypes = [i, i, i, i]
+        L.w2a8_linear_host.argtypes = [vp, i, i, vp, vp, i, i, vp, vp, sz, vp]
+        for name in ("w2_pack", "a8_quantize", "w2a8_workspace_init", "w2a8_gemm",
+                     "w2a8_gemm_partials", "w2a8_linear_host"):
+            getattr(L, name).restype = i
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().w2a8_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise W2A8Error(status, where)
+
+
+def _stream(stream=None) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def w2a8_version() -> int:
+    return int(lib().w2a8_version())
+
+
+def w2_packed_bytes(N: int, K: int) -> int:
+    return int(lib().w2_packed_bytes(N, K))
+
+
+def w2a8_workspace_bytes(M: int, N: int, K: int, group: int) -> int:
+    return int(lib().w2a8_workspace_bytes(M, N, K, group))
+
+
+def w2a8_linear_host_workspace_bytes(M: int, N: int, K: int, group: int) -> int:
+    return int(lib().w2a8_linear_host_workspace_bytes(M, N, K, group))
+
+
+def new_workspace(nbytes: int, device="cuda", stream=None) -> torch.Tensor:
+    """Allocate and zero-fill a workspace of at least `nbytes` bytes."""
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    w2a8_workspace_init(ws, stream)
+    return ws
+
+
+def w2a8_workspace_init(workspace: torch.Tensor, stream=None):
+    _check(lib().w2a8_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                     _stream(stream)), "w2a8_workspace_init")
+
+
+def w2_pack(codes: torch.Tensor, packed: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """codes uint8 [N][K] (device) -> packed int32 [N][K/16] (bit pattern of uint32)."""
+    N, K = codes.shape
+    if packed is None:
+        packed = torch.empty((N, max(K // 16, 1)), dtype=torch.int32, device=codes.device)
+    _check(lib().w2_pack(_ptr(codes), N, K, _ptr(packed), _stream(stream)), "w2_pack")
+    return packed
+
+
+def a8_quantize(x_bf16: torch.Tensor, a: torch.Tensor | None = None,
+                a_scale: torch.Tensor | None = None, stream=None):
+    """x bf16 [M][K] (device) -> (a int8 [M][K], a_scale fp32 [M])."""
+    M, K = x_bf16.shape
+    if a is None:
+        a = torch.empty((M, K), dtype=torch.int8, device=x_bf16.device)
+    if a_scale is None:
+        a_scale = torch.empty((M,), dtype=torch.float32, device=x_bf16.device)
+    _check(lib().a8_quantize(_ptr(x_bf16), M, K, _ptr(a), _ptr(a_scale), _stream(stream)),
+           "a8_quantize")
+    return a, a_scale
+
+
+def w2a8_gemm(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor, w_scale: torch.Tensor,
+              group: int, workspace: torch.Tensor, y: torch.Tensor | None = None, stream=None):
+    """y fp32 [M][N] = scaled W2A8 product; see w2a8_gemm in include/w2a8.h."""
+    M, K = a.shape
+    N = packed.shape[0]
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=a.device)
+    _check(lib().w2a8_gemm(_ptr(a), _ptr(a_scale), _ptr(packed), _ptr(w_scale), _ptr(y), M, N, K,
+                           group, _ptr(workspace), workspace.numel() * workspace.element_size(),
+                           _stream(stream)), "w2a8_gemm")
+    return y
+
+
+def w2a8_gemm_partials(a: torch.Tensor, packed: torch.Tensor, group: int, workspace: torch.Tensor,
+                       partials: torch.Tensor | None = None, stream=None):
+    """Exact int32 per-group sums P[M][N][K/group] (parity/debug export)."""
+    M, K = a.shape
+    N = packed.shape[0]
+    if partials is None:
+        partials = torch.empty((M, N, K // group), dtype=torch.int32, device=a.device)
+    _check(lib().w2a8_gemm_partials(_ptr(a), _ptr(packed), _ptr(partials), M, N, K, group,
+                                    _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                    _stream(stream)), "w2a8_gemm_partials")
+    return partials
+
+
+def w2a8_linear_host(x_host: torch.Tensor, packed: torch.Tensor, w_scale: torch.Tensor, group: int,
+                     y_host: torch.Tensor, workspace: torch.Tensor, stream=None):
+    """Host bf16 x [M][K] -> host fp32 y [M][N]; copies, quantiser and GEMM enqueued on the stream."""
+    M, K = x_host.shape
+    N = packed.shape[0]
+    _check(lib().w2a8_linear_host(_ptr(x_host), M, K, _ptr(packed), _ptr(w_scale), N, group,
+                                  _ptr(y_host), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream(stream)),
+           "w2a8_linear_host")
+    return y_host

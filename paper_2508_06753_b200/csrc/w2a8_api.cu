@@ -1,0 +1,253 @@
+// C ABI of the W2A8 library, the off-line weight packer and the per-token
+// activation quantiser.  Declarations and contracts: include/w2a8.h.
+#include <math.h>
+#include <stdlib.h>
+
+#include "w2a8_common.cuh"
+
+namespace w2a8 {
+
+int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
+                  const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
+                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st);
+size_t decode_workspace_bytes(int M, int N, const ShapeInfo &si);
+
+int env_int(const char *name, int dflt) {
+    const char *v = getenv(name);
+    return (v && *v) ? atoi(v) : dflt;
+}
+
+bool pdl_enabled() {
+    static const bool on = env_int("W2A8_PDL", 1) != 0;
+    return on;
+}
+
+int check_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return W2A8_ERR_CUDA;
+    static int cached_dev = -1, cached_status = 0;
+    if (dev == cached_dev) return cached_status;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return W2A8_ERR_CUDA;
+    cached_status = (major == 10) ? W2A8_OK : W2A8_ERR_ARCH;
+    cached_dev = dev;
+    return cached_status;
+}
+
+// ---- w2_pack ---------------------------------------------------------------------
+// One thread builds one 32-bit word from 16 consecutive codes of a row.
+__global__ void __launch_bounds__(256)
+w2_pack_kernel(const uint8_t *__restrict__ codes, uint32_t *__restrict__ packed, int N, int K,
+               int blocks, int tail_slices) {
+    const int wpr = K / kWordK;
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)N * wpr) return;
+    const int n = (int)(idx / wpr), wi = (int)(idx % wpr);
+    const int b = wi / 16, r = wi % 16;
+    const int R = (b == blocks - 1) ? tail_slices : 4;
+    const int t = r / R, s = r % R;
+    const int k0 = kBlockK * b + kSliceK * s + kWordK * t;
+    const uint4 v = *reinterpret_cast<const uint4 *>(codes + (size_t)n * K + k0);
+    // byte lane bb of v.{x,y,z,w} is code l = 4 j + bb (j = 0..3 for x..w);
+    // it goes to bits [8 bb + 2 j, 8 bb + 2 j + 1]
+    const uint32_t m = 0x03030303u;
+    packed[idx] = (v.x & m) | ((v.y & m) << 2) | ((v.z & m) << 4) | ((v.w & m) << 6);
+}
+
+// ---- a8_quantize -----------------------------------------------------------------
+// One CTA per token.  Pass 1: abs-max over the row (bf16 magnitudes order like
+// their bit patterns).  Pass 2: x * (1 / (amax / 127)), round to nearest even,
+// clamp, store 8 int8 per thread and step.  The row is re-read from L1/L2.
+constexpr int kQuantThreads = 256;
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
+
+__device__ __forceinline__ uint32_t quant4(uint32_t lo, uint32_t hi, float inv) {
+    // lo, hi: two 32-bit words holding four consecutive bf16 values
+    const float x0 = __uint_as_float(lo << 16), x1 = __uint_as_float(lo & 0xFFFF0000u);
+    const float x2 = __uint_as_float(hi << 16), x3 = __uint_as_float(hi & 0xFFFF0000u);
+    int q0 = __float2int_rn(__fmul_rn(x0, inv)), q1 = __float2int_rn(__fmul_rn(x1, inv));
+    int q2 = __float2int_rn(__fmul_rn(x2, inv)), q3 = __float2int_rn(__fmul_rn(x3, inv));
+    q0 = max(-127, min(127, q0)); q1 = max(-127, min(127, q1));
+    q2 = max(-127, min(127, q2)); q3 = max(-127, min(127, q3));
+    return (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) |
+           ((uint32_t)(q3 & 0xFF) << 24);
+}
+
+__global__ void __launch_bounds__(kQuantThreads)
+a8_quantize_kernel(const uint16_t *__restrict__ x, int M, int K, int8_t *__restrict__ a,
+                   float *__restrict__ a_scale) {
+    pdl_launch_dependents();
+    pdl_wait();   // x may come from the previous kernel of the stream
+    const int m = blockIdx.x;
+    const uint4 *xr = reinterpret_cast<const uint4 *>(x + (size_t)m * K);
+    const int nvec = K / 8;
+    uint32_t amax_bits = 0;
+    for (int i = threadIdx.x; i < nvec; i += kQuantThreads) {
+        const uint4 v = xr[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            amax_bits = max(amax_bits, w[j] & 0x7FFFu);
+            amax_bits = max(amax_bits, (w[j] >> 16) & 0x7FFFu);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax_bits = max(amax_bits, __shfl_xor_sync(0xFFFFFFFFu, amax_bits, o));
+    __shared__ uint32_t wmax[kQuantThreads / 32];
+    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = amax_bits;
+    __syncthreads();
+    amax_bits = 0;
+#pragma unroll
+    for (int w = 0; w < kQuantThreads / 32; ++w) amax_bits = max(amax_bits, wmax[w]);
+
+    const float amax = bf16_bits_to_float(amax_bits);
+    const float s = __fdiv_rn(amax, 127.0f);
+    float inv = __fdiv_rn(1.0f, s);
+    const bool dead = !(amax > 0.0f) || !(fabsf(inv) <= 3.402823466e38f);
+    if (dead) inv = 0.0f;
+    if (threadIdx.x == 0) a_scale[m] = dead ? 0.0f : s;
+
+    uint2 *ar = reinterpret_cast<uint2 *>(a + (size_t)m * K);
+    for (int i = threadIdx.x; i < nvec; i += kQuantThreads) {
+        const uint4 v = xr[i];
+        uint2 o;
+        o.x = quant4(v.x, v.y, inv);
+        o.y = quant4(v.z, v.w, inv);
+        ar[i] = o;
+    }
+}
+
+}  // namespace w2a8
+
+// ====================================================================== C ABI ==
+using namespace w2a8;
+
+extern "C" {
+
+int w2a8_version(void) { return 100; }
+
+const char *w2a8_status_string(int status) {
+    switch (status) {
+        case W2A8_OK: return "ok";
+        case W2A8_ERR_NULL: return "null pointer argument";
+        case W2A8_ERR_SHAPE: return "unsupported shape (need K % 64 == 0, N % 16 == 0, M >= 1, "
+                                    "group in {64, 128, multiple of 256, K} dividing K)";
+        case W2A8_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case W2A8_ERR_WORKSPACE: return "workspace missing or too small";
+        case W2A8_ERR_CUDA: return "CUDA runtime or launch error";
+        case W2A8_ERR_ARCH: return "device is not sm_100";
+        default: return "unknown status";
+    }
+}
+
+size_t w2_packed_bytes(int N, int K) {
+    if (!shape_ok(1, N, K, 64, nullptr)) return 0;
+    return (size_t)N * K / 4;
+}
+
+int w2_pack(const uint8_t *codes, int N, int K, uint32_t *packed, void *stream) {
+    if (!codes || !packed) return W2A8_ERR_NULL;
+    ShapeInfo si;
+    if (!shape_ok(1, N, K, 64, &si)) return W2A8_ERR_SHAPE;
+    if (!aligned16(codes) || !aligned16(packed)) return W2A8_ERR_ALIGN;
+    if (int st = check_device()) return st;
+    const size_t words = (size_t)N * si.words_per_row;
+    const unsigned grid = (unsigned)((words + 255) / 256);
+    cudaError_t e = launch_kernel(w2_pack_kernel, dim3(grid), dim3(256), 0, (cudaStream_t)stream,
+                                  false, codes, packed, N, K, si.blocks, si.tail_slices);
+    return e == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
+}
+
+int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, void *stream) {
+    if (!x_bf16 || !a || !a_scale) return W2A8_ERR_NULL;
+    if (M < 1 || K < 64 || K % 64 != 0) return W2A8_ERR_SHAPE;
+    if (!aligned16(x_bf16) || !aligned16(a) || (reinterpret_cast<uintptr_t>(a_scale) & 3u))
+        return W2A8_ERR_ALIGN;
+    if (int st = check_device()) return st;
+    cudaError_t e = launch_kernel(a8_quantize_kernel, dim3(M), dim3(kQuantThreads), 0,
+                                  (cudaStream_t)stream, pdl_enabled(),
+                                  reinterpret_cast<const uint16_t *>(x_bf16), M, K, a, a_scale);
+    return e == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
+}
+
+size_t w2a8_workspace_bytes(int M, int N, int K, int group) {
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return 0;
+    return decode_workspace_bytes(M, N, si);
+}
+
+int w2a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream) {
+    if (!workspace) return W2A8_ERR_NULL;
+    if (cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream) != cudaSuccess)
+        return W2A8_ERR_CUDA;
+    return W2A8_OK;
+}
+
+static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *packed,
+                       const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
+                       int group, void *workspace, size_t workspace_bytes, void *stream) {
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
+    if (!aligned16(a) || !aligned16(packed) || (y && !aligned16(y)) ||
+        (w_scale && !aligned16(w_scale)) || (partials && !aligned16(partials)) ||
+        (a_scale && (reinterpret_cast<uintptr_t>(a_scale) & 3u)))
+        return W2A8_ERR_ALIGN;
+    const size_t need = decode_workspace_bytes(M, N, si);
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
+    if (int st = check_device()) return st;
+    return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,
+                         (cudaStream_t)stream);
+}
+
+int w2a8_gemm(const int8_t *a, const float *a_scale, const uint32_t *packed, const float *w_scale,
+              float *y, int M, int N, int K, int group, void *workspace, size_t workspace_bytes,
+              void *stream) {
+    if (!a || !a_scale || !packed || !w_scale || !y) return W2A8_ERR_NULL;
+    return gemm_common(a, a_scale, packed, w_scale, y, nullptr, M, N, K, group, workspace,
+                       workspace_bytes, stream);
+}
+
+int w2a8_gemm_partials(const int8_t *a, const uint32_t *packed, int32_t *partials, int M, int N,
+                       int K, int group, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!a || !packed || !partials) return W2A8_ERR_NULL;
+    return gemm_common(a, nullptr, packed, nullptr, nullptr, partials, M, N, K, group, workspace,
+                       workspace_bytes, stream);
+}
+
+static inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+
+size_t w2a8_linear_host_workspace_bytes(int M, int N, int K, int group) {
+    const size_t g = w2a8_workspace_bytes(M, N, K, group);
+    if (g == 0) return 0;
+    return up256(g) + up256((size_t)M * K * 2) + up256((size_t)M * K) + up256((size_t)M * 4) +
+           up256((size_t)M * N * 4);
+}
+
+int w2a8_linear_host(const void *x_host, int M, int K, const uint32_t *packed,
+                     const float *w_scale, int N, int group, float *y_host, void *workspace,
+                     size_t workspace_bytes, void *stream) {
+    if (!x_host || !packed || !w_scale || !y_host) return W2A8_ERR_NULL;
+    const size_t need = w2a8_linear_host_workspace_bytes(M, N, K, group);
+    if (need == 0) return W2A8_ERR_SHAPE;
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char *p = reinterpret_cast<char *>(workspace);
+    const size_t gemm_ws = w2a8_workspace_bytes(M, N, K, group);
+    void *ws = p;                     p += up256(gemm_ws);
+    void *x_dev = p;                  p += up256((size_t)M * K * 2);
+    int8_t *a = (int8_t *)p;          p += up256((size_t)M * K);
+    float *a_scale = (float *)p;      p += up256((size_t)M * 4);
+    float *y_dev = (float *)p;
+    if (cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return W2A8_ERR_CUDA;
+    if (int s = a8_quantize(x_dev, M, K, a, a_scale, stream)) return s;
+    if (int s = w2a8_gemm(a, a_scale, packed, w_scale, y_dev, M, N, K, group, ws, gemm_ws, stream))
+        return s;
+    if (cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return W2A8_ERR_CUDA;
+    return W2A8_OK;
+}
+
+}  // extern "C"

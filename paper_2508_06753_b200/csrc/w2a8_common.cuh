@@ -1,0 +1,99 @@
+// Shared device/host helpers of the W2A8 CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "w2a8.h"
+
+namespace w2a8 {
+
+// ---- W2P layout constants (see w2_pack in w2a8.h) -------------------------
+constexpr int kSliceK = 64;    // k per slice = smallest scale group
+constexpr int kBlockK = 256;   // k per block = four slices
+constexpr int kWordK = 16;     // codes per 32-bit word
+
+// The unpack puts each 2-bit code into the two top bits of an int8 lane:
+//   lane = ((word << (6 - 2 j)) & 0xC0C0C0C0) ^ 0x80808080  =  64 * (code - 2)
+// (offset binary -> two's complement is the XOR of the top bit).  All integer
+// sums therefore carry an exact factor 64 that the epilogue removes.
+constexpr uint32_t kTopMask = 0xC0C0C0C0u;
+constexpr uint32_t kSignFlip = 0x80808080u;
+constexpr int kCodeGain = 64;
+
+// int32 accumulators start at the bit pattern of 1.5 * 2^23; as long as the
+// accumulated integer stays below 2^22 in magnitude, reinterpreting the
+// accumulator as fp32 and subtracting 1.5 * 2^23 converts it exactly, with no
+// integer-to-float instruction.
+constexpr int kMagicInt = 0x4B400000;
+constexpr float kMagicFloat = 12582912.0f;
+
+__device__ __forceinline__ uint32_t lane_codes(uint32_t word, int j) {
+    // j is a compile-time constant after unrolling
+    return (((j == 3) ? word : (word << (6 - 2 * j))) & kTopMask) ^ kSignFlip;
+}
+
+// Programmatic dependent launch: wait until the previous kernel of the stream
+// has completed and its writes are visible / let the next kernel start early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+__device__ __forceinline__ void mma_s8_16x8x32(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// ---- host side --------------------------------------------------------------
+struct ShapeInfo {
+    int slices;        // K / 64
+    int blocks;        // ceil(K / 256)
+    int tail_slices;   // slices in the last block (1..4)
+    int words_per_row; // K / 16
+    int G;             // K / group
+    int spp;           // slices per scale group, capped at 4 (1, 2 or 4)
+};
+
+inline bool shape_ok(int M, int N, int K, int group, ShapeInfo *out) {
+    if (M < 1 || N < 16 || K < 64 || group < 64) return false;
+    if (K % 64 != 0 || N % 16 != 0 || K % group != 0) return false;
+    if (!(group == 64 || group == 128 || group % 256 == 0 || group == K)) return false;
+    if ((long long)M * N >= (1ll << 40)) return false;
+    if (out) {
+        out->slices = K / 64;
+        out->blocks = (K + 255) / 256;
+        out->tail_slices = out->slices - 4 * (out->blocks - 1);
+        out->words_per_row = K / 16;
+        out->G = K / group;
+        out->spp = group == 64 ? 1 : (group == 128 ? 2 : 4);
+    }
+    return true;
+}
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t stream, bool pdl, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+bool pdl_enabled();
+int check_device();  // W2A8_OK or W2A8_ERR_ARCH / W2A8_ERR_CUDA
+
+}  // namespace w2a8

@@ -1,0 +1,98 @@
+"""CPU-side checks of the C-ABI library: it builds, loads without a GPU, exports
+every symbol the header declares, and rejects bad arguments on the host
+before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from conftest import ROOT
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2508_06753_b200 import build, binding
+    build.build()
+    return binding.lib()
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "w2a8.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b([A-Za-z_][A-Za-z0-9_]*)\s*\([^;{}]*\)\s*;", text)
+    return sorted(set(names))
+
+
+def test_header_declares_expected_entry_points():
+    names = _declared_functions()
+    for must in ("w2_pack", "a8_quantize", "w2a8_gemm", "w2a8_gemm_partials", "w2a8_linear_host"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in _declared_functions():
+        assert hasattr(lib, name), name
+
+
+def test_binding_lists_every_declared_symbol():
+    from paper_2508_06753_b200 import binding
+    assert sorted(binding.EXPORTS) == _declared_functions()
+    for name in binding.EXPORTS:
+        assert hasattr(binding, name) or name == "w2a8_status_string"
+
+
+def test_sizes_and_version(lib):
+    assert lib.w2a8_version() >= 100
+    assert lib.w2_packed_bytes(2048, 2048) == 2048 * 2048 // 4
+    assert lib.w2_packed_bytes(16, 1600) == 16 * 1600 // 4
+    assert lib.w2_packed_bytes(15, 64) == 0 and lib.w2_packed_bytes(16, 100) == 0
+    assert lib.w2a8_workspace_bytes(1, 2048, 2048, 64) > 0
+    assert lib.w2a8_workspace_bytes(1, 2048, 2048, 96) == 0      # group not allowed
+    assert lib.w2a8_workspace_bytes(1, 2048, 2048, 192) == 0
+    assert lib.w2a8_workspace_bytes(0, 2048, 2048, 64) == 0
+    assert lib.w2a8_workspace_bytes(4, 4096, 14336, 14336) > 0   # group == K
+    assert lib.w2a8_linear_host_workspace_bytes(4, 4096, 4096, 64) > lib.w2a8_workspace_bytes(4, 4096, 4096, 64)
+
+
+def test_status_strings(lib):
+    seen = set()
+    for code in range(0, -7, -1):
+        s = lib.w2a8_status_string(code).decode()
+        assert s and s != "unknown status"
+        seen.add(s)
+    assert len(seen) == 7
+    assert lib.w2a8_status_string(-99).decode() == "unknown status"
+
+
+def test_argument_errors_are_detected_on_the_host(lib):
+    # no GPU here: every call below must return before touching the device
+    buf = ctypes.create_string_buffer(1 << 16)
+    base = ctypes.addressof(buf)
+    p = (base + 15) // 16 * 16          # 16-byte aligned fake pointer
+    NULLP, SHAPE, ALIGN, WS = -1, -2, -3, -4
+    assert lib.w2_pack(None, 16, 64, p, None) == NULLP
+    assert lib.w2_pack(p, 16, 65, p, None) == SHAPE
+    assert lib.w2_pack(p + 4, 16, 64, p, None) == ALIGN
+    assert lib.a8_quantize(None, 1, 64, p, p, None) == NULLP
+    assert lib.a8_quantize(p, 0, 64, p, p, None) == SHAPE
+    assert lib.a8_quantize(p, 1, 64, p + 1, p, None) == ALIGN
+    assert lib.w2a8_gemm(None, p, p, p, p, 1, 16, 64, 64, p, 1 << 15, None) == NULLP
+    assert lib.w2a8_gemm(p, p, p, p, p, 1, 16, 64, 32, p, 1 << 15, None) == SHAPE
+    assert lib.w2a8_gemm(p, p, p, p, p, 1, 24, 64, 64, p, 1 << 15, None) == SHAPE
+    assert lib.w2a8_gemm(p, p, p + 8, p, p, 1, 16, 64, 64, p, 1 << 15, None) == ALIGN
+    assert lib.w2a8_gemm(p, p, p, p, p, 1, 16, 64, 64, None, 0, None) == WS
+    assert lib.w2a8_gemm(p, p, p, p, p, 1, 16, 64, 64, p, 8, None) == WS
+    assert lib.w2a8_gemm_partials(p, p, None, 1, 16, 64, 64, p, 1 << 15, None) == NULLP
+    assert lib.w2a8_linear_host(None, 1, 64, p, p, 16, 64, p, p, 1 << 15, None) == NULLP
+    assert lib.w2a8_linear_host(p, 1, 64, p, p, 16, 48, p, p, 1 << 15, None) == SHAPE
+    assert lib.w2a8_linear_host(p, 1, 64, p, p, 16, 64, p, p, 16, None) == WS
+    assert lib.w2a8_workspace_init(None, 16, None) == NULLP
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    from paper_2508_06753_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(FileNotFoundError):
+        binding.lib()

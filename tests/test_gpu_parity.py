@@ -1,0 +1,290 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU
+reference on the same seeded inputs.  Bit-exact for packed weights, int8
+activations, activation scales and int32 per-group sums; fp32 outputs within
+1e-4 * max|row| (the tolerance of the target statement)."""
+import os
+
+import numpy as np
+import pytest
+
+from paper_2508_06753_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2508_06753_b200 import binding, build
+    build.build()
+    binding.lib()
+    return torch, binding
+
+
+def _dev(torch, arr):
+    return torch.from_numpy(np.ascontiguousarray(arr)).cuda()
+
+
+def _bf16_dev(torch, bits):
+    return _dev(torch, bits.view(np.int16)).view(torch.bfloat16)
+
+
+def _row_err_ok(y, y_ref):
+    err = np.abs(y.astype(np.float64) - y_ref.astype(np.float64)).max(axis=1)
+    bound = TOL * np.abs(y_ref).max(axis=1)
+    return (err <= bound).all(), float((err / np.maximum(bound, 1e-30)).max())
+
+
+# ------------------------------------------------------------------- pack
+@pytest.mark.parametrize("N,K", [(16, 64), (16, 256), (32, 448), (48, 1600), (2048, 2048),
+                                 (1024, 4096), (16, 28672), (4096, 14336)])
+def test_pack_bit_exact(gpu, oracle, N, K):
+    torch, b = gpu
+    codes = synth.weight_codes(N + K, N, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    torch.cuda.synchronize()
+    got = packed.cpu().numpy().view(np.uint32)
+    assert got.nbytes == N * K // 4 == b.w2_packed_bytes(N, K)
+    assert np.array_equal(got, oracle.pack(codes))
+
+
+def test_pack_masks_high_bits(gpu, oracle):
+    torch, b = gpu
+    rng = np.random.default_rng(1)
+    codes = rng.integers(0, 256, size=(32, 512), dtype=np.uint8)
+    got = b.w2_pack(_dev(torch, codes)).cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, oracle.pack(codes & 3))
+
+
+# --------------------------------------------------------------- quantiser
+@pytest.mark.parametrize("M,K,frac", [(1, 64, 0.0), (1, 2048, 0.0), (4, 4096, 0.0), (16, 14336, 0.0),
+                                      (8, 8192, 0.01), (32, 28672, 0.01), (3, 1600, 0.0),
+                                      (300, 4096, 0.0)])
+def test_quantize_bit_exact(gpu, oracle, M, K, frac):
+    torch, b = gpu
+    bits = synth.activations_bf16(M * 7 + K, M, K, frac)
+    a, s = b.a8_quantize(_bf16_dev(torch, bits))
+    torch.cuda.synchronize()
+    a_ref, s_ref = oracle.quantize(bits)
+    assert np.array_equal(a.cpu().numpy(), a_ref)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+
+
+def test_quantize_all_bf16_patterns(gpu, oracle):
+    torch, b = gpu
+    allb = np.arange(1 << 16, dtype=np.uint32)
+    finite = allb[((allb >> 7) & 0xFF) != 0xFF].astype(np.uint16)
+    rows = []
+    for amax_bits in (0x3F80, 0x4040, 0x4088, 0x41A0, 0x42FE, 0x3580, 0x5DC0, 0x0080, 0x0001, 0x7F7F):
+        keep = finite[(finite & 0x7FFF) <= amax_bits]
+        row = np.zeros(65536, dtype=np.uint16)
+        row[:keep.size] = keep
+        row[keep.size] = amax_bits
+        rows.append(row)
+    bits = np.stack(rows)
+    a, s = b.a8_quantize(_bf16_dev(torch, bits))
+    a_ref, s_ref = oracle.quantize(bits)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(a.cpu().numpy(), a_ref)
+
+
+def test_quantize_degenerate_rows(gpu, oracle):
+    torch, b = gpu
+    bits = synth.activations_bf16(3, 4, 256)
+    bits[1, :] = 0
+    bits[1, 7] = 0x8000
+    bits[2, :] = 0
+    bits[2, 9] = 0x0003
+    a, s = b.a8_quantize(_bf16_dev(torch, bits))
+    a_ref, s_ref = oracle.quantize(bits)
+    assert np.array_equal(a.cpu().numpy(), a_ref)
+    assert np.array_equal(s.cpu().numpy(), s_ref)
+    assert not a.cpu().numpy()[1:3].any() and s_ref[1] == 0 and s_ref[2] == 0
+
+
+# ------------------------------------------------------- partials / outputs
+def _problem(seed, M, N, K, group, ternary=False, frac=0.0):
+    g = K if group == 0 else group
+    codes, s_w = synth.make_linear(seed, K, N, g, ternary)
+    bits = synth.activations_bf16(seed, M, K, frac)
+    return codes, s_w, bits, g
+
+
+def _run_gpu(torch, b, codes, s_w, bits, g, want_partials=True):
+    M, K = bits.shape
+    N = codes.shape[0]
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_bf16_dev(torch, bits))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
+    y2 = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
+    P = b.w2a8_gemm_partials(a, packed, g, ws) if want_partials else None
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2), "repeated calls must be bitwise equal"
+    return (a.cpu().numpy(), s_a.cpu().numpy(), y.cpu().numpy(),
+            None if P is None else P.cpu().numpy())
+
+
+CASES = [
+    # M, N, K, group (0 = K), ternary, outlier fraction
+    (1, 2048, 2048, 64, False, 0.0),       # configuration 0 in full
+    (1, 16, 64, 64, False, 0.0),           # smallest legal problem
+    (2, 16, 256, 64, False, 0.0),
+    (3, 48, 448, 64, False, 0.0),          # ragged K: trailing block of three slices
+    (1, 1600, 1600, 64, False, 0.0),       # the paper's smallest shape (Sec. III-B)
+    (5, 32, 1600, 0, True, 0.0),           # ragged K, one scale per channel
+    (4, 1040, 4096, 64, False, 0.0),       # N not a multiple of anything but 16
+    (8, 256, 4096, 128, False, 0.01),
+    (9, 256, 2048, 128, False, 0.0),       # two token tiles, ragged
+    (16, 512, 4096, 64, False, 0.0),
+    (17, 128, 1024, 256, False, 0.0),
+    (32, 256, 8192, 128, False, 0.01),
+    (8, 128, 4096, 0, True, 0.0),          # ternary, group = K
+    (1, 64, 14336, 0, True, 0.0),
+    (33, 64, 512, 64, False, 0.0),         # more than one 32-token chunk
+    (70, 48, 768, 128, False, 0.0),
+    (1, 16, 28672, 128, False, 0.01),      # longest K of any configuration
+]
+
+
+@pytest.mark.parametrize("M,N,K,group,ternary,frac", CASES)
+def test_gemm_against_reference(gpu, oracle, M, N, K, group, ternary, frac):
+    torch, b = gpu
+    codes, s_w, bits, g = _problem(M * 31 + N + K, M, N, K, group, ternary, frac)
+    a, s_a, y, P = _run_gpu(torch, b, codes, s_w, bits, g)
+    a_ref, s_ref = oracle.quantize(bits)
+    assert np.array_equal(a, a_ref) and np.array_equal(s_a.view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(P, oracle.partials(a_ref, codes, g)), "int32 per-group sums must be exact"
+    ok, worst = _row_err_ok(y, oracle.gemm(a_ref, s_ref, codes, s_w, g))
+    assert ok, f"worst error / bound = {worst}"
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 7])
+@pytest.mark.parametrize("M", [1, 12])
+def test_forced_split_k(gpu, oracle, splits, M, monkeypatch):
+    torch, b = gpu
+    monkeypatch.setenv("W2A8_SPLITS", str(splits))
+    N, K, g = 64, 14336, 64
+    codes, s_w, bits, g = _problem(99 + splits, M, N, K, g)
+    a, s_a, y, _ = _run_gpu(torch, b, codes, s_w, bits, g, want_partials=False)
+    ok, worst = _row_err_ok(y, oracle.gemm(a, s_a, codes, s_w, g))
+    assert ok, f"worst error / bound = {worst}"
+
+
+def test_extreme_magnitudes_no_overflow(gpu, oracle):
+    torch, b = gpu
+    M, N, K = 2, 16, 28672
+    codes = np.zeros((N, K), np.uint8)                       # value -2 everywhere
+    codes[1::2] = 3                                          # value +1 on odd channels
+    x = np.full((M, K), -3.0, np.float32)                    # quantises to -127
+    x[1] = 3.0
+    bits = synth.float_to_bf16_bits(x)
+    s_w = np.ones((N, 1), np.float32)
+    a, s_a, y, P = _run_gpu(torch, b, codes, s_w, bits, K)
+    assert P[0, 0, 0] == 254 * K and P[1, 0, 0] == -254 * K and P[1, 1, 0] == 127 * K
+    assert np.array_equal(P, oracle.partials(a, codes, K))
+    ok, worst = _row_err_ok(y, oracle.gemm(a, s_a, codes, s_w, K))
+    assert ok, worst
+    for g in (64, 128, 256):                                 # largest sums inside one accumulator
+        s_w = np.ones((N, K // g), np.float32)
+        a, s_a, y, P = _run_gpu(torch, b, codes, s_w, bits, g)
+        assert (P[0, 0] == 254 * g).all()
+        assert np.array_equal(P, oracle.partials(a, codes, g))
+
+
+def test_zero_token_row_and_zero_weights(gpu, oracle):
+    torch, b = gpu
+    M, N, K, g = 4, 32, 512, 64
+    codes, s_w, bits, g = _problem(5, M, N, K, g)
+    bits[2, :] = 0                                           # dead token
+    codes[3, :] = 2                                          # channel of zeros
+    a, s_a, y, P = _run_gpu(torch, b, codes, s_w, bits, g)
+    assert not y[2].any() and not y[:, 3].any()
+    ok, worst = _row_err_ok(y, oracle.gemm(a, s_a, codes, s_w, g))
+    assert ok, worst
+
+
+def test_linear_host_end_to_end(gpu, oracle):
+    torch, b = gpu
+    M, N, K, g = 4, 1024, 4096, 64
+    codes, s_w, bits, g = _problem(77, M, N, K, g)
+    packed = b.w2_pack(_dev(torch, codes))
+    s_w_d = _dev(torch, s_w)
+    x_host = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    y_host = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    ws = b.new_workspace(b.w2a8_linear_host_workspace_bytes(M, N, K, g))
+    for _ in range(2):
+        y_host.zero_()
+        b.w2a8_linear_host(x_host, packed, s_w_d, g, y_host, ws)
+        torch.cuda.synchronize()
+        a_ref, s_ref = oracle.quantize(bits)
+        ok, worst = _row_err_ok(y_host.numpy(), oracle.gemm(a_ref, s_ref, codes, s_w, g))
+        assert ok, worst
+
+
+def test_pdl_off_matches(gpu, oracle):
+    # the same library with plain launches, in a child process (the switch is read once)
+    import subprocess
+    import sys
+    code = (
+        "import numpy as np, torch\n"
+        "from paper_2508_06753_b200 import binding as b, synth\n"
+        "import oracle\n"
+        "codes, s_w = synth.make_linear(3, 2048, 256, 64)\n"
+        "bits = synth.activations_bf16(3, 4, 2048)\n"
+        "d = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()\n"
+        "packed = b.w2_pack(d(codes)); a, s = b.a8_quantize(d(bits.view(np.int16)).view(torch.bfloat16))\n"
+        "ws = b.new_workspace(b.w2a8_workspace_bytes(4, 256, 2048, 64))\n"
+        "y = b.w2a8_gemm(a, s, packed, d(s_w), 64, ws).cpu().numpy()\n"
+        "a_ref, s_ref = oracle.quantize(bits)\n"
+        "ref = oracle.gemm(a_ref, s_ref, codes, s_w, 64)\n"
+        "assert np.abs(y - ref).max() <= 1e-4 * np.abs(ref).max(), 'mismatch'\n"
+        "print('ok')\n")
+    env = dict(os.environ, W2A8_PDL="0")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
+
+
+# ---------------------------------------------- full-size shapes, sampled channels
+FULL = [
+    (1, "8b"), (16, "8b"), (8, "8b-ternary"), (32, "70b"),
+]
+
+
+@pytest.mark.parametrize("M,which", FULL)
+def test_full_size_layers_sampled(gpu, oracle, M, which):
+    """Every linear of a layer at full size, in the launch configuration the
+    benchmark times; the reference is evaluated on 96 sampled output channels
+    (channels are independent) plus the first and last 16."""
+    torch, b = gpu
+    cfg = {"8b": synth.CONFIGS[1], "8b-ternary": synth.CONFIGS[2], "70b": synth.CONFIGS[3]}[which]
+    rng = np.random.default_rng(17)
+    for idx, (name, K, N) in enumerate(cfg["shapes"]):
+        if name in ("v", "up", "o"):                       # same shapes as k, gate, q
+            continue
+        g = synth.config_group(cfg, K)
+        codes, s_w = synth.make_linear(synth.shape_seed(cfg, idx), K, N, g, cfg["ternary"])
+        bits = synth.activations_bf16(synth.shape_seed(cfg, idx), M, K, cfg["outlier_frac"])
+        packed = b.w2_pack(_dev(torch, codes))
+        a, s_a = b.a8_quantize(_bf16_dev(torch, bits))
+        ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+        y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws).cpu().numpy()
+        P = b.w2a8_gemm_partials(a, packed, g, ws).cpu().numpy()
+        sel = np.unique(np.concatenate([np.arange(16), np.arange(N - 16, N),
+                                        rng.choice(N, size=96, replace=False)]))
+        a_ref, s_ref = oracle.quantize(bits)
+        assert np.array_equal(a.cpu().numpy(), a_ref)
+        assert np.array_equal(P[:, sel], oracle.partials(a_ref, codes[sel], g)), name
+        y_ref = oracle.gemm(a_ref, s_ref, codes[sel], s_w[sel], g)
+        err = np.abs(y[:, sel].astype(np.float64) - y_ref).max(axis=1)
+        assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), name
+        # properties that hold for every channel: finite, and bounded by sum |s_w| * 254 g * s_a
+        assert np.isfinite(y).all()
+        bound = (np.abs(s_w).sum(axis=1) * 254.0 * g)[None, :] * s_ref[:, None]
+        assert (np.abs(y) <= bound * (1 + 1e-5)).all()
+        del packed, codes
