@@ -162,7 +162,7 @@ def test_gemm_against_reference(gpu, oracle, M, N, K, group, ternary, frac):
     assert ok, f"worst error / bound = {worst}"
 
 
-@pytest.mark.parametrize("splits", [1, 2, 3, 7])
+@pytest.mark.parametrize("splits", [1, 8, 9, 14, 56])
 @pytest.mark.parametrize("M", [1, 12])
 def test_forced_split_k(gpu, oracle, splits, M, monkeypatch):
     torch, b = gpu
