@@ -525,6 +525,43 @@ def run_ours(args):
     print(json.dumps(out))
 
 
+def run_kernel_profile(args):
+    """Small stand-alone run of one GEMM shape for profilers: a few direct
+    launches of w2a8_gemm over rotating weight copies (total > 2x L2, a few
+    hundred MB), timed with CUDA events.  Prints one JSON line."""
+    import torch
+    from paper_2508_06753_b200 import binding as b, build
+    build.build()
+    K, N = (int(v) for v in args.profile_shape.split("x"))
+    M, g = args.profile_m, (args.profile_group or K)
+    dev = torch.device("cuda", 0)
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    per = K * N // 4 + (K // g) * N * 4
+    copies = max(2, int(np.ceil(2.0 * l2 / per)))
+    mats = []
+    for c in range(copies):
+        codes, s_w = synth.make_linear(7000 + c, K, N, g)
+        mats.append((b.w2_pack(torch.from_numpy(codes).to(dev)), torch.from_numpy(s_w).to(dev)))
+    x = torch.from_numpy(synth.activations_bf16(7, M, K).view(np.int16)).to(dev).view(torch.bfloat16)
+    a, s_a = b.a8_quantize(x)
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g), device=dev)
+    y = torch.empty((M, N), dtype=torch.float32, device=dev)
+    for i in range(args.profile_reps):                      # warm-up
+        b.w2a8_gemm(a, s_a, mats[i % copies][0], mats[i % copies][1], g, ws, y)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.profile_reps):
+        b.w2a8_gemm(a, s_a, mats[i % copies][0], mats[i % copies][1], g, ws, y)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / args.profile_reps
+    print(json.dumps({"profile_shape": f"{K}x{N}", "M": M, "group": g, "copies": copies,
+                      "launches": 2 * args.profile_reps, "us_per_launch_direct": us,
+                      "bytes_per_launch": gemm_bytes(M, N, K, g),
+                      "gbs": gemm_bytes(M, N, K, g) / us / 1e3}))
+
+
 def time_steps_local(torch, runners, steps, warmup):
     for i in range(warmup):
         runners[i % len(runners)]()
@@ -546,7 +583,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-shape", default=None, help="KxN: run only a few launches of this GEMM")
+    ap.add_argument("--profile-m", type=int, default=1)
+    ap.add_argument("--profile-group", type=int, default=64)
+    ap.add_argument("--profile-reps", type=int, default=10)
     args = ap.parse_args()
+    if args.profile_shape:
+        run_kernel_profile(args)
+        return
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)

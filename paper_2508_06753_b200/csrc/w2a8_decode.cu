@@ -3,19 +3,23 @@
 // MMAs (mma.sync m16n8k32) whose A operand is a 16-channel x 32-k weight tile
 // and whose B operand is 32 k x 8 tokens.  The up-convert-and-compute idea is
 // that of Sec. II-C, the K-splitting that of Sec. II-D; the thread/tile mapping
-// and the asynchronous staging are specific to sm_100a.
+// and the launch overlap are specific to sm_100a.
 //
-// Work split: a CTA of 4 warps owns 64 output channels (one 16-channel tile per
-// warp) and one chunk of up to 8 consecutive 256-k blocks; grid.y walks the
-// chunks (split-K), grid.z walks 8*MT-token slabs.  A "cell" is one tile x one
-// block: 1 KB of packed weights + its scales.
+// Work split.  A "cell" is one 16-channel tile x one 256-k block: 1 KB of packed
+// weights plus its scales.  A CTA of 8 warps owns TG tiles and one chunk of the
+// contraction; its warps are arranged TG tiles x KS = 8 / TG K-lanes, and the
+// K-lanes take interleaved blocks of the chunk.  The K-lanes of a tile are
+// summed through shared memory in a fixed order; chunks (grid.y, only used when
+// the shape would otherwise leave SMs idle or the activations would not fit in
+// shared memory) are summed through the workspace by the last CTA to arrive,
+// also in a fixed order.  grid.z walks 8*MT-token slabs.
 //
-// Pipeline: every lane posts the cp.async copies of ALL its cells into a
-// lane-private shared-memory FIFO before it waits for the previous kernel of
-// the stream (weights and scales are frozen, only activations depend on it),
-// so the whole chunk is in flight at once and, under programmatic dependent
-// launch, while the previous kernel is still draining.  The activations of the
-// chunk are then staged once per CTA and shared by its four warps.
+// Pipeline.  Each lane keeps the next cell's weights and scales in flight in
+// registers while it computes the current one.  The first cell is requested
+// before the kernel waits for the previous kernel of the stream (weights and
+// scales are frozen; only activations depend on it), so under programmatic
+// dependent launch the weight stream starts while the previous kernel drains.
+// The chunk's activations are staged once per CTA in shared memory.
 //
 // In the W2P layout one 128-bit unit per lane and channel holds word t of each
 // of the four 64-k slices of a block -- exactly what the four lanes of an MMA
@@ -24,13 +28,10 @@
 
 namespace w2a8 {
 
-constexpr int kCellsMax = 8;                   // FIFO depth = cells per chunk
-constexpr int kDecodeWarps = 4;
+constexpr int kDecodeWarps = 8;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kTileGroupRows = 16 * kDecodeWarps;
-constexpr int kFifoWBytes = kCellsMax * 2 * 32 * 16;   // per warp: weights
-constexpr int kFifoSBytes = kCellsMax * 2 * 8 * 16;    // per warp: scales (<= 4 floats / row)
 constexpr int kActPad = 64;                    // row stride = chunk bytes + 64: conflict-free LDS.128
+constexpr int kActSmemMax = 96 * 1024;         // staged activations per CTA
 
 struct DecodeParams {
     const int8_t *a;
@@ -40,96 +41,188 @@ struct DecodeParams {
     float *y;
     int32_t *partials;
     float *ws;            // [chunks][M][N] partial outputs (chunks > 1)
-    unsigned *counters;   // [grid.z][N/16] arrival counters (chunks > 1)
+    unsigned *counters;   // [grid.z][tile groups] arrival counters (chunks > 1)
     int M, N, K, G, group;
     int blocks, tail_slices, words_per_row;
-    int chunks, cells_per_chunk;
+    int chunks, blocks_per_chunk;
     int act_stride;       // bytes per staged token row
+    int vec_ok;           // K % 256 == 0: scale rows can be read as float4 / float2
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+__device__ __forceinline__ uint4 ld_stream_v4(const uint32_t *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
 }
 
-template <int MT, int SPP, bool PARTIALS>
-__global__ void __launch_bounds__(kDecodeThreads)
+// Optional timeline trace (build with -DW2A8_TRACE): every warp records the
+// global timer at a few points of the kernel into a caller-provided buffer.
+#ifdef W2A8_TRACE
+__device__ unsigned long long *g_trace = nullptr;
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long v;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(v));
+    return v;
+}
+#define W2A8_TRACE_POINT(i)                                                                      \
+    do {                                                                                         \
+        if (g_trace && (threadIdx.x & 31) == 0)                                                  \
+            g_trace[((((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) *  \
+                         kDecodeWarps + (threadIdx.x >> 5)) * 8 + (i)] = global_ns();            \
+    } while (0)
+#else
+#define W2A8_TRACE_POINT(i) do { } while (0)
+#endif
+
+template <int SPP>
+struct Cell {
+    uint32_t w[2][4];                 // [channel g / g+8][slice]
+    float sc[2][4 / SPP];             // [channel][scale group inside the block]
+};
+
+template <int SPP, bool PARTIALS>
+__device__ __forceinline__ void load_cell(const DecodeParams &p, Cell<SPP> &c, int n0, int gq,
+                                          int t, int kb) {
+    const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const size_t row = (size_t)(n0 + gq + 8 * r);
+        const uint32_t *wp = p.packed + row * p.words_per_row + 16 * kb;
+        if (R == 4) {
+            const uint4 v = ld_stream_v4(wp + 4 * t);
+            c.w[r][0] = v.x; c.w[r][1] = v.y; c.w[r][2] = v.z; c.w[r][3] = v.w;
+        } else {   // trailing block with fewer slices: words t*R .. t*R+R-1
+#pragma unroll
+            for (int s = 0; s < 4; ++s) c.w[r][s] = (s < R) ? __ldg(wp + t * R + s) : 0u;
+        }
+        if constexpr (PARTIALS) {
+            // the parity export has no scales
+        } else if constexpr (SPP == 1) {
+            const float *sp = p.w_scale + row * p.G + 4 * kb;
+            if (R == 4 && p.vec_ok) {
+                const float4 v = __ldg(reinterpret_cast<const float4 *>(sp));
+                c.sc[r][0] = v.x; c.sc[r][1] = v.y; c.sc[r][2] = v.z; c.sc[r][3] = v.w;
+            } else {
+#pragma unroll
+                for (int s = 0; s < 4; ++s) c.sc[r][s] = (s < R) ? __ldg(sp + s) : 0.f;
+            }
+        } else if constexpr (SPP == 2) {
+            const float *sp = p.w_scale + row * p.G + 2 * kb;
+            if (R == 4 && p.vec_ok) {
+                const float2 v = __ldg(reinterpret_cast<const float2 *>(sp));
+                c.sc[r][0] = v.x; c.sc[r][1] = v.y;
+            } else {
+#pragma unroll
+                for (int s = 0; s < 2; ++s) c.sc[r][s] = (2 * s < R) ? __ldg(sp + s) : 0.f;
+            }
+        } else {
+            c.sc[r][0] = __ldg(p.w_scale + row * p.G + (int)(((long long)kb * kBlockK) / p.group));
+        }
+    }
+}
+
+// One cell: 4 slices x (unpack, 2 MMAs per token slab, promotion at group ends).
+template <int MT, int SPP, bool ONE, bool PARTIALS>
+__device__ __forceinline__ void compute_cell(const DecodeParams &p, const Cell<SPP> &c,
+                                             const unsigned char *const (&brow)[MT], int kcol,
+                                             int kb, int n0, int m0, int gq, int t,
+                                             float (&acc)[MT][4], int (&D)[MT][4]) {
+    const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
+    const int magic[4] = {kMagicInt, kMagicInt, kMagicInt, kMagicInt};
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        if (s < R) {
+            const uint32_t w0 = c.w[0][s], w1 = c.w[1][s];
+            const uint32_t a0 = lane_codes(w0, 0), a1 = lane_codes(w1, 0);
+            const uint32_t a2 = lane_codes(w0, 1), a3 = lane_codes(w1, 1);
+            const uint32_t a4 = lane_codes(w0, 2), a5 = lane_codes(w1, 2);
+            const uint32_t a6 = lane_codes(w0, 3), a7 = lane_codes(w1, 3);
+            const bool first = (s % SPP) == 0;
+            const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const uint4 b = *reinterpret_cast<const uint4 *>(brow[mt] + kcol + s * kSliceK);
+                if (first) mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, magic);
+                else       mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, D[mt]);
+                mma_s8_16x8x32(D[mt], a4, a5, a6, a7, b.z, b.w, D[mt]);
+                if (last) {
+                    if constexpr (PARTIALS) {
+                        const int gi = (SPP == 1) ? 4 * kb + s
+                                     : (SPP == 2) ? 2 * kb + (s >> 1)
+                                                  : (int)(((long long)kb * kBlockK) / p.group);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int mm = m0 + 8 * mt + 2 * t + (i & 1);
+                            const int nn = n0 + gq + 8 * (i >> 1);
+                            if (mm < p.M)
+                                atomicAdd(p.partials + ((size_t)mm * p.N + nn) * p.G + gi,
+                                          (D[mt][i] - kMagicInt) >> 6);
+                        }
+                    } else {
+                        const float s0 = c.sc[0][s / SPP], s1 = c.sc[1][s / SPP];
+                        acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
+                        acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
+                        if constexpr (!ONE) {
+                            acc[mt][1] = fmaf(s0, __int_as_float(D[mt][1]) - kMagicFloat, acc[mt][1]);
+                            acc[mt][3] = fmaf(s1, __int_as_float(D[mt][3]) - kMagicFloat, acc[mt][3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+// MT: 8-token slabs per CTA; SPP: 64-k slices per scale group (capped at 4);
+// TG: tiles per CTA (K-lanes per tile = 8 / TG); ONE: a single token (half of
+// each accumulator quad is dead and is not promoted).
+template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
+__global__ void __launch_bounds__(kDecodeThreads, (MT == 1 ? 4 : (MT == 2 ? 3 : 2)))
 w2a8_decode_kernel(const DecodeParams p) {
+    constexpr int KS = kDecodeWarps / TG;
     extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, t = lane & 3;
-    const int tile = blockIdx.x * kDecodeWarps + warp;
+    const int tl = warp % TG, ks = warp / TG;
+    const int tile = blockIdx.x * TG + tl;
     const bool tile_ok = tile * 16 < p.N;
     const int n0 = tile * 16;
     const int chunk = blockIdx.y;
-    const int kb0 = chunk * p.cells_per_chunk;
-    const int ncells = min(p.cells_per_chunk, p.blocks - kb0);
+    const int kb_begin = chunk * p.blocks_per_chunk;
+    const int kb_end = min(kb_begin + p.blocks_per_chunk, p.blocks);
     const int m0 = blockIdx.z * (8 * MT);
     const int mrows = min(8 * MT, p.M - m0);
+    W2A8_TRACE_POINT(0);
 
-    unsigned char *fifo_w = smem + warp * (kFifoWBytes + kFifoSBytes);
-    unsigned char *fifo_s = fifo_w + kFifoWBytes;
-    unsigned char *acts = smem + kDecodeWarps * (kFifoWBytes + kFifoSBytes);
-    constexpr int SPB = 4 / SPP;               // scales per block and channel
-
-    // ---- post every cell of the chunk (independent of the previous kernel) ----
-#pragma unroll
-    for (int c = 0; c < kCellsMax; ++c) {
-        if (tile_ok && c < ncells) {
-            const int kb = kb0 + c;
-            const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const size_t row = (size_t)(n0 + gq + 8 * r);
-                const uint32_t *wp = p.packed + row * p.words_per_row + 16 * kb;
-                unsigned char *dst = fifo_w + ((c * 2 + r) * 32 + lane) * 16;
-                if (R == 4) {
-                    cp_async16(smem_u32(dst), wp + 4 * t);
-                } else {   // trailing block with fewer slices: words t*R .. t*R+R-1
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    v.x = __ldg(wp + t * R);
-                    if (R > 1) v.y = __ldg(wp + t * R + 1);
-                    if (R > 2) v.z = __ldg(wp + t * R + 2);
-                    *reinterpret_cast<uint4 *>(dst) = v;
-                }
-                // scales of this block: lane t brings scale t of channel row (the parity
-                // export has no scales: w_scale is null there)
-                const int nsc = (SPP == 4) ? 1 : (R + SPP - 1) / SPP;
-                const float *sp = (SPP == 4)
-                    ? p.w_scale + row * p.G + (int)(((long long)kb * kBlockK) / p.group)
-                    : p.w_scale + row * p.G + SPB * kb;
-                if (!PARTIALS && t < nsc) cp_async4(smem_u32(fifo_s + ((c * 2 + r) * 8 + gq) * 16 + 4 * t), sp + t);
-            }
-        }
-        cp_async_commit();
-    }
+    // ---- request the first cell (independent of the previous kernel) ----------
+    int kb = kb_begin + ks;
+    Cell<SPP> cA, cB;
+    if (tile_ok && kb < kb_end) load_cell<SPP, PARTIALS>(p, cA, n0, gq, t, kb);
+    W2A8_TRACE_POINT(1);
     pdl_launch_dependents();
     pdl_wait();
+    W2A8_TRACE_POINT(2);
 
-    // ---- stage the activations of this chunk: [mrows][ncells * 256 (+pad)] ----
+    // ---- stage the activations of this chunk: [mrows + 1][chunk k (+pad)]; the
+    //      extra row is zeros and stands in for tokens beyond M --------------------
+    unsigned char *acts = smem;
     {
-        const int row_units = ncells * (kBlockK / 16);
-        const int klen = min(ncells * kBlockK, p.K - kb0 * kBlockK);   // trailing block may be short
-        for (int u = threadIdx.x; u < mrows * row_units; u += kDecodeThreads) {
+        const int row_units = (kb_end - kb_begin) * (kBlockK / 16);
+        const int klen = min((kb_end - kb_begin) * kBlockK, p.K - kb_begin * kBlockK);
+        for (int u = threadIdx.x; u < (mrows + 1) * row_units; u += kDecodeThreads) {
             const int r = u / row_units, cu = u % row_units;
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (cu * 16 < klen)
-                v = *reinterpret_cast<const uint4 *>(p.a + (size_t)(m0 + r) * p.K + (size_t)kb0 * kBlockK + cu * 16);
+            if (r < mrows && cu * 16 < klen)
+                v = *reinterpret_cast<const uint4 *>(p.a + (size_t)(m0 + r) * p.K +
+                                                     (size_t)kb_begin * kBlockK + cu * 16);
             *reinterpret_cast<uint4 *>(acts + r * p.act_stride + cu * 16) = v;
         }
     }
     __syncthreads();
-    if (!tile_ok) return;
+    W2A8_TRACE_POINT(3);
 
     float acc[MT][4];
     int D[MT][4];
@@ -138,196 +231,181 @@ w2a8_decode_kernel(const DecodeParams p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) { acc[mt][i] = 0.f; D[mt][i] = kMagicInt; }
 
+    if (tile_ok) {
+        const unsigned char *brow[MT];   // this lane's token row of each slab (or the zero row)
 #pragma unroll
-    for (int c = 0; c < kCellsMax; ++c) {
-        if (c < ncells) {
-            switch (c) {   // groups are committed in cell order
-                case 0: cp_async_wait<kCellsMax - 1>(); break;
-                case 1: cp_async_wait<kCellsMax - 2>(); break;
-                case 2: cp_async_wait<kCellsMax - 3>(); break;
-                case 3: cp_async_wait<kCellsMax - 4>(); break;
-                case 4: cp_async_wait<kCellsMax - 5>(); break;
-                case 5: cp_async_wait<kCellsMax - 6>(); break;
-                case 6: cp_async_wait<kCellsMax - 7>(); break;
-                default: cp_async_wait<0>(); break;
-            }
-            __syncwarp();   // scales were brought by the other lanes of the quad
-            const int kb = kb0 + c;
-            const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
-            const uint4 wa = *reinterpret_cast<const uint4 *>(fifo_w + ((c * 2 + 0) * 32 + lane) * 16);
-            const uint4 wb = *reinterpret_cast<const uint4 *>(fifo_w + ((c * 2 + 1) * 32 + lane) * 16);
-            const float4 sa = *reinterpret_cast<const float4 *>(fifo_s + ((c * 2 + 0) * 8 + gq) * 16);
-            const float4 sb = *reinterpret_cast<const float4 *>(fifo_s + ((c * 2 + 1) * 8 + gq) * 16);
-            const uint32_t w0s[4] = {wa.x, wa.y, wa.z, wa.w};
-            const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
-            const float s0s[4] = {sa.x, sa.y, sa.z, sa.w};
-            const float s1s[4] = {sb.x, sb.y, sb.z, sb.w};
-#pragma unroll
-            for (int s = 0; s < 4; ++s) {
-                if (s < R) {
-                    const uint32_t w0 = w0s[s], w1 = w1s[s];
-                    const uint32_t a0 = lane_codes(w0, 0), a1 = lane_codes(w1, 0);
-                    const uint32_t a2 = lane_codes(w0, 1), a3 = lane_codes(w1, 1);
-                    const uint32_t a4 = lane_codes(w0, 2), a5 = lane_codes(w1, 2);
-                    const uint32_t a6 = lane_codes(w0, 3), a7 = lane_codes(w1, 3);
-                    const bool first = (s % SPP) == 0;
-                    const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        uint4 b = make_uint4(0u, 0u, 0u, 0u);
-                        if (8 * mt + gq < mrows)
-                            b = *reinterpret_cast<const uint4 *>(acts + (8 * mt + gq) * p.act_stride +
-                                                                 c * kBlockK + s * kSliceK + t * 16);
-                        if (first) {
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) D[mt][i] = kMagicInt;
-                        }
-                        mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y);
-                        mma_s8_16x8x32(D[mt], a4, a5, a6, a7, b.z, b.w);
-                        if (last) {
-                            if constexpr (PARTIALS) {
-                                const int gi = (SPP == 1) ? 4 * kb + s
-                                             : (SPP == 2) ? 2 * kb + (s >> 1)
-                                                          : (int)(((long long)kb * kBlockK) / p.group);
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    const int mm = m0 + 8 * mt + 2 * t + (i & 1);
-                                    const int nn = n0 + gq + 8 * (i >> 1);
-                                    if (mm < p.M)
-                                        atomicAdd(p.partials + ((size_t)mm * p.N + nn) * p.G + gi,
-                                                  (D[mt][i] - kMagicInt) >> 6);
-                                }
-                            } else {
-                                const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
-                                acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
-                                acc[mt][1] = fmaf(s0, __int_as_float(D[mt][1]) - kMagicFloat, acc[mt][1]);
-                                acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
-                                acc[mt][3] = fmaf(s1, __int_as_float(D[mt][3]) - kMagicFloat, acc[mt][3]);
-                            }
-                        }
-                    }
-                }
-            }
+        for (int mt = 0; mt < MT; ++mt)
+            brow[mt] = acts + ((8 * mt + gq < mrows) ? (8 * mt + gq) : mrows) * p.act_stride + t * 16;
+        // two cells in flight, alternating register sets
+        while (kb < kb_end) {
+            const int kb1 = kb + KS;
+            if (kb1 < kb_end) load_cell<SPP, PARTIALS>(p, cB, n0, gq, t, kb1);
+            compute_cell<MT, SPP, ONE, PARTIALS>(p, cA, brow, (kb - kb_begin) * kBlockK, kb, n0, m0,
+                                                 gq, t, acc, D);
+            if (kb1 >= kb_end) break;
+            const int kb2 = kb1 + KS;
+            if (kb2 < kb_end) load_cell<SPP, PARTIALS>(p, cA, n0, gq, t, kb2);
+            compute_cell<MT, SPP, ONE, PARTIALS>(p, cB, brow, (kb1 - kb_begin) * kBlockK, kb1, n0,
+                                                 m0, gq, t, acc, D);
+            kb = kb2;
         }
     }
+    W2A8_TRACE_POINT(5);
 
     if constexpr (!PARTIALS) {
+        // ---- sum the K-lanes of each tile in a fixed order -----------------------
         // lane (gq, t) holds channels n0+gq, n0+gq+8 for tokens 2t, 2t+1 of each slab
-        if (p.chunks == 1) {
+        float *red = reinterpret_cast<float *>(smem);   // [KS][TG][MT*4][32], reuses the staging area
+        __syncthreads();   // everyone is done reading the staged activations
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
+        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int mm = m0 + 8 * mt + 2 * t + (i & 1);
-                    const int nn = n0 + gq + 8 * (i >> 1);
-                    if (mm < p.M)
-                        p.y[(size_t)mm * p.N + nn] = acc[mt][i] * (p.a_scale[mm] * (1.0f / kCodeGain));
-                }
-            return;
-        }
-        // split-K: park the partial outputs; the last warp to arrive for this tile
-        // and slab sums all chunks in chunk order (repeatable to the bit).
+            for (int i = 0; i < 4; ++i)
+                red[((ks * TG + tl) * (MT * 4) + mt * 4 + i) * 32 + lane] = acc[mt][i];
+        __syncthreads();
         const size_t MN = (size_t)p.M * p.N;
+        // element e of the CTA: (tile etl, slab mt, quad register i, lane el)
+        for (int e = threadIdx.x; e < TG * MT * 128; e += kDecodeThreads) {
+            const int el = e & 31, ei = (e >> 5) % (MT * 4), etl = e / (MT * 128);
+            const int mt = ei >> 2, i = ei & 3;
+            float v = 0.f;
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int mm = m0 + 8 * mt + 2 * t + (i & 1);
-                const int nn = n0 + gq + 8 * (i >> 1);
-                if (mm < p.M) __stcg(p.ws + chunk * MN + (size_t)mm * p.N + nn, acc[mt][i]);
+            for (int k2 = 0; k2 < KS; ++k2) v += red[((k2 * TG + etl) * (MT * 4) + ei) * 32 + el];
+            const int mm = m0 + 8 * mt + 2 * (el & 3) + (i & 1);
+            const int nn = (blockIdx.x * TG + etl) * 16 + (el >> 2) + 8 * (i >> 1);
+            if (mm < p.M && nn < p.N) {
+                if (p.chunks == 1) p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
+                else __stcg(p.ws + chunk * MN + (size_t)mm * p.N + nn, v);
             }
+        }
+        W2A8_TRACE_POINT(6);
+        if (p.chunks == 1) return;
+
+        // ---- split-K: the last CTA to arrive sums the partial outputs in order ---
         __threadfence();
-        __syncwarp();
-        unsigned *counter = p.counters + (size_t)blockIdx.z * (p.N / 16) + tile;
-        unsigned ticket = 0;
-        if (lane == 0) ticket = atomicAdd(counter, 1u);
-        ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
-        if (ticket != (unsigned)p.chunks - 1u) return;
+        __syncthreads();
+        unsigned *counter = p.counters + (size_t)blockIdx.z * gridDim.x + blockIdx.x;
+        if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) == (unsigned)p.chunks - 1u);
+        __syncthreads();
+        if (!is_last) return;
         __threadfence();
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int mm = m0 + 8 * mt + 2 * t + (i & 1);
-                const int nn = n0 + gq + 8 * (i >> 1);
-                if (mm < p.M) {
-                    float v = 0.f;
-                    for (int ch = 0; ch < p.chunks; ++ch) v += __ldcg(p.ws + ch * MN + (size_t)mm * p.N + nn);
-                    p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
-                }
+        for (int e = threadIdx.x; e < TG * MT * 128; e += kDecodeThreads) {
+            const int el = e & 31, ei = (e >> 5) % (MT * 4), etl = e / (MT * 128);
+            const int mt = ei >> 2, i = ei & 3;
+            const int mm = m0 + 8 * mt + 2 * (el & 3) + (i & 1);
+            const int nn = (blockIdx.x * TG + etl) * 16 + (el >> 2) + 8 * (i >> 1);
+            if (mm < p.M && nn < p.N) {
+                float v = 0.f;
+                for (int ch = 0; ch < p.chunks; ++ch) v += __ldcg(p.ws + ch * MN + (size_t)mm * p.N + nn);
+                p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
             }
-        if (lane == 0) *counter = 0u;   // leave the workspace reusable
+        }
+        if (threadIdx.x == 0) *counter = 0u;   // leave the workspace reusable
+        W2A8_TRACE_POINT(7);
     }
 }
+
+#ifdef W2A8_TRACE
+extern "C" int w2a8_debug_set_trace(void *buffer) {
+    unsigned long long *b = reinterpret_cast<unsigned long long *>(buffer);
+    return cudaMemcpyToSymbol(g_trace, &b, sizeof(b)) == cudaSuccess ? 0 : W2A8_ERR_CUDA;
+}
+#endif
 
 // ---- host side -----------------------------------------------------------------
 int env_int(const char *name, int dflt);
 
-// Number of K-chunks (grid.y).  At least ceil(blocks / 8) because a chunk holds at
-// most 8 blocks; more when the grid would otherwise leave SMs idle.
-int decode_chunks(int M, int N, const ShapeInfo &si) {
-    const int min_chunks = (si.blocks + kCellsMax - 1) / kCellsMax;
-    const int forced = env_int("W2A8_SPLITS", 0);
-    int c;
-    if (forced > 0) {
-        c = forced;
-    } else {
-        const int groups = (N + kTileGroupRows - 1) / kTileGroupRows;
-        const int slabs = M > 32 ? (M + 31) / 32 : 1;
-        c = (296 + groups * slabs - 1) / (groups * slabs);
-    }
-    if (c < min_chunks) c = min_chunks;
-    if (c > si.blocks) c = si.blocks;
-    // equalise: the smallest chunk count that gives the same cells per chunk
-    const int cells = (si.blocks + c - 1) / c;
-    return (si.blocks + cells - 1) / cells;
-}
-
 static inline int decode_mt(int M) { return M > 32 ? 4 : (M + 7) / 8; }
 
+struct DecodePlan {
+    int mt, tg, chunks, blocks_per_chunk, slabs, groups;
+    size_t smem;
+};
+
+// Tiles per CTA and K-chunks.  One tile per CTA (8 K-lanes) keeps each warp's
+// serial work shortest; several tiles per CTA share the staged activations,
+// which matters once there are many tokens.  Chunks are added when the staged
+// activations would not fit, or when the grid would leave most SMs idle.
+static DecodePlan decode_plan(int M, int N, const ShapeInfo &si) {
+    DecodePlan pl;
+    pl.mt = decode_mt(M);
+    pl.slabs = (M + 8 * pl.mt - 1) / (8 * pl.mt);
+    const int forced_tg = env_int("W2A8_TG", 0);
+    pl.tg = (forced_tg == 1 || forced_tg == 2 || forced_tg == 4 || forced_tg == 8)
+                ? forced_tg : (pl.mt == 1 ? 1 : (pl.mt == 2 ? 2 : 4));
+    pl.groups = (N / 16 + pl.tg - 1) / pl.tg;
+    const int mrows = M < 8 * pl.mt ? M : 8 * pl.mt;
+    int max_blocks = (kActSmemMax / (mrows + 1) - kActPad) / kBlockK;    // activations must fit
+    if (max_blocks < 1) max_blocks = 1;
+    int chunks = (si.blocks + max_blocks - 1) / max_blocks;
+    const int ks = kDecodeWarps / pl.tg;
+    const int forced = env_int("W2A8_CHUNKS", 0);
+    if (forced > 0) {
+        if (forced > chunks) chunks = forced;
+    } else {
+        // fewer than ~2 CTAs per SM: split K further while each K-lane keeps >= 1 block
+        while ((long long)pl.groups * pl.slabs * chunks < 296 && (si.blocks / (chunks * 2)) >= ks)
+            chunks *= 2;
+    }
+    if (chunks > si.blocks) chunks = si.blocks;
+    pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
+    pl.chunks = (si.blocks + pl.blocks_per_chunk - 1) / pl.blocks_per_chunk;
+    const size_t act = (size_t)(mrows + 1) * (pl.blocks_per_chunk * kBlockK + kActPad);
+    const size_t red = (size_t)kDecodeWarps * pl.mt * 4 * 32 * sizeof(float);
+    pl.smem = act > red ? act : red;
+    return pl;
+}
+
 size_t decode_workspace_bytes(int M, int N, const ShapeInfo &si) {
-    const int mt = decode_mt(M);
-    const int slabs = (M + 8 * mt - 1) / (8 * mt);
-    size_t counters = ((size_t)4 * (N / 16) * slabs + 255) / 256 * 256;
-    // room for one partial output per block of K: covers every chunk count
-    size_t part = (size_t)si.blocks * M * N * sizeof(float);
-    const int chunks = decode_chunks(M, N, si);
-    if (env_int("W2A8_SPLITS", 0) <= 0) part = (size_t)(chunks > 1 ? chunks : 0) * M * N * sizeof(float);
+    const DecodePlan pl = decode_plan(M, N, si);
+    size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;   // >= any tile grouping
+    // with an environment override in force, size for the finest split
+    const int chunks = (env_int("W2A8_CHUNKS", 0) > 0 || env_int("W2A8_TG", 0) > 0) ? si.blocks : pl.chunks;
+    size_t part = (size_t)(chunks > 1 ? chunks : 0) * M * N * sizeof(float);
     return counters + part;
 }
 
-template <int MT, int SPP, bool PARTIALS>
+template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
 static cudaError_t launch_decode_inst(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
     static bool configured = false;   // one attribute call per instantiation and process
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, PARTIALS>,
+        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, TG, ONE, PARTIALS>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return launch_kernel(w2a8_decode_kernel<MT, SPP, PARTIALS>, grid, dim3(kDecodeThreads), smem, st,
-                         pdl_enabled(), p);
+    return launch_kernel(w2a8_decode_kernel<MT, SPP, TG, ONE, PARTIALS>, grid, dim3(kDecodeThreads),
+                         smem, st, pdl_enabled(), p);
+}
+
+template <int MT, int SPP, int TG>
+static cudaError_t launch_decode_tg(const DecodeParams &p, bool want_partials, dim3 grid, size_t smem,
+                                    cudaStream_t st) {
+    if (want_partials) return launch_decode_inst<MT, SPP, TG, false, true>(p, grid, smem, st);
+    if (MT == 1 && p.M == 1) return launch_decode_inst<1, SPP, TG, true, false>(p, grid, smem, st);
+    return launch_decode_inst<MT, SPP, TG, false, false>(p, grid, smem, st);
 }
 
 template <int MT, int SPP>
-static cudaError_t launch_decode_mt(const DecodeParams &p, bool want_partials, dim3 grid, size_t smem,
+static cudaError_t launch_decode_mt(const DecodeParams &p, const DecodePlan &pl, bool want_partials,
                                     cudaStream_t st) {
-    return want_partials ? launch_decode_inst<MT, SPP, true>(p, grid, smem, st)
-                         : launch_decode_inst<MT, SPP, false>(p, grid, smem, st);
+    dim3 grid(pl.groups, pl.chunks, pl.slabs);
+    switch (pl.tg) {
+        case 1: return launch_decode_tg<MT, SPP, 1>(p, want_partials, grid, pl.smem, st);
+        case 2: return launch_decode_tg<MT, SPP, 2>(p, want_partials, grid, pl.smem, st);
+        case 4: return launch_decode_tg<MT, SPP, 4>(p, want_partials, grid, pl.smem, st);
+        default: return launch_decode_tg<MT, SPP, 8>(p, want_partials, grid, pl.smem, st);
+    }
 }
 
 template <int SPP>
-static cudaError_t launch_decode_spp(DecodeParams &p, bool want_partials, cudaStream_t st) {
-    const int mt = decode_mt(p.M);
-    const int mrows = p.M < 8 * mt ? p.M : 8 * mt;
-    p.act_stride = p.cells_per_chunk * kBlockK + kActPad;
-    const size_t smem = (size_t)kDecodeWarps * (kFifoWBytes + kFifoSBytes) + (size_t)mrows * p.act_stride;
-    dim3 grid((p.N + kTileGroupRows - 1) / kTileGroupRows, p.chunks, (p.M + 8 * mt - 1) / (8 * mt));
-    switch (mt) {
-        case 1: return launch_decode_mt<1, SPP>(p, want_partials, grid, smem, st);
-        case 2: return launch_decode_mt<2, SPP>(p, want_partials, grid, smem, st);
-        case 3: return launch_decode_mt<3, SPP>(p, want_partials, grid, smem, st);
-        default: return launch_decode_mt<4, SPP>(p, want_partials, grid, smem, st);
+static cudaError_t launch_decode_spp(const DecodeParams &p, const DecodePlan &pl, bool want_partials,
+                                     cudaStream_t st) {
+    switch (pl.mt) {
+        case 1: return launch_decode_mt<1, SPP>(p, pl, want_partials, st);
+        case 2: return launch_decode_mt<2, SPP>(p, pl, want_partials, st);
+        case 3: return launch_decode_mt<3, SPP>(p, pl, want_partials, st);
+        default: return launch_decode_mt<4, SPP>(p, pl, want_partials, st);
     }
 }
 
@@ -335,16 +413,16 @@ static cudaError_t launch_decode_spp(DecodeParams &p, bool want_partials, cudaSt
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st) {
+    const DecodePlan pl = decode_plan(M, N, si);
     DecodeParams p;
     p.a = a; p.a_scale = a_scale; p.packed = packed; p.w_scale = w_scale;
     p.y = y; p.partials = partials;
     p.M = M; p.N = N; p.K = K; p.G = si.G; p.group = group;
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
-    p.chunks = decode_chunks(M, N, si);
-    p.cells_per_chunk = (si.blocks + p.chunks - 1) / p.chunks;
-    const int mt = decode_mt(M);
-    const int slabs = (M + 8 * mt - 1) / (8 * mt);
-    size_t counters = ((size_t)4 * (N / 16) * slabs + 255) / 256 * 256;
+    p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;
+    p.act_stride = pl.blocks_per_chunk * kBlockK + kActPad;
+    p.vec_ok = (K % 256 == 0) ? 1 : 0;
+    size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
     p.counters = reinterpret_cast<unsigned *>(workspace);
     p.ws = reinterpret_cast<float *>(reinterpret_cast<char *>(workspace) + counters);
     if (partials) {
@@ -352,9 +430,9 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
         if (cudaMemsetAsync(partials, 0, (size_t)M * N * si.G * sizeof(int32_t), st) != cudaSuccess)
             return W2A8_ERR_CUDA;
     }
-    cudaError_t e = si.spp == 1 ? launch_decode_spp<1>(p, partials != nullptr, st)
-                  : si.spp == 2 ? launch_decode_spp<2>(p, partials != nullptr, st)
-                                : launch_decode_spp<4>(p, partials != nullptr, st);
+    cudaError_t e = si.spp == 1 ? launch_decode_spp<1>(p, pl, partials != nullptr, st)
+                  : si.spp == 2 ? launch_decode_spp<2>(p, pl, partials != nullptr, st)
+                                : launch_decode_spp<4>(p, pl, partials != nullptr, st);
     return e == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
 

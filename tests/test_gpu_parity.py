@@ -162,14 +162,18 @@ def test_gemm_against_reference(gpu, oracle, M, N, K, group, ternary, frac):
     assert ok, f"worst error / bound = {worst}"
 
 
-@pytest.mark.parametrize("splits", [1, 8, 9, 14, 56])
-@pytest.mark.parametrize("M", [1, 12])
-def test_forced_split_k(gpu, oracle, splits, M, monkeypatch):
+@pytest.mark.parametrize("chunks,tg", [(1, 1), (2, 2), (5, 4), (59, 8), (3, 1)])
+@pytest.mark.parametrize("M,group", [(1, 64), (12, 64), (3, 128), (20, 0)])
+def test_forced_chunking(gpu, oracle, chunks, tg, M, group, monkeypatch):
+    """Every tile grouping and several split-K factors on a long contraction with
+    a ragged last chunk and a ragged last tile group."""
     torch, b = gpu
-    monkeypatch.setenv("W2A8_SPLITS", str(splits))
-    N, K, g = 64, 14336, 64
-    codes, s_w, bits, g = _problem(99 + splits, M, N, K, g)
-    a, s_a, y, _ = _run_gpu(torch, b, codes, s_w, bits, g, want_partials=False)
+    monkeypatch.setenv("W2A8_CHUNKS", str(chunks))
+    monkeypatch.setenv("W2A8_TG", str(tg))
+    N, K = 80, 14336 + 256 * 3
+    codes, s_w, bits, g = _problem(99 + chunks, M, N, K, group)
+    a, s_a, y, P = _run_gpu(torch, b, codes, s_w, bits, g)
+    assert np.array_equal(P, oracle.partials(a, codes, g))
     ok, worst = _row_err_ok(y, oracle.gemm(a, s_a, codes, s_w, g))
     assert ok, f"worst error / bound = {worst}"
 
