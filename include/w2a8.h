@@ -42,7 +42,8 @@ typedef enum {
     W2A8_ERR_ALIGN = -3,     /* a pointer is not 16-byte aligned */
     W2A8_ERR_WORKSPACE = -4, /* workspace missing or too small */
     W2A8_ERR_CUDA = -5,      /* a CUDA runtime call or launch failed */
-    W2A8_ERR_ARCH = -6       /* the current device is not sm_100 */
+    W2A8_ERR_ARCH = -6,      /* the current device is not sm_100 */
+    W2A8_ERR_TIMEOUT = -7    /* a bounded device-side wait gave up (see w2a8_workspace_status) */
 } w2a8_status;
 
 /* Library version: major * 10000 + minor * 100 + patch. */
@@ -102,6 +103,15 @@ size_t w2a8_workspace_bytes(int M, int N, int K, int group);
 
 /* Zero-fill a workspace (asynchronous, on `stream`). */
 int w2a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Read back the device status word kept at the start of a workspace.  Every
+ * wait inside the kernels (on an asynchronous-copy barrier) is bounded; a wait
+ * that gives up records W2A8_ERR_TIMEOUT here and the kernel returns without
+ * producing valid outputs instead of hanging.  Synchronises `stream`.  Returns
+ * the recorded status (W2A8_OK if none), or W2A8_ERR_CUDA / W2A8_ERR_NULL.
+ */
+int w2a8_workspace_status(const void *workspace, void *stream);
 
 /*
  * w2a8_gemm -- y[m][n] = a_scale[m] * sum_gi w_scale[n][gi] * P[m][n][gi] with

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libw2a8.so")
 
 EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
-    "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_gemm", "w2a8_gemm_partials",
+    "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
     "w2a8_linear_host_workspace_bytes", "w2a8_linear_host",
 ]
 
@@ -50,12 +50,13 @@ def lib() -> ctypes.CDLL:
         L.w2a8_workspace_bytes.restype = sz
         L.w2a8_workspace_bytes.argtypes = [i, i, i, i]
         L.w2a8_workspace_init.argtypes = [vp, sz, vp]
+        L.w2a8_workspace_status.argtypes = [vp, vp]
         L.w2a8_gemm.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_partials.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear_host_workspace_bytes.restype = sz
         L.w2a8_linear_host_workspace_bytes.argtypes = [i, i, i, i]
         L.w2a8_linear_host.argtypes = [vp, i, i, vp, vp, i, i, vp, vp, sz, vp]
-        for name in ("w2_pack", "a8_quantize", "w2a8_workspace_init", "w2a8_gemm",
+        for name in ("w2_pack", "a8_quantize", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm",
                      "w2a8_gemm_partials", "w2a8_linear_host"):
             getattr(L, name).restype = i
         _lib = L
@@ -106,6 +107,11 @@ def new_workspace(nbytes: int, device="cuda", stream=None) -> torch.Tensor:
 def w2a8_workspace_init(workspace: torch.Tensor, stream=None):
     _check(lib().w2a8_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
                                      _stream(stream)), "w2a8_workspace_init")
+
+
+def w2a8_workspace_status(workspace: torch.Tensor, stream=None) -> int:
+    """Device status word of a workspace (0 = ok); synchronises the stream."""
+    return int(lib().w2a8_workspace_status(_ptr(workspace), _stream(stream)))
 
 
 def w2_pack(codes: torch.Tensor, packed: torch.Tensor | None = None, stream=None) -> torch.Tensor:

@@ -10,7 +10,7 @@ namespace w2a8 {
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st);
-size_t decode_workspace_bytes(int M, int N, const ShapeInfo &si);
+size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
 
 int env_int(const char *name, int dflt) {
     const char *v = getenv(name);
@@ -138,6 +138,7 @@ const char *w2a8_status_string(int status) {
         case W2A8_ERR_WORKSPACE: return "workspace missing or too small";
         case W2A8_ERR_CUDA: return "CUDA runtime or launch error";
         case W2A8_ERR_ARCH: return "device is not sm_100";
+        case W2A8_ERR_TIMEOUT: return "a bounded device-side wait gave up";
         default: return "unknown status";
     }
 }
@@ -175,7 +176,7 @@ int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, voi
 size_t w2a8_workspace_bytes(int M, int N, int K, int group) {
     ShapeInfo si;
     if (!shape_ok(M, N, K, group, &si)) return 0;
-    return decode_workspace_bytes(M, N, si);
+    return decode_workspace_bytes(M, N, K, si);
 }
 
 int w2a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream) {
@@ -183,6 +184,16 @@ int w2a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream) {
     if (cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream) != cudaSuccess)
         return W2A8_ERR_CUDA;
     return W2A8_OK;
+}
+
+int w2a8_workspace_status(const void *workspace, void *stream) {
+    if (!workspace) return W2A8_ERR_NULL;
+    int status = 0;
+    if (cudaMemcpyAsync(&status, workspace, sizeof(int), cudaMemcpyDeviceToHost,
+                        (cudaStream_t)stream) != cudaSuccess)
+        return W2A8_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return W2A8_ERR_CUDA;
+    return status;
 }
 
 static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *packed,
@@ -194,7 +205,7 @@ static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *pa
         (w_scale && !aligned16(w_scale)) || (partials && !aligned16(partials)) ||
         (a_scale && (reinterpret_cast<uintptr_t>(a_scale) & 3u)))
         return W2A8_ERR_ALIGN;
-    const size_t need = decode_workspace_bytes(M, N, si);
+    const size_t need = decode_workspace_bytes(M, N, K, si);
     if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
     if (int st = check_device()) return st;
     return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,

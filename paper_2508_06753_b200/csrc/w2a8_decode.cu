@@ -2,36 +2,41 @@
 // 2-bit weights once, unpacks them in registers and feeds int8 tensor-core
 // MMAs (mma.sync m16n8k32) whose A operand is a 16-channel x 32-k weight tile
 // and whose B operand is 32 k x 8 tokens.  The up-convert-and-compute idea is
-// that of Sec. II-C, the K-splitting that of Sec. II-D; the thread/tile mapping
-// and the launch overlap are specific to sm_100a.
+// that of Sec. II-C, the K-splitting that of Sec. II-D; the staging, the
+// thread/tile mapping and the launch overlap are specific to sm_100a.
 //
 // Work split.  A "cell" is one 16-channel tile x one 256-k block: 1 KB of packed
-// weights plus its scales.  A CTA of 8 warps owns TG tiles and one chunk of the
-// contraction; its warps are arranged TG tiles x KS = 8 / TG K-lanes, and the
+// weights plus its scales.  A CTA of 4 warps owns TG tiles and one chunk of the
+// contraction; its warps are arranged TG tiles x KS = 4 / TG K-lanes, and the
 // K-lanes take interleaved blocks of the chunk.  The K-lanes of a tile are
 // summed through shared memory in a fixed order; chunks (grid.y, only used when
-// the shape would otherwise leave SMs idle or the activations would not fit in
-// shared memory) are summed through the workspace by the last CTA to arrive,
-// also in a fixed order.  grid.z walks 8*MT-token slabs.
+// the shape would otherwise leave SMs idle or the data would not fit in shared
+// memory) are summed through the workspace by the last CTA to arrive, also in a
+// fixed order.  grid.z walks 8*MT-token slabs.
 //
-// Pipeline.  Each lane keeps the next cell's weights and scales in flight in
-// registers while it computes the current one.  The first cell is requested
-// before the kernel waits for the previous kernel of the stream (weights and
-// scales are frozen; only activations depend on it), so under programmatic
-// dependent launch the weight stream starts while the previous kernel drains.
-// The chunk's activations are staged once per CTA in shared memory.
+// Pipeline.  In the W2P layout the weights of a tile are 16 row segments of
+// plain contiguous bytes, so one warp fetches the CTA's whole share with a few
+// bulk asynchronous copies (cp.async.bulk, global -> shared, completion on an
+// mbarrier), in two phases along K so that compute starts when the first half
+// has landed.  The copies are issued before the kernel waits for the previous
+// kernel of the stream (weights and scales are frozen; only activations depend
+// on it), so under programmatic dependent launch the weight stream of this
+// kernel overlaps the tail of the previous one.  Activations of the chunk are
+// staged once per CTA after that wait.
 //
-// In the W2P layout one 128-bit unit per lane and channel holds word t of each
-// of the four 64-k slices of a block -- exactly what the four lanes of an MMA
-// quad must supply so that every MMA sums k of a single scale group.
+// One 128-bit unit per lane and channel holds word t of each of the four 64-k
+// slices of a block -- exactly what the four lanes of an MMA quad must supply
+// so that every MMA sums k of a single scale group.
 #include "w2a8_common.cuh"
 
 namespace w2a8 {
 
-constexpr int kDecodeWarps = 8;
+constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kActPad = 64;                    // row stride = chunk bytes + 64: conflict-free LDS.128
-constexpr int kActSmemMax = 96 * 1024;         // staged activations per CTA
+constexpr int kActPad = 64;                    // activation row stride = chunk bytes + 64
+constexpr int kSmemBudget = 100 * 1024;        // per CTA: weights + scales + activations
+constexpr int kPhases = 4;
+constexpr unsigned kWaitPolls = 1u << 20;      // bounded mbarrier wait (each poll may suspend)
 
 struct DecodeParams {
     const int8_t *a;
@@ -42,20 +47,62 @@ struct DecodeParams {
     int32_t *partials;
     float *ws;            // [chunks][M][N] partial outputs (chunks > 1)
     unsigned *counters;   // [grid.z][tile groups] arrival counters (chunks > 1)
+    int *status;          // device status word (0 = ok)
     int M, N, K, G, group;
     int blocks, tail_slices, words_per_row;
     int chunks, blocks_per_chunk;
+    int w_stride;         // bytes per staged weight row
+    int s_stride;         // bytes per staged scale row
     int act_stride;       // bytes per staged token row
-    int vec_ok;           // K % 256 == 0: scale rows can be read as float4 / float2
+    int s_bulk;           // scale rows can be fetched by bulk copies (16-byte granularity holds)
+    int off_s, off_a;     // byte offsets of the scale and activation areas in shared memory
 };
 
-__device__ __forceinline__ uint4 ld_stream_v4(const uint32_t *p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
+// ---- PTX wrappers ------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the barrier did not complete within kWaitPolls polls.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, unsigned parity) {
+    for (unsigned i = 0; i < kWaitPolls; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// global -> shared bulk copy; size and both addresses are multiples of 16 bytes
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, unsigned bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// per-thread asynchronous copies (activations, and scales that bulk copies cannot take)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // Optional timeline trace (build with -DW2A8_TRACE): every warp records the
 // global timer at a few points of the kernel into a caller-provided buffer.
@@ -76,65 +123,49 @@ __device__ __forceinline__ unsigned long long global_ns() {
 #define W2A8_TRACE_POINT(i) do { } while (0)
 #endif
 
-template <int SPP>
-struct Cell {
-    uint32_t w[2][4];                 // [channel g / g+8][slice]
-    float sc[2][4 / SPP];             // [channel][scale group inside the block]
-};
-
-template <int SPP, bool PARTIALS>
-__device__ __forceinline__ void load_cell(const DecodeParams &p, Cell<SPP> &c, int n0, int gq,
-                                          int t, int kb) {
-    const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        const size_t row = (size_t)(n0 + gq + 8 * r);
-        const uint32_t *wp = p.packed + row * p.words_per_row + 16 * kb;
-        if (R == 4) {
-            const uint4 v = ld_stream_v4(wp + 4 * t);
-            c.w[r][0] = v.x; c.w[r][1] = v.y; c.w[r][2] = v.z; c.w[r][3] = v.w;
-        } else {   // trailing block with fewer slices: words t*R .. t*R+R-1
-#pragma unroll
-            for (int s = 0; s < 4; ++s) c.w[r][s] = (s < R) ? __ldg(wp + t * R + s) : 0u;
-        }
-        if constexpr (PARTIALS) {
-            // the parity export has no scales
-        } else if constexpr (SPP == 1) {
-            const float *sp = p.w_scale + row * p.G + 4 * kb;
-            if (R == 4 && p.vec_ok) {
-                const float4 v = __ldg(reinterpret_cast<const float4 *>(sp));
-                c.sc[r][0] = v.x; c.sc[r][1] = v.y; c.sc[r][2] = v.z; c.sc[r][3] = v.w;
-            } else {
-#pragma unroll
-                for (int s = 0; s < 4; ++s) c.sc[r][s] = (s < R) ? __ldg(sp + s) : 0.f;
-            }
-        } else if constexpr (SPP == 2) {
-            const float *sp = p.w_scale + row * p.G + 2 * kb;
-            if (R == 4 && p.vec_ok) {
-                const float2 v = __ldg(reinterpret_cast<const float2 *>(sp));
-                c.sc[r][0] = v.x; c.sc[r][1] = v.y;
-            } else {
-#pragma unroll
-                for (int s = 0; s < 2; ++s) c.sc[r][s] = (2 * s < R) ? __ldg(sp + s) : 0.f;
-            }
-        } else {
-            c.sc[r][0] = __ldg(p.w_scale + row * p.G + (int)(((long long)kb * kBlockK) / p.group));
-        }
-    }
-}
-
 // One cell: 4 slices x (unpack, 2 MMAs per token slab, promotion at group ends).
+// wrow0/wrow1: staged weight rows of channels n0+gq and n0+gq+8, already offset
+// by this lane's quarter t; srow0/srow1: staged scale rows of the same channels.
 template <int MT, int SPP, bool ONE, bool PARTIALS>
-__device__ __forceinline__ void compute_cell(const DecodeParams &p, const Cell<SPP> &c,
-                                             const unsigned char *const (&brow)[MT], int kcol,
+__device__ __forceinline__ void compute_cell(const DecodeParams &p, const unsigned char *wrow0,
+                                             const unsigned char *wrow1, const unsigned char *srow0,
+                                             const unsigned char *srow1,
+                                             const unsigned char *const (&brow)[MT], int kl,
                                              int kb, int n0, int m0, int gq, int t,
                                              float (&acc)[MT][4], int (&D)[MT][4]) {
     const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
     const int magic[4] = {kMagicInt, kMagicInt, kMagicInt, kMagicInt};
+    uint32_t w0s[4], w1s[4];
+    if (R == 4) {
+        const uint4 va = *reinterpret_cast<const uint4 *>(wrow0 + kl * 64);
+        const uint4 vb = *reinterpret_cast<const uint4 *>(wrow1 + kl * 64);
+        w0s[0] = va.x; w0s[1] = va.y; w0s[2] = va.z; w0s[3] = va.w;
+        w1s[0] = vb.x; w1s[1] = vb.y; w1s[2] = vb.z; w1s[3] = vb.w;
+    } else {   // trailing block with fewer slices: words t*R .. t*R+R-1 (wrow has +16 t)
+        const uint32_t *q0 = reinterpret_cast<const uint32_t *>(wrow0 + kl * 64 - 16 * t) + t * R;
+        const uint32_t *q1 = reinterpret_cast<const uint32_t *>(wrow1 + kl * 64 - 16 * t) + t * R;
+#pragma unroll
+        for (int s = 0; s < 4; ++s) { w0s[s] = (s < R) ? q0[s] : 0u; w1s[s] = (s < R) ? q1[s] : 0u; }
+    }
+    float s0s[4 / SPP], s1s[4 / SPP];
+    if constexpr (!PARTIALS) {
+        if constexpr (SPP == 4) {
+            const int gi = (int)(((long long)kb * kBlockK) / p.group);
+            s0s[0] = reinterpret_cast<const float *>(srow0)[gi];
+            s1s[0] = reinterpret_cast<const float *>(srow1)[gi];
+        } else {
+            constexpr int SPB = 4 / SPP;
+#pragma unroll
+            for (int j = 0; j < SPB; ++j) {
+                s0s[j] = (j * SPP < R) ? reinterpret_cast<const float *>(srow0)[kl * SPB + j] : 0.f;
+                s1s[j] = (j * SPP < R) ? reinterpret_cast<const float *>(srow1)[kl * SPB + j] : 0.f;
+            }
+        }
+    }
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
         if (s < R) {
-            const uint32_t w0 = c.w[0][s], w1 = c.w[1][s];
+            const uint32_t w0 = w0s[s], w1 = w1s[s];
             const uint32_t a0 = lane_codes(w0, 0), a1 = lane_codes(w1, 0);
             const uint32_t a2 = lane_codes(w0, 1), a3 = lane_codes(w1, 1);
             const uint32_t a4 = lane_codes(w0, 2), a5 = lane_codes(w1, 2);
@@ -143,7 +174,7 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const Cell<S
             const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
-                const uint4 b = *reinterpret_cast<const uint4 *>(brow[mt] + kcol + s * kSliceK);
+                const uint4 b = *reinterpret_cast<const uint4 *>(brow[mt] + kl * kBlockK + s * kSliceK);
                 if (first) mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, magic);
                 else       mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, D[mt]);
                 mma_s8_16x8x32(D[mt], a4, a5, a6, a7, b.z, b.w, D[mt]);
@@ -161,7 +192,7 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const Cell<S
                                           (D[mt][i] - kMagicInt) >> 6);
                         }
                     } else {
-                        const float s0 = c.sc[0][s / SPP], s1 = c.sc[1][s / SPP];
+                        const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
                         acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
                         acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
                         if constexpr (!ONE) {
@@ -176,13 +207,14 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const Cell<S
 }
 
 // MT: 8-token slabs per CTA; SPP: 64-k slices per scale group (capped at 4);
-// TG: tiles per CTA (K-lanes per tile = 8 / TG); ONE: a single token (half of
+// TG: tiles per CTA (K-lanes per tile = 4 / TG); ONE: a single token (half of
 // each accumulator quad is dead and is not promoted).
 template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
-__global__ void __launch_bounds__(kDecodeThreads, (MT == 1 ? 4 : (MT == 2 ? 3 : 2)))
+__global__ void __launch_bounds__(kDecodeThreads, (MT == 1 ? 7 : (MT == 2 ? 5 : 4)))
 w2a8_decode_kernel(const DecodeParams p) {
     constexpr int KS = kDecodeWarps / TG;
     extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long bars[kPhases];
     __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, t = lane & 3;
@@ -193,35 +225,101 @@ w2a8_decode_kernel(const DecodeParams p) {
     const int chunk = blockIdx.y;
     const int kb_begin = chunk * p.blocks_per_chunk;
     const int kb_end = min(kb_begin + p.blocks_per_chunk, p.blocks);
+    const int nb = kb_end - kb_begin;
     const int m0 = blockIdx.z * (8 * MT);
     const int mrows = min(8 * MT, p.M - m0);
+    unsigned char *sm_w = smem;                 // [TG * 16][w_stride]
+    unsigned char *sm_s = smem + p.off_s;       // [TG * 16][s_stride]
+    unsigned char *acts = smem + p.off_a;       // [mrows + 1][act_stride]
     W2A8_TRACE_POINT(0);
 
-    // ---- request the first cell (independent of the previous kernel) ----------
-    int kb = kb_begin + ks;
-    Cell<SPP> cA, cB;
-    if (tile_ok && kb < kb_end) load_cell<SPP, PARTIALS>(p, cA, n0, gq, t, kb);
+    // The chunk is fetched in kPhases pieces along K, one mbarrier each.  Piece 0
+    // is requested before the dependency wait; the activations are requested
+    // next (right behind piece 0 in the memory queues, so compute can start while
+    // the rest streams in); the remaining pieces follow.
+    const int nbp = (nb + kPhases - 1) / kPhases;                 // blocks per piece
+    const int words_end = min(16 * kb_end, p.words_per_row);      // last block may be short
+    constexpr int SPB = 4 / SPP;                                  // scales per block and channel
+    const int sc_begin = (SPP == 4) ? 0 : SPB * kb_begin;
+    const int sc_end = (SPP == 4) ? p.G : min(SPB * kb_end, p.G);
+    // scale rows go by bulk copy only where every piece is a whole number of 16-byte
+    // units (the host has checked the row pitch and the chunk starts); SPP == 1 only
+    const bool sbulk = (!PARTIALS) && (SPP == 1) && p.s_bulk;
+    const int tiles_here = min(TG, p.N / 16 - blockIdx.x * TG);
+    const int rows_here = tiles_here * 16;
+
+    auto post_piece = [&](int ph) {   // executed by warp 0
+        const int b0 = min(ph * nbp, nb), b1 = min((ph + 1) * nbp, nb);
+        const int w0 = 16 * (kb_begin + b0), w1 = min(16 * (kb_begin + b1), words_end);
+        const unsigned wbytes = w1 > w0 ? (unsigned)(w1 - w0) * 4u : 0u;
+        const int s0 = SPB * (kb_begin + b0), s1 = min(SPB * (kb_begin + b1), p.G);
+        const unsigned sbytes = (sbulk && s1 > s0) ? (unsigned)(s1 - s0) * 4u : 0u;
+        const uint32_t bar = smem_u32(&bars[ph]);
+        unsigned tx = 0;
+        for (int r = lane; r < rows_here; r += 32) {
+            const size_t row = (size_t)blockIdx.x * TG * 16 + r;
+            if (wbytes) {
+                bulk_g2s(smem_u32(sm_w + r * p.w_stride) + (unsigned)(w0 - 16 * kb_begin) * 4u,
+                         p.packed + row * p.words_per_row + w0, wbytes, bar);
+                tx += wbytes;
+            }
+            if (sbytes) {
+                bulk_g2s(smem_u32(sm_s + r * p.s_stride) + (unsigned)(s0 - sc_begin) * 4u,
+                         p.w_scale + row * p.G + s0, sbytes, bar);
+                tx += sbytes;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) tx += __shfl_xor_sync(0xFFFFFFFFu, tx, o);
+        if (lane == 0) mbar_arrive_expect_tx(bar, tx);
+    };
+
+    // ---- piece 0 and the scales that cannot go by bulk copy (all independent of
+    //      the previous kernel) ---------------------------------------------------
+    if (warp == 0) {
+        if (lane == 0) {
+#pragma unroll
+            for (int ph = 0; ph < kPhases; ++ph) mbar_init(smem_u32(&bars[ph]), 1);
+            mbar_fence_init();
+        }
+        __syncwarp();
+        post_piece(0);
+    }
+    if ((!PARTIALS) && !sbulk) {
+        const int nsc = sc_end - sc_begin;
+        for (int u = threadIdx.x; u < rows_here * nsc; u += kDecodeThreads) {
+            const int r = u / nsc, j = u % nsc;
+            cp_async4(smem_u32(sm_s + r * p.s_stride + 4 * j),
+                      p.w_scale + ((size_t)blockIdx.x * TG * 16 + r) * p.G + sc_begin + j);
+        }
+    }
     W2A8_TRACE_POINT(1);
     pdl_launch_dependents();
     pdl_wait();
     W2A8_TRACE_POINT(2);
 
-    // ---- stage the activations of this chunk: [mrows + 1][chunk k (+pad)]; the
+    // ---- request the activations of this chunk: [mrows + 1][chunk k (+pad)]; the
     //      extra row is zeros and stands in for tokens beyond M --------------------
-    unsigned char *acts = smem;
     {
-        const int row_units = (kb_end - kb_begin) * (kBlockK / 16);
-        const int klen = min((kb_end - kb_begin) * kBlockK, p.K - kb_begin * kBlockK);
+        const int row_units = nb * (kBlockK / 16);
+        const int klen = min(nb * kBlockK, p.K - kb_begin * kBlockK);
         for (int u = threadIdx.x; u < (mrows + 1) * row_units; u += kDecodeThreads) {
             const int r = u / row_units, cu = u % row_units;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            unsigned char *dst = acts + r * p.act_stride + cu * 16;
             if (r < mrows && cu * 16 < klen)
-                v = *reinterpret_cast<const uint4 *>(p.a + (size_t)(m0 + r) * p.K +
-                                                     (size_t)kb_begin * kBlockK + cu * 16);
-            *reinterpret_cast<uint4 *>(acts + r * p.act_stride + cu * 16) = v;
+                cp_async16(smem_u32(dst), p.a + (size_t)(m0 + r) * p.K + (size_t)kb_begin * kBlockK + cu * 16);
+            else
+                *reinterpret_cast<uint4 *>(dst) = make_uint4(0u, 0u, 0u, 0u);
         }
+        cp_async_commit();
     }
-    __syncthreads();
+    // ---- the remaining pieces -----------------------------------------------------
+    if (warp == 0) {
+#pragma unroll
+        for (int ph = 1; ph < kPhases; ++ph) post_piece(ph);
+    }
+    cp_async_wait_all();
+    __syncthreads();   // activations and fallback scales staged; barriers initialised
     W2A8_TRACE_POINT(3);
 
     float acc[MT][4];
@@ -231,31 +329,41 @@ w2a8_decode_kernel(const DecodeParams p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) { acc[mt][i] = 0.f; D[mt][i] = kMagicInt; }
 
+    bool timed_out = false;
     if (tile_ok) {
         const unsigned char *brow[MT];   // this lane's token row of each slab (or the zero row)
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
             brow[mt] = acts + ((8 * mt + gq < mrows) ? (8 * mt + gq) : mrows) * p.act_stride + t * 16;
-        // two cells in flight, alternating register sets
-        while (kb < kb_end) {
-            const int kb1 = kb + KS;
-            if (kb1 < kb_end) load_cell<SPP, PARTIALS>(p, cB, n0, gq, t, kb1);
-            compute_cell<MT, SPP, ONE, PARTIALS>(p, cA, brow, (kb - kb_begin) * kBlockK, kb, n0, m0,
-                                                 gq, t, acc, D);
-            if (kb1 >= kb_end) break;
-            const int kb2 = kb1 + KS;
-            if (kb2 < kb_end) load_cell<SPP, PARTIALS>(p, cA, n0, gq, t, kb2);
-            compute_cell<MT, SPP, ONE, PARTIALS>(p, cB, brow, (kb1 - kb_begin) * kBlockK, kb1, n0,
-                                                 m0, gq, t, acc, D);
-            kb = kb2;
+        const unsigned char *wrow0 = sm_w + (tl * 16 + gq) * p.w_stride + t * 16;
+        const unsigned char *wrow1 = wrow0 + 8 * p.w_stride;
+        const unsigned char *srow0 = sm_s + (tl * 16 + gq) * p.s_stride;   // floats from sc_begin on
+        const unsigned char *srow1 = srow0 + 8 * p.s_stride;
+        int phase_ready = -1;
+        for (int kl = ks; kl < nb; kl += KS) {
+            const int need = kl / nbp;
+            while (phase_ready < need) {
+                ++phase_ready;
+                if (!mbar_wait_bounded(smem_u32(&bars[phase_ready]), 0)) timed_out = true;
+            }
+            if (timed_out) break;
+            compute_cell<MT, SPP, ONE, PARTIALS>(p, wrow0, wrow1, srow0, srow1, brow, kl, kb_begin + kl,
+                                                 n0, m0, gq, t, acc, D);
         }
     }
     W2A8_TRACE_POINT(5);
 
+    // Nobody may leave while bulk copies into this CTA's shared memory are in
+    // flight: every thread passes every barrier (bounded) before the CTA retires.
+#pragma unroll
+    for (int ph = 0; ph < kPhases; ++ph)
+        if (!mbar_wait_bounded(smem_u32(&bars[ph]), 0)) timed_out = true;
+    if (timed_out) atomicExch(p.status, W2A8_ERR_TIMEOUT);
+
     if constexpr (!PARTIALS) {
         // ---- sum the K-lanes of each tile in a fixed order -----------------------
         // lane (gq, t) holds channels n0+gq, n0+gq+8 for tokens 2t, 2t+1 of each slab
-        float *red = reinterpret_cast<float *>(smem);   // [KS][TG][MT*4][32], reuses the staging area
+        float *red = reinterpret_cast<float *>(acts);   // [KS][TG][MT*4][32], reuses the staging area
         __syncthreads();   // everyone is done reading the staged activations
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
@@ -316,29 +424,53 @@ extern "C" int w2a8_debug_set_trace(void *buffer) {
 int env_int(const char *name, int dflt);
 
 static inline int decode_mt(int M) { return M > 32 ? 4 : (M + 7) / 8; }
+static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct DecodePlan {
     int mt, tg, chunks, blocks_per_chunk, slabs, groups;
+    int w_stride, s_stride, act_stride, off_s, off_a, s_bulk;
     size_t smem;
 };
 
-// Tiles per CTA and K-chunks.  One tile per CTA (8 K-lanes) keeps each warp's
+// Shared-memory footprint of a CTA that stages `nb` blocks of K.
+static void plan_smem(DecodePlan &pl, int M, int K, int G, int spp, int nb) {
+    const int mrows = M < 8 * pl.mt ? M : 8 * pl.mt;
+    // weight rows: 64 bytes per block; stride = 64 mod 128 keeps the 8 channel
+    // rows of a quarter-warp LDS.128 on distinct banks
+    int wseg = nb * 64;
+    pl.w_stride = round_up(wseg, 128) + 64;
+    // scale rows: stride = 16 mod 128 spreads the 8 channels of a warp read
+    const int nsc = spp == 4 ? G : (4 / spp) * nb;
+    pl.s_stride = round_up(nsc * 4, 128) + 16;
+    pl.act_stride = nb * kBlockK + kActPad;
+    pl.off_s = pl.tg * 16 * pl.w_stride;
+    pl.off_a = round_up(pl.off_s + pl.tg * 16 * pl.s_stride, 128);
+    const size_t act = (size_t)(mrows + 1) * pl.act_stride;
+    const size_t red = (size_t)kDecodeWarps * pl.mt * 4 * 32 * sizeof(float);
+    pl.smem = pl.off_a + (act > red ? act : red);
+    (void)K;
+}
+
+// Tiles per CTA and K-chunks.  One tile per CTA (4 K-lanes) keeps each warp's
 // serial work shortest; several tiles per CTA share the staged activations,
 // which matters once there are many tokens.  Chunks are added when the staged
-// activations would not fit, or when the grid would leave most SMs idle.
-static DecodePlan decode_plan(int M, int N, const ShapeInfo &si) {
+// data would not fit, or when the grid would leave most SMs idle.
+static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
     DecodePlan pl;
     pl.mt = decode_mt(M);
     pl.slabs = (M + 8 * pl.mt - 1) / (8 * pl.mt);
     const int forced_tg = env_int("W2A8_TG", 0);
-    pl.tg = (forced_tg == 1 || forced_tg == 2 || forced_tg == 4 || forced_tg == 8)
+    pl.tg = (forced_tg == 1 || forced_tg == 2 || forced_tg == 4)
                 ? forced_tg : (pl.mt == 1 ? 1 : (pl.mt == 2 ? 2 : 4));
     pl.groups = (N / 16 + pl.tg - 1) / pl.tg;
-    const int mrows = M < 8 * pl.mt ? M : 8 * pl.mt;
-    int max_blocks = (kActSmemMax / (mrows + 1) - kActPad) / kBlockK;    // activations must fit
-    if (max_blocks < 1) max_blocks = 1;
-    int chunks = (si.blocks + max_blocks - 1) / max_blocks;
     const int ks = kDecodeWarps / pl.tg;
+    int chunks = 1;
+    for (;;) {   // smallest chunk count whose staging fits the budget
+        const int bpc = (si.blocks + chunks - 1) / chunks;
+        plan_smem(pl, M, K, si.G, si.spp, bpc);
+        if ((int)pl.smem <= kSmemBudget || bpc == 1) break;
+        ++chunks;
+    }
     const int forced = env_int("W2A8_CHUNKS", 0);
     if (forced > 0) {
         if (forced > chunks) chunks = forced;
@@ -350,19 +482,22 @@ static DecodePlan decode_plan(int M, int N, const ShapeInfo &si) {
     if (chunks > si.blocks) chunks = si.blocks;
     pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
     pl.chunks = (si.blocks + pl.blocks_per_chunk - 1) / pl.blocks_per_chunk;
-    const size_t act = (size_t)(mrows + 1) * (pl.blocks_per_chunk * kBlockK + kActPad);
-    const size_t red = (size_t)kDecodeWarps * pl.mt * 4 * 32 * sizeof(float);
-    pl.smem = act > red ? act : red;
+    plan_smem(pl, M, K, si.G, si.spp, pl.blocks_per_chunk);
+    // bulk-copy granularity for scales (group 64 only: four floats per block): the
+    // row pitch must be a multiple of 16 bytes
+    pl.s_bulk = (si.spp == 1) && (si.G % 4 == 0) && (K % 256 == 0);
     return pl;
 }
 
-size_t decode_workspace_bytes(int M, int N, const ShapeInfo &si) {
-    const DecodePlan pl = decode_plan(M, N, si);
+constexpr size_t kStatusBytes = 256;   // workspace header: status word
+
+size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si) {
+    const DecodePlan pl = decode_plan(M, N, K, si);
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;   // >= any tile grouping
     // with an environment override in force, size for the finest split
     const int chunks = (env_int("W2A8_CHUNKS", 0) > 0 || env_int("W2A8_TG", 0) > 0) ? si.blocks : pl.chunks;
     size_t part = (size_t)(chunks > 1 ? chunks : 0) * M * N * sizeof(float);
-    return counters + part;
+    return kStatusBytes + counters + part;
 }
 
 template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
@@ -393,8 +528,7 @@ static cudaError_t launch_decode_mt(const DecodeParams &p, const DecodePlan &pl,
     switch (pl.tg) {
         case 1: return launch_decode_tg<MT, SPP, 1>(p, want_partials, grid, pl.smem, st);
         case 2: return launch_decode_tg<MT, SPP, 2>(p, want_partials, grid, pl.smem, st);
-        case 4: return launch_decode_tg<MT, SPP, 4>(p, want_partials, grid, pl.smem, st);
-        default: return launch_decode_tg<MT, SPP, 8>(p, want_partials, grid, pl.smem, st);
+        default: return launch_decode_tg<MT, SPP, 4>(p, want_partials, grid, pl.smem, st);
     }
 }
 
@@ -413,18 +547,20 @@ static cudaError_t launch_decode_spp(const DecodeParams &p, const DecodePlan &pl
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st) {
-    const DecodePlan pl = decode_plan(M, N, si);
+    const DecodePlan pl = decode_plan(M, N, K, si);
     DecodeParams p;
     p.a = a; p.a_scale = a_scale; p.packed = packed; p.w_scale = w_scale;
     p.y = y; p.partials = partials;
     p.M = M; p.N = N; p.K = K; p.G = si.G; p.group = group;
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
     p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;
-    p.act_stride = pl.blocks_per_chunk * kBlockK + kActPad;
-    p.vec_ok = (K % 256 == 0) ? 1 : 0;
+    p.w_stride = pl.w_stride; p.s_stride = pl.s_stride; p.act_stride = pl.act_stride;
+    p.off_s = pl.off_s; p.off_a = pl.off_a; p.s_bulk = pl.s_bulk;
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
-    p.counters = reinterpret_cast<unsigned *>(workspace);
-    p.ws = reinterpret_cast<float *>(reinterpret_cast<char *>(workspace) + counters);
+    char *base = reinterpret_cast<char *>(workspace);
+    p.status = reinterpret_cast<int *>(base);
+    p.counters = reinterpret_cast<unsigned *>(base + kStatusBytes);
+    p.ws = reinterpret_cast<float *>(base + kStatusBytes + counters);
     if (partials) {
         // several warps add their share of a large group: start from zero
         if (cudaMemsetAsync(partials, 0, (size_t)M * N * si.G * sizeof(int32_t), st) != cudaSuccess)

@@ -57,11 +57,11 @@ def test_sizes_and_version(lib):
 
 def test_status_strings(lib):
     seen = set()
-    for code in range(0, -7, -1):
+    for code in range(0, -8, -1):
         s = lib.w2a8_status_string(code).decode()
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 7
+    assert len(seen) == 8
     assert lib.w2a8_status_string(-99).decode() == "unknown status"
 
 
@@ -88,6 +88,7 @@ def test_argument_errors_are_detected_on_the_host(lib):
     assert lib.w2a8_linear_host(p, 1, 64, p, p, 16, 48, p, p, 1 << 15, None) == SHAPE
     assert lib.w2a8_linear_host(p, 1, 64, p, p, 16, 64, p, p, 16, None) == WS
     assert lib.w2a8_workspace_init(None, 16, None) == NULLP
+    assert lib.w2a8_workspace_status(None, None) == NULLP
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
