@@ -474,6 +474,13 @@ def run_ours(args):
     probes = []
     e2e = None
     cpu = None
+    if args.only_headline:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world,
+                              "steps": args.steps, "warmup": args.warmup,
+                              "ms_per_step": ms_all / args.steps, "launch": mode, "clocks": clocks,
+                              "gpu_launches": args.steps * len(cfg["Ms"]) * rep.kernels_per_pass}))
+        return
     if rank == 0:
         for M in cfg["Ms"]:
             sub = dict(cfg, Ms=[M])
@@ -583,6 +590,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only-headline", action="store_true",
+                    help="time the steps only (no per-M breakdown, kernel probe, e2e or CPU baseline); "
+                         "short command for profilers")
     ap.add_argument("--profile-shape", default=None, help="KxN: run only a few launches of this GEMM")
     ap.add_argument("--profile-m", type=int, default=1)
     ap.add_argument("--profile-group", type=int, default=64)

@@ -14,15 +14,15 @@
 // memory) are summed through the workspace by the last CTA to arrive, also in a
 // fixed order.  grid.z walks 8*MT-token slabs.
 //
-// Pipeline.  In the W2P layout the weights of a tile are 16 row segments of
-// plain contiguous bytes, so one warp fetches the CTA's whole share with a few
-// bulk asynchronous copies (cp.async.bulk, global -> shared, completion on an
-// mbarrier), in two phases along K so that compute starts when the first half
-// has landed.  The copies are issued before the kernel waits for the previous
-// kernel of the stream (weights and scales are frozen; only activations depend
-// on it), so under programmatic dependent launch the weight stream of this
-// kernel overlaps the tail of the previous one.  Activations of the chunk are
-// staged once per CTA after that wait.
+// Pipeline.  A warp works in rounds of up to four cells.  Each lane requests the
+// weights of a whole round with 128-bit loads into registers; the first half of
+// the first round is requested before the kernel waits for the previous kernel
+// of the stream (weights and scales are frozen; only activations depend on it),
+// so under programmatic dependent launch the weight stream of this kernel
+// overlaps the tail of the previous one.  The activations of the chunk are
+// requested right behind that first half (so that they do not queue behind the
+// whole weight stream), then the second half.  Scales and activations are
+// staged once per CTA in shared memory by per-thread asynchronous copies.
 //
 // One 128-bit unit per lane and channel holds word t of each of the four 64-k
 // slices of a block -- exactly what the four lanes of an MMA quad must supply
@@ -34,9 +34,8 @@ namespace w2a8 {
 constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kActPad = 64;                    // activation row stride = chunk bytes + 64
-constexpr int kSmemBudget = 100 * 1024;        // per CTA: weights + scales + activations
-constexpr int kPhases = 4;
-constexpr unsigned kWaitPolls = 1u << 20;      // bounded mbarrier wait (each poll may suspend)
+constexpr int kSmemBudget = 64 * 1024;         // per CTA: scales + activations
+constexpr int kRound = 4;                      // cells whose weights a lane holds at once
 
 struct DecodeParams {
     const int8_t *a;
@@ -51,49 +50,23 @@ struct DecodeParams {
     int M, N, K, G, group;
     int blocks, tail_slices, words_per_row;
     int chunks, blocks_per_chunk;
-    int w_stride;         // bytes per staged weight row
     int s_stride;         // bytes per staged scale row
     int act_stride;       // bytes per staged token row
-    int s_bulk;           // scale rows can be fetched by bulk copies (16-byte granularity holds)
-    int off_s, off_a;     // byte offsets of the scale and activation areas in shared memory
+    int s_vec;            // scale rows can be copied in 16-byte units
+    int off_a;            // byte offset of the activation area in shared memory
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ void mbar_init(uint32_t bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+__device__ __forceinline__ uint4 ld_stream_v4(const uint32_t *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
 }
-__device__ __forceinline__ void mbar_fence_init() {
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the barrier did not complete within kWaitPolls polls.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, unsigned parity) {
-    for (unsigned i = 0; i < kWaitPolls; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// global -> shared bulk copy; size and both addresses are multiples of 16 bytes
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, unsigned bytes, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
 // per-thread asynchronous copies (activations, and scales that bulk copies cannot take)
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -124,42 +97,32 @@ __device__ __forceinline__ unsigned long long global_ns() {
 #endif
 
 // One cell: 4 slices x (unpack, 2 MMAs per token slab, promotion at group ends).
-// wrow0/wrow1: staged weight rows of channels n0+gq and n0+gq+8, already offset
-// by this lane's quarter t; srow0/srow1: staged scale rows of the same channels.
+// w0s/w1s: this lane's four words (one per slice) of channels n0+gq and n0+gq+8;
+// srow0/srow1: staged scale rows of the same channels.
 template <int MT, int SPP, bool ONE, bool PARTIALS>
-__device__ __forceinline__ void compute_cell(const DecodeParams &p, const unsigned char *wrow0,
-                                             const unsigned char *wrow1, const unsigned char *srow0,
+__device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32_t (&w0s)[4],
+                                             const uint32_t (&w1s)[4], const unsigned char *srow0,
                                              const unsigned char *srow1,
                                              const unsigned char *const (&brow)[MT], int kl,
                                              int kb, int n0, int m0, int gq, int t,
                                              float (&acc)[MT][4], int (&D)[MT][4]) {
     const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
     const int magic[4] = {kMagicInt, kMagicInt, kMagicInt, kMagicInt};
-    uint32_t w0s[4], w1s[4];
-    if (R == 4) {
-        const uint4 va = *reinterpret_cast<const uint4 *>(wrow0 + kl * 64);
-        const uint4 vb = *reinterpret_cast<const uint4 *>(wrow1 + kl * 64);
-        w0s[0] = va.x; w0s[1] = va.y; w0s[2] = va.z; w0s[3] = va.w;
-        w1s[0] = vb.x; w1s[1] = vb.y; w1s[2] = vb.z; w1s[3] = vb.w;
-    } else {   // trailing block with fewer slices: words t*R .. t*R+R-1 (wrow has +16 t)
-        const uint32_t *q0 = reinterpret_cast<const uint32_t *>(wrow0 + kl * 64 - 16 * t) + t * R;
-        const uint32_t *q1 = reinterpret_cast<const uint32_t *>(wrow1 + kl * 64 - 16 * t) + t * R;
-#pragma unroll
-        for (int s = 0; s < 4; ++s) { w0s[s] = (s < R) ? q0[s] : 0u; w1s[s] = (s < R) ? q1[s] : 0u; }
-    }
     float s0s[4 / SPP], s1s[4 / SPP];
     if constexpr (!PARTIALS) {
         if constexpr (SPP == 4) {
             const int gi = (int)(((long long)kb * kBlockK) / p.group);
             s0s[0] = reinterpret_cast<const float *>(srow0)[gi];
             s1s[0] = reinterpret_cast<const float *>(srow1)[gi];
+        } else if constexpr (SPP == 2) {   // staged rows are 16-byte aligned: 8-byte loads are fine
+            const float2 v0 = reinterpret_cast<const float2 *>(srow0)[kl];
+            const float2 v1 = reinterpret_cast<const float2 *>(srow1)[kl];
+            s0s[0] = v0.x; s0s[1] = v0.y; s1s[0] = v1.x; s1s[1] = v1.y;
         } else {
-            constexpr int SPB = 4 / SPP;
-#pragma unroll
-            for (int j = 0; j < SPB; ++j) {
-                s0s[j] = (j * SPP < R) ? reinterpret_cast<const float *>(srow0)[kl * SPB + j] : 0.f;
-                s1s[j] = (j * SPP < R) ? reinterpret_cast<const float *>(srow1)[kl * SPB + j] : 0.f;
-            }
+            const float4 v0 = reinterpret_cast<const float4 *>(srow0)[kl];
+            const float4 v1 = reinterpret_cast<const float4 *>(srow1)[kl];
+            s0s[0] = v0.x; s0s[1] = v0.y; s0s[2] = v0.z; s0s[3] = v0.w;
+            s1s[0] = v1.x; s1s[1] = v1.y; s1s[2] = v1.z; s1s[3] = v1.w;
         }
     }
 #pragma unroll
@@ -214,7 +177,6 @@ __global__ void __launch_bounds__(kDecodeThreads, (MT == 1 ? 7 : (MT == 2 ? 5 : 
 w2a8_decode_kernel(const DecodeParams p) {
     constexpr int KS = kDecodeWarps / TG;
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) unsigned long long bars[kPhases];
     __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, t = lane & 3;
@@ -228,69 +190,56 @@ w2a8_decode_kernel(const DecodeParams p) {
     const int nb = kb_end - kb_begin;
     const int m0 = blockIdx.z * (8 * MT);
     const int mrows = min(8 * MT, p.M - m0);
-    unsigned char *sm_w = smem;                 // [TG * 16][w_stride]
-    unsigned char *sm_s = smem + p.off_s;       // [TG * 16][s_stride]
+    unsigned char *sm_s = smem;                 // [TG * 16][s_stride]
     unsigned char *acts = smem + p.off_a;       // [mrows + 1][act_stride]
     W2A8_TRACE_POINT(0);
 
-    // The chunk is fetched in kPhases pieces along K, one mbarrier each.  Piece 0
-    // is requested before the dependency wait; the activations are requested
-    // next (right behind piece 0 in the memory queues, so compute can start while
-    // the rest streams in); the remaining pieces follow.
-    const int nbp = (nb + kPhases - 1) / kPhases;                 // blocks per piece
-    const int words_end = min(16 * kb_end, p.words_per_row);      // last block may be short
     constexpr int SPB = 4 / SPP;                                  // scales per block and channel
     const int sc_begin = (SPP == 4) ? 0 : SPB * kb_begin;
     const int sc_end = (SPP == 4) ? p.G : min(SPB * kb_end, p.G);
-    // scale rows go by bulk copy only where every piece is a whole number of 16-byte
-    // units (the host has checked the row pitch and the chunk starts); SPP == 1 only
-    const bool sbulk = (!PARTIALS) && (SPP == 1) && p.s_bulk;
     const int tiles_here = min(TG, p.N / 16 - blockIdx.x * TG);
     const int rows_here = tiles_here * 16;
 
-    auto post_piece = [&](int ph) {   // executed by warp 0
-        const int b0 = min(ph * nbp, nb), b1 = min((ph + 1) * nbp, nb);
-        const int w0 = 16 * (kb_begin + b0), w1 = min(16 * (kb_begin + b1), words_end);
-        const unsigned wbytes = w1 > w0 ? (unsigned)(w1 - w0) * 4u : 0u;
-        const int s0 = SPB * (kb_begin + b0), s1 = min(SPB * (kb_begin + b1), p.G);
-        const unsigned sbytes = (sbulk && s1 > s0) ? (unsigned)(s1 - s0) * 4u : 0u;
-        const uint32_t bar = smem_u32(&bars[ph]);
-        unsigned tx = 0;
-        for (int r = lane; r < rows_here; r += 32) {
-            const size_t row = (size_t)blockIdx.x * TG * 16 + r;
-            if (wbytes) {
-                bulk_g2s(smem_u32(sm_w + r * p.w_stride) + (unsigned)(w0 - 16 * kb_begin) * 4u,
-                         p.packed + row * p.words_per_row + w0, wbytes, bar);
-                tx += wbytes;
-            }
-            if (sbytes) {
-                bulk_g2s(smem_u32(sm_s + r * p.s_stride) + (unsigned)(s0 - sc_begin) * 4u,
-                         p.w_scale + row * p.G + s0, sbytes, bar);
-                tx += sbytes;
+    // this lane's weight words of up to kRound cells: [cell][channel gq / gq+8][slice]
+    uint32_t wreg[kRound][2][4];
+    auto request_cell = [&](int j, int kl) {
+        const int kb = kb_begin + kl;
+        const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const uint32_t *wp = p.packed + (size_t)(n0 + gq + 8 * r) * p.words_per_row + 16 * kb;
+            if (R == 4) {
+                const uint4 v = ld_stream_v4(wp + 4 * t);
+                wreg[j][r][0] = v.x; wreg[j][r][1] = v.y; wreg[j][r][2] = v.z; wreg[j][r][3] = v.w;
+            } else {   // trailing block with fewer slices: words t*R .. t*R+R-1
+#pragma unroll
+                for (int s2 = 0; s2 < 4; ++s2) wreg[j][r][s2] = (s2 < R) ? __ldg(wp + t * R + s2) : 0u;
             }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) tx += __shfl_xor_sync(0xFFFFFFFFu, tx, o);
-        if (lane == 0) mbar_arrive_expect_tx(bar, tx);
     };
 
-    // ---- piece 0 and the scales that cannot go by bulk copy (all independent of
-    //      the previous kernel) ---------------------------------------------------
-    if (warp == 0) {
-        if (lane == 0) {
+    // ---- first half of the first round, and the scales of the whole chunk (all
+    //      independent of the previous kernel) ------------------------------------
+    if (tile_ok) {
 #pragma unroll
-            for (int ph = 0; ph < kPhases; ++ph) mbar_init(smem_u32(&bars[ph]), 1);
-            mbar_fence_init();
-        }
-        __syncwarp();
-        post_piece(0);
+        for (int j = 0; j < kRound / 2; ++j)
+            if (ks + j * KS < nb) request_cell(j, ks + j * KS);
     }
-    if ((!PARTIALS) && !sbulk) {
+    if constexpr (!PARTIALS) {
         const int nsc = sc_end - sc_begin;
-        for (int u = threadIdx.x; u < rows_here * nsc; u += kDecodeThreads) {
-            const int r = u / nsc, j = u % nsc;
-            cp_async4(smem_u32(sm_s + r * p.s_stride + 4 * j),
-                      p.w_scale + ((size_t)blockIdx.x * TG * 16 + r) * p.G + sc_begin + j);
+        if (p.s_vec && (nsc % 4 == 0)) {
+            const int nu = nsc / 4;
+            for (int u = threadIdx.x; u < rows_here * nu; u += kDecodeThreads) {
+                const int r = u / nu, j = u % nu;
+                cp_async16(smem_u32(sm_s + r * p.s_stride + 16 * j),
+                           p.w_scale + ((size_t)blockIdx.x * TG * 16 + r) * p.G + sc_begin + 4 * j);
+            }
+        } else {
+            for (int u = threadIdx.x; u < rows_here * nsc; u += kDecodeThreads) {
+                const int r = u / nsc, j = u % nsc;
+                cp_async4(smem_u32(sm_s + r * p.s_stride + 4 * j),
+                          p.w_scale + ((size_t)blockIdx.x * TG * 16 + r) * p.G + sc_begin + j);
+            }
         }
     }
     W2A8_TRACE_POINT(1);
@@ -313,13 +262,14 @@ w2a8_decode_kernel(const DecodeParams p) {
         }
         cp_async_commit();
     }
-    // ---- the remaining pieces -----------------------------------------------------
-    if (warp == 0) {
+    // ---- second half of the first round ---------------------------------------------
+    if (tile_ok) {
 #pragma unroll
-        for (int ph = 1; ph < kPhases; ++ph) post_piece(ph);
+        for (int j = kRound / 2; j < kRound; ++j)
+            if (ks + j * KS < nb) request_cell(j, ks + j * KS);
     }
     cp_async_wait_all();
-    __syncthreads();   // activations and fallback scales staged; barriers initialised
+    __syncthreads();   // scales and activations staged
     W2A8_TRACE_POINT(3);
 
     float acc[MT][4];
@@ -329,36 +279,29 @@ w2a8_decode_kernel(const DecodeParams p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) { acc[mt][i] = 0.f; D[mt][i] = kMagicInt; }
 
-    bool timed_out = false;
     if (tile_ok) {
         const unsigned char *brow[MT];   // this lane's token row of each slab (or the zero row)
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
             brow[mt] = acts + ((8 * mt + gq < mrows) ? (8 * mt + gq) : mrows) * p.act_stride + t * 16;
-        const unsigned char *wrow0 = sm_w + (tl * 16 + gq) * p.w_stride + t * 16;
-        const unsigned char *wrow1 = wrow0 + 8 * p.w_stride;
         const unsigned char *srow0 = sm_s + (tl * 16 + gq) * p.s_stride;   // floats from sc_begin on
         const unsigned char *srow1 = srow0 + 8 * p.s_stride;
-        int phase_ready = -1;
-        for (int kl = ks; kl < nb; kl += KS) {
-            const int need = kl / nbp;
-            while (phase_ready < need) {
-                ++phase_ready;
-                if (!mbar_wait_bounded(smem_u32(&bars[phase_ready]), 0)) timed_out = true;
+        for (int kl0 = ks; kl0 < nb; kl0 += kRound * KS) {
+            if (kl0 != ks) {   // later rounds: request, then compute
+#pragma unroll
+                for (int j = 0; j < kRound; ++j)
+                    if (kl0 + j * KS < nb) request_cell(j, kl0 + j * KS);
             }
-            if (timed_out) break;
-            compute_cell<MT, SPP, ONE, PARTIALS>(p, wrow0, wrow1, srow0, srow1, brow, kl, kb_begin + kl,
-                                                 n0, m0, gq, t, acc, D);
+#pragma unroll
+            for (int j = 0; j < kRound; ++j) {
+                const int kl = kl0 + j * KS;
+                if (kl < nb)
+                    compute_cell<MT, SPP, ONE, PARTIALS>(p, wreg[j][0], wreg[j][1], srow0, srow1, brow,
+                                                         kl, kb_begin + kl, n0, m0, gq, t, acc, D);
+            }
         }
     }
     W2A8_TRACE_POINT(5);
-
-    // Nobody may leave while bulk copies into this CTA's shared memory are in
-    // flight: every thread passes every barrier (bounded) before the CTA retires.
-#pragma unroll
-    for (int ph = 0; ph < kPhases; ++ph)
-        if (!mbar_wait_bounded(smem_u32(&bars[ph]), 0)) timed_out = true;
-    if (timed_out) atomicExch(p.status, W2A8_ERR_TIMEOUT);
 
     if constexpr (!PARTIALS) {
         // ---- sum the K-lanes of each tile in a fixed order -----------------------
@@ -428,27 +371,21 @@ static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct DecodePlan {
     int mt, tg, chunks, blocks_per_chunk, slabs, groups;
-    int w_stride, s_stride, act_stride, off_s, off_a, s_bulk;
+    int s_stride, act_stride, off_a, s_vec;
     size_t smem;
 };
 
 // Shared-memory footprint of a CTA that stages `nb` blocks of K.
-static void plan_smem(DecodePlan &pl, int M, int K, int G, int spp, int nb) {
+static void plan_smem(DecodePlan &pl, int M, int G, int spp, int nb) {
     const int mrows = M < 8 * pl.mt ? M : 8 * pl.mt;
-    // weight rows: 64 bytes per block; stride = 64 mod 128 keeps the 8 channel
-    // rows of a quarter-warp LDS.128 on distinct banks
-    int wseg = nb * 64;
-    pl.w_stride = round_up(wseg, 128) + 64;
-    // scale rows: stride = 16 mod 128 spreads the 8 channels of a warp read
+    // scale rows: stride = 16 mod 128 spreads the 8 channels of a warp read over the banks
     const int nsc = spp == 4 ? G : (4 / spp) * nb;
     pl.s_stride = round_up(nsc * 4, 128) + 16;
     pl.act_stride = nb * kBlockK + kActPad;
-    pl.off_s = pl.tg * 16 * pl.w_stride;
-    pl.off_a = round_up(pl.off_s + pl.tg * 16 * pl.s_stride, 128);
+    pl.off_a = round_up(pl.tg * 16 * pl.s_stride, 128);
     const size_t act = (size_t)(mrows + 1) * pl.act_stride;
     const size_t red = (size_t)kDecodeWarps * pl.mt * 4 * 32 * sizeof(float);
     pl.smem = pl.off_a + (act > red ? act : red);
-    (void)K;
 }
 
 // Tiles per CTA and K-chunks.  One tile per CTA (4 K-lanes) keeps each warp's
@@ -467,7 +404,7 @@ static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
     int chunks = 1;
     for (;;) {   // smallest chunk count whose staging fits the budget
         const int bpc = (si.blocks + chunks - 1) / chunks;
-        plan_smem(pl, M, K, si.G, si.spp, bpc);
+        plan_smem(pl, M, si.G, si.spp, bpc);
         if ((int)pl.smem <= kSmemBudget || bpc == 1) break;
         ++chunks;
     }
@@ -478,14 +415,16 @@ static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
         // fewer than ~2 CTAs per SM: split K further while each K-lane keeps >= 1 block
         while ((long long)pl.groups * pl.slabs * chunks < 296 && (si.blocks / (chunks * 2)) >= ks)
             chunks *= 2;
+        // at most two rounds of kRound cells per warp: the second round's loads are exposed
+        while ((si.blocks + chunks - 1) / chunks > 2 * kRound * ks && chunks < si.blocks) ++chunks;
     }
     if (chunks > si.blocks) chunks = si.blocks;
     pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
     pl.chunks = (si.blocks + pl.blocks_per_chunk - 1) / pl.blocks_per_chunk;
-    plan_smem(pl, M, K, si.G, si.spp, pl.blocks_per_chunk);
-    // bulk-copy granularity for scales (group 64 only: four floats per block): the
-    // row pitch must be a multiple of 16 bytes
-    pl.s_bulk = (si.spp == 1) && (si.G % 4 == 0) && (K % 256 == 0);
+    plan_smem(pl, M, si.G, si.spp, pl.blocks_per_chunk);
+    // scale rows can be copied in 16-byte units when row pitch and chunk starts allow
+    const int spb = si.spp == 4 ? 0 : 4 / si.spp;
+    pl.s_vec = (si.spp != 4) && (si.G % 4 == 0) && ((spb * pl.blocks_per_chunk) % 4 == 0);
     return pl;
 }
 
@@ -554,8 +493,8 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
     p.M = M; p.N = N; p.K = K; p.G = si.G; p.group = group;
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
     p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;
-    p.w_stride = pl.w_stride; p.s_stride = pl.s_stride; p.act_stride = pl.act_stride;
-    p.off_s = pl.off_s; p.off_a = pl.off_a; p.s_bulk = pl.s_bulk;
+    p.s_stride = pl.s_stride; p.act_stride = pl.act_stride;
+    p.off_a = pl.off_a; p.s_vec = pl.s_vec;
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
     char *base = reinterpret_cast<char *>(workspace);
     p.status = reinterpret_cast<int *>(base);
