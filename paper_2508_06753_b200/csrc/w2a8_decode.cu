@@ -286,18 +286,17 @@ w2a8_decode_kernel(const DecodeParams p) {
             brow[mt] = acts + ((8 * mt + gq < mrows) ? (8 * mt + gq) : mrows) * p.act_stride + t * 16;
         const unsigned char *srow0 = sm_s + (tl * 16 + gq) * p.s_stride;   // floats from sc_begin on
         const unsigned char *srow1 = srow0 + 8 * p.s_stride;
+        // Software pipeline over rounds: as soon as a cell has been consumed, its
+        // registers take the weights of the same slot of the next round.
         for (int kl0 = ks; kl0 < nb; kl0 += kRound * KS) {
-            if (kl0 != ks) {   // later rounds: request, then compute
-#pragma unroll
-                for (int j = 0; j < kRound; ++j)
-                    if (kl0 + j * KS < nb) request_cell(j, kl0 + j * KS);
-            }
 #pragma unroll
             for (int j = 0; j < kRound; ++j) {
                 const int kl = kl0 + j * KS;
-                if (kl < nb)
+                if (kl < nb) {
                     compute_cell<MT, SPP, ONE, PARTIALS>(p, wreg[j][0], wreg[j][1], srow0, srow1, brow,
                                                          kl, kb_begin + kl, n0, m0, gq, t, acc, D);
+                    if (kl + kRound * KS < nb) request_cell(j, kl + kRound * KS);
+                }
             }
         }
     }
@@ -412,11 +411,16 @@ static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
     if (forced > 0) {
         if (forced > chunks) chunks = forced;
     } else {
-        // fewer than ~2 CTAs per SM: split K further while each K-lane keeps >= 1 block
-        while ((long long)pl.groups * pl.slabs * chunks < 296 && (si.blocks / (chunks * 2)) >= ks)
+        // Measured on B200: a warp should hold all its cells in one round (its later
+        // rounds wait a full memory latency each), and the whole grid should field
+        // about 2000 warps or more so that enough loads are in flight; beyond that
+        // the cross-CTA sum costs more than further splitting gains.
+        const int one_round = (si.blocks + kRound * ks - 1) / (kRound * ks);
+        if (one_round > chunks) chunks = one_round;
+        const int min_warps = env_int("W2A8_MIN_WARPS", 2000);
+        while ((long long)pl.groups * pl.slabs * kDecodeWarps * chunks < min_warps &&
+               (si.blocks / (chunks * 2)) >= ks)
             chunks *= 2;
-        // at most two rounds of kRound cells per warp: the second round's loads are exposed
-        while ((si.blocks + chunks - 1) / chunks > 2 * kRound * ks && chunks < si.blocks) ++chunks;
     }
     if (chunks > si.blocks) chunks = si.blocks;
     pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
