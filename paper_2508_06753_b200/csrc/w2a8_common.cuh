@@ -29,8 +29,11 @@ constexpr int kMagicInt = 0x4B400000;
 constexpr float kMagicFloat = 12582912.0f;
 
 __device__ __forceinline__ uint32_t lane_codes(uint32_t word, int j) {
-    // j is a compile-time constant after unrolling
-    return (((j == 3) ? word : (word << (6 - 2 * j))) & kTopMask) ^ kSignFlip;
+    // j is a compile-time constant after unrolling; (x & mask) ^ flip is one LOP3 (LUT 0x6A)
+    const uint32_t x = (j == 3) ? word : (word << (6 - 2 * j));
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(r) : "r"(x), "r"(kTopMask), "r"(kSignFlip));
+    return r;
 }
 
 // Programmatic dependent launch: wait until the previous kernel of the stream

@@ -227,19 +227,16 @@ w2a8_decode_kernel(const DecodeParams p) {
     }
     if constexpr (!PARTIALS) {
         const int nsc = sc_end - sc_begin;
+        const float *sbase = p.w_scale + (size_t)blockIdx.x * TG * 16 * p.G + sc_begin;
         if (p.s_vec && (nsc % 4 == 0)) {
             const int nu = nsc / 4;
-            for (int u = threadIdx.x; u < rows_here * nu; u += kDecodeThreads) {
-                const int r = u / nu, j = u % nu;
-                cp_async16(smem_u32(sm_s + r * p.s_stride + 16 * j),
-                           p.w_scale + ((size_t)blockIdx.x * TG * 16 + r) * p.G + sc_begin + 4 * j);
-            }
+            for (int r = warp; r < rows_here; r += kDecodeWarps)
+                for (int j = lane; j < nu; j += 32)
+                    cp_async16(smem_u32(sm_s + r * p.s_stride + 16 * j), sbase + (size_t)r * p.G + 4 * j);
         } else {
-            for (int u = threadIdx.x; u < rows_here * nsc; u += kDecodeThreads) {
-                const int r = u / nsc, j = u % nsc;
-                cp_async4(smem_u32(sm_s + r * p.s_stride + 4 * j),
-                          p.w_scale + ((size_t)blockIdx.x * TG * 16 + r) * p.G + sc_begin + j);
-            }
+            for (int r = warp; r < rows_here; r += kDecodeWarps)
+                for (int j = lane; j < nsc; j += 32)
+                    cp_async4(smem_u32(sm_s + r * p.s_stride + 4 * j), sbase + (size_t)r * p.G + j);
         }
     }
     W2A8_TRACE_POINT(1);
