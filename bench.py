@@ -33,6 +33,10 @@ from paper_2508_06753_b200 import synth
 CFG_INDEX = 1
 METRIC = "W2A8 GEMM HBM GB/s at M=1-16 (Llama-3-8B decoder-layer linears, M in {1,4,16}, group 64)"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode kernel on the
+# 4096x14336, M=1, group-64 GEMM (ncu capture summarised in profiles/decode_gate_m1_ncu.md);
+# the algorithmic bytes of that launch are 18,411,524.
+NCU_TRAFFIC_BYTES_GATE_M1 = 18_397_440
 
 
 # --------------------------------------------------------------------- accounting
@@ -396,15 +400,23 @@ class OracleWorkload:
         return float(min(1.0, max(1.0 / 896, (1.0 / 64) * seconds_per_step / max(dt, 1e-6))))
 
 
-def cpu_baseline(cfg, budget_s=20.0):
+def cpu_baseline(cfg, budget_s=20.0, min_wall_s=1.5):
     """The reference as it stands on this machine's host cores, on a bounded
-    sample (about `budget_s` seconds) of the benchmark workload."""
+    sample of the benchmark workload: whole steps (restricted to a leading
+    fraction of the output channels if one step alone would exceed `budget_s`),
+    repeated until about `min_wall_s` seconds of wall time have been measured."""
     w = OracleWorkload(cfg)
     frac = w.frac_for(budget_s)
-    nbytes, dt = w.step(frac)
-    return dict(value=nbytes / dt / 1e9, unit="GB/s", cores=w.oracle.num_threads(), kind="oracle",
-                seconds=dt,
-                sample=f"one step (M in {cfg['Ms']}, 4 quantise + 7 GEMM calls each) restricted to "
+    tot_b, tot_s, n = 0, 0.0, 0
+    while tot_s < min_wall_s and n < 64:
+        nbytes, dt = w.step(frac)
+        tot_b += nbytes
+        tot_s += dt
+        n += 1
+    cores = w.oracle.num_threads()
+    return dict(value=tot_b / tot_s / 1e9, unit="GB/s", cores=cores, kind="oracle",
+                seconds=tot_s, cpu_core_seconds=tot_s * cores,
+                sample=f"{n} step(s) (M in {cfg['Ms']}, 4 quantise + 7 GEMM calls each) restricted to "
                        f"the first {frac:.4f} of the output channels of every linear")
 
 
@@ -507,7 +519,7 @@ def run_ours(args):
 
     dom = probes[0]
     roofline = {"bound": "hbm", "achieved": dom["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": dom["gbs"] / peaks["hbm_gbs"], "traffic": None,
+                "frac": dom["gbs"] / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES_GATE_M1,
                 "peak_source": peaks["source"],
                 "kernel": "w2a8_decode_kernel<MT=1,SPP=1> on gate/up 4096x14336, M=1",
                 "bytes_per_launch": dom["bytes_per_launch"], "us_per_launch": dom["us_per_launch"],
