@@ -161,6 +161,41 @@ int w2a8_linear_host(const void *x_host, int M, int K, const uint32_t *packed,
                      const float *w_scale, int N, int group, float *y_host,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * w2a8_gemm_static -- w2a8_gemm without a workspace argument.  (The paper has no
+ * counterpart; this entry exists for integration reasons only.)
+ *
+ * Who needs it: callers that are not in a position to allocate device memory
+ * and have no workspace to pass -- for instance a serving runtime that handed
+ * the whole GPU to its own memory pool at start-up, a custom-operator slot that
+ * only receives input and output pointers, or a latency-critical loop in which
+ * an allocation (and the implicit synchronisation it can bring) is forbidden.
+ * For them the scratch of the kernel (status word, split-K arrival counters and
+ * split-K partial outputs) is a fixed array of W2A8_STATIC_SCRATCH_BYTES bytes
+ * inside the library image.  Every GPU that loads the library holds that array
+ * until the process exits.  The call performs no cudaMalloc / cudaFree and calls
+ * no allocating library routine.
+ *
+ * Arguments and result: exactly those of w2a8_gemm (same kernel, same launch
+ * configuration, same bits in y).  Problems whose scratch need
+ * (w2a8_workspace_bytes) exceeds W2A8_STATIC_SCRATCH_BYTES are refused with
+ * W2A8_ERR_WORKSPACE; nothing is launched.
+ *
+ * First use on a device: the first call made while a given device is current
+ * looks up the device address of the array (a host-side query, no allocation).
+ * Make that first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the same array, which keeps the contents
+ * the previous call left; each call clears the part that must start at zero
+ * (on `stream`, before the kernel).  Two calls that can overlap on the device
+ * (different streams, or different host threads on different streams) race on
+ * it and give undefined results: keep such calls on one stream, or use
+ * w2a8_gemm with separate workspaces.
+ */
+#define W2A8_STATIC_SCRATCH_BYTES (8u << 20)
+int w2a8_gemm_static(const int8_t *a, const float *a_scale, const uint32_t *packed,
+                     const float *w_scale, float *y, int M, int N, int K, int group, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libw2a8.so")
 EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
-    "w2a8_linear_host_workspace_bytes", "w2a8_linear_host",
+    "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
 ]
 
 _lib = None
@@ -56,8 +56,9 @@ def lib() -> ctypes.CDLL:
         L.w2a8_linear_host_workspace_bytes.restype = sz
         L.w2a8_linear_host_workspace_bytes.argtypes = [i, i, i, i]
         L.w2a8_linear_host.argtypes = [vp, i, i, vp, vp, i, i, vp, vp, sz, vp]
+        L.w2a8_gemm_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp]
         for name in ("w2_pack", "a8_quantize", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm",
-                     "w2a8_gemm_partials", "w2a8_linear_host"):
+                     "w2a8_gemm_partials", "w2a8_linear_host", "w2a8_gemm_static"):
             getattr(L, name).restype = i
         _lib = L
     return _lib
@@ -172,3 +173,21 @@ def w2a8_linear_host(x_host: torch.Tensor, packed: torch.Tensor, w_scale: torch.
                                   workspace.numel() * workspace.element_size(), _stream(stream)),
            "w2a8_linear_host")
     return y_host
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def w2a8_gemm_static(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor,
+                     w_scale: torch.Tensor, group: int, y: torch.Tensor | None = None, stream=None):
+    """w2a8_gemm for callers with no workspace to give: the kernel's scratch is a fixed
+    array inside the library (at most STATIC_SCRATCH_BYTES; larger problems raise), so
+    nothing is allocated on the library side.  Calls share that array: keep them on one
+    stream.  See w2a8_gemm_static in include/w2a8.h."""
+    M, K = a.shape
+    N = packed.shape[0]
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=a.device)
+    _check(lib().w2a8_gemm_static(_ptr(a), _ptr(a_scale), _ptr(packed), _ptr(w_scale), _ptr(y), M, N, K,
+                                  group, _stream(stream)), "w2a8_gemm_static")
+    return y

@@ -440,6 +440,13 @@ size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si) {
     return kStatusBytes + counters + part;
 }
 
+// Bytes at the start of the workspace that must be zero before a launch: the
+// status word and the arrival counters.
+size_t decode_workspace_header_bytes(int M, int N, int K, const ShapeInfo &si) {
+    const DecodePlan pl = decode_plan(M, N, K, si);
+    return kStatusBytes + ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
+}
+
 template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
 static cudaError_t launch_decode_inst(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
     static bool configured = false;   // one attribute call per instantiation and process

@@ -20,6 +20,7 @@ def lib():
 def _declared_functions():
     text = open(os.path.join(ROOT, "include", "w2a8.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"^\s*#.*$", "", text, flags=re.M)      # preprocessor lines
     names = re.findall(r"\b([A-Za-z_][A-Za-z0-9_]*)\s*\([^;{}]*\)\s*;", text)
     return sorted(set(names))
 
