@@ -11,6 +11,10 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st);
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
+bool prefill_supported(int M, int N, int K, int group);
+int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const float *w_scale,
+                   float *y, int32_t *partials, int M, int N, int K, int group, int *status,
+                   cudaStream_t st);
 
 int env_int(const char *name, int dflt) {
     const char *v = getenv(name);
@@ -208,6 +212,10 @@ static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *pa
     const size_t need = decode_workspace_bytes(M, N, K, si);
     if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
     if (int st = check_device()) return st;
+    // many tokens: tensor-core path (tcgen05); few tokens, or shapes it does not tile: streaming path
+    if (prefill_supported(M, N, K, group) && env_int("W2A8_PREFILL", 1) != 0)
+        return launch_prefill(a, a_scale, packed, w_scale, y, partials, M, N, K, group,
+                              reinterpret_cast<int *>(workspace), (cudaStream_t)stream);
     return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,
                          (cudaStream_t)stream);
 }

@@ -1,0 +1,403 @@
+// Compute-bound W2A8 kernel for many tokens (prefill): 5th-generation tensor
+// cores (tcgen05.mma kind::i8) with accumulators in tensor memory.  It is the
+// sm_100a counterpart of the paper's fused GEMM for the compute-bound case
+// (Sec. II-D: tiles of the output, low-bit weights fed to the matrix unit,
+// int32 -> float dequantisation in registers), with the 2-bit -> int8
+// up-convert of Sec. II-C done into shared memory because the tensor core has
+// no 2-bit operand type.
+//
+// One CTA computes a 128-channel x 128-token tile of y.
+//   A operand (UMMA M = 128): weights.  Two "unpack" warps read the packed words
+//     of 128 channels x one 256-k block, expand them to int8 lanes (value
+//     64 * (code - 2): one shift + one LOP3 per four weights) and store them
+//     K-major with the 128-byte swizzle the tensor core expects.
+//   B operand (UMMA N = 128): int8 activations, 128 tokens x 256 k, brought by TMA
+//     with the same swizzle.
+//   D: int32 in tensor memory, lane = channel, column = token.  Because a lane is
+//     a channel, a drain thread needs one weight scale per group, not one per value.
+// Per 64-k group (or whatever the scale group is) the MMA warp issues K = 32
+// steps into one of two accumulator buffers; four "drain" warps read the other
+// buffer with tcgen05.ld, convert to fp32 and accumulate scale * value in
+// registers (128 fp32 per thread).  Every wait on an mbarrier is bounded; a wait
+// that gives up sets the status word of the workspace and the CTA winds down.
+#include <cuda.h>
+
+#include "w2a8_common.cuh"
+
+namespace w2a8 {
+
+constexpr int kPfThreads = 256;          // 8 warps: TMA, MMA, 2 unpack, 4 drain
+constexpr int kPfBM = 128;               // channels per tile (UMMA M)
+constexpr int kPfBN = 128;               // tokens per tile (UMMA N)
+constexpr int kPfBK = 256;               // k per stage = one W2P block
+constexpr int kPfStages = 3;
+constexpr int kPfHalfBytes = 128 * 128;  // one [128 rows][128 B] swizzled sub-tile
+constexpr int kPfStageBytes = 4 * kPfHalfBytes;   // A: 2 halves, B: 2 halves
+constexpr int kPfTmemCols = 2 * kPfBN;   // two accumulator buffers
+constexpr unsigned kPfWaitPolls = 1u << 20;
+
+struct PrefillParams {
+    const uint32_t *packed;
+    const float *w_scale;
+    const float *a_scale;
+    float *y;
+    int32_t *partials;
+    int *status;
+    int M, N, K, G, group;
+    int words_per_row;
+    int slices_per_group;    // group / 64
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------
+__device__ __forceinline__ uint32_t pf_smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void pf_mbar_init(uint32_t bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void pf_mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void pf_mbar_arrive_expect_tx(uint32_t bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool pf_mbar_try_wait(uint32_t bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; also gives up as soon as another role has raised the abort flag.
+__device__ __forceinline__ bool pf_wait(uint32_t bar, unsigned parity, volatile int *abort_flag) {
+    for (unsigned i = 0; i < kPfWaitPolls; ++i) {
+        if (pf_mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 63u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void pf_tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void pf_fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void pf_tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void pf_tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void pf_tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void pf_tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void pf_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// mbarrier arrive once all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void pf_mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void pf_tmem_ld32(uint32_t taddr, int (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void pf_tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major [rows][128 B] tile stored with the
+// 128-byte swizzle: start address, 8-row stride of 1024 B, descriptor version 1,
+// layout type 2 (128-byte swizzle).  A K step of 32 bytes inside the 128-byte row
+// is taken by adding 32 to the start address.
+__device__ __forceinline__ uint64_t pf_smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);            // bits 0-13: start address / 16
+    d |= (uint64_t)1 << 16;                              // bits 16-29: leading byte offset / 16 (unused here)
+    d |= (uint64_t)(1024 >> 4) << 32;                    // bits 32-45: stride byte offset / 16
+    d |= (uint64_t)1 << 46;                              // bits 46-47: descriptor version
+    d |= (uint64_t)2 << 61;                              // bits 61-63: 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: int32 accumulate, signed 8-bit A and B, both K-major, M x N.
+__host__ __device__ constexpr uint32_t pf_instr_desc(int m, int n) {
+    return (2u << 4)                      // D format: S32
+         | (1u << 7) | (1u << 10)         // A, B format: signed 8-bit
+         | ((uint32_t)(n >> 3) << 17)     // N / 8
+         | ((uint32_t)(m >> 4) << 24);    // M / 16
+}
+
+template <bool PARTIALS>
+__global__ void __launch_bounds__(kPfThreads, 1)
+w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillParams p) {
+    extern __shared__ unsigned char pf_smem_raw[];
+    __shared__ __align__(8) unsigned long long bar_full_a[kPfStages], bar_full_b[kPfStages], bar_empty[kPfStages];
+    __shared__ __align__(8) unsigned long long bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+    __shared__ float a_scale_s[kPfBN];
+    volatile int *abort_flag = &abort_flag_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * kPfBM;      // first channel of the tile
+    const int m0 = blockIdx.y * kPfBN;      // first token of the tile
+    const int nstages_total = p.K / kPfBK;
+    const int dps = p.slices_per_group;     // 64-k slices between two drains
+    // stage buffers, 1024-byte aligned (swizzle atom = 8 rows x 128 B)
+    const uint32_t smem_base = (pf_smem_u32(pf_smem_raw) + 1023u) & ~1023u;
+    unsigned char *smem_gen = pf_smem_raw + (smem_base - pf_smem_u32(pf_smem_raw));
+
+    if (threadIdx.x == 0) {
+        abort_flag_s = 0;
+        for (int s = 0; s < kPfStages; ++s) {
+            pf_mbar_init(pf_smem_u32(&bar_full_a[s]), 2);     // one arrive per unpack warp
+            pf_mbar_init(pf_smem_u32(&bar_full_b[s]), 1);     // TMA producer + transaction bytes
+            pf_mbar_init(pf_smem_u32(&bar_empty[s]), 1);      // tcgen05.commit
+        }
+        for (int b = 0; b < 2; ++b) {
+            pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);   // tcgen05.commit
+            pf_mbar_init(pf_smem_u32(&bar_acc_empty[b]), 4);  // one arrive per drain warp
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        pf_fence_proxy_async();
+    }
+    if (warp == 1) pf_tmem_alloc(pf_smem_u32(&tmem_base_slot), kPfTmemCols);
+    if (threadIdx.x < kPfBN) {
+        const int m = m0 + threadIdx.x;
+        a_scale_s[threadIdx.x] = (!PARTIALS && m < p.M) ? p.a_scale[m] * (1.0f / kCodeGain) : 0.f;
+    }
+    pf_tc_fence_before();
+    __syncthreads();
+    pf_tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // ===== TMA producer: activations, 128 tokens x 256 k per stage ==============
+        if (lane == 0) {
+            for (int it = 0; it < nstages_total; ++it) {
+                const int s = it % kPfStages, round = it / kPfStages;
+                if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
+                const uint32_t bar = pf_smem_u32(&bar_full_b[s]);
+                const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
+                pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
+                pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
+                pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
+            }
+        }
+    } else if (warp == 1) {
+        // ===== MMA issuer (one thread) ================================================
+        if (lane == 0) {
+            constexpr uint32_t idesc = pf_instr_desc(kPfBM, kPfBN);
+            int slice_idx = 0;          // 64-k slices issued so far
+            int buf = 0, buf_uses[2] = {0, 0};
+            bool ok = true;
+            for (int it = 0; it < nstages_total && ok; ++it) {
+                const int s = it % kPfStages, round = it / kPfStages;
+                ok = pf_wait(pf_smem_u32(&bar_full_a[s]), round & 1, abort_flag) &&
+                     pf_wait(pf_smem_u32(&bar_full_b[s]), round & 1, abort_flag);
+                if (!ok) break;
+                pf_tc_fence_after();
+                const uint32_t a_base = smem_base + s * kPfStageBytes;
+                const uint32_t b_base = a_base + 2 * kPfHalfBytes;
+                for (int q = 0; q < 4 && ok; ++q, ++slice_idx) {
+                    const bool group_start = (slice_idx % dps) == 0;
+                    if (group_start && buf_uses[buf] > 0) {
+                        // the drain warps must have emptied this buffer's previous group
+                        ok = pf_wait(pf_smem_u32(&bar_acc_empty[buf]), (buf_uses[buf] - 1) & 1, abort_flag);
+                        if (!ok) break;
+                        pf_tc_fence_after();
+                    }
+                    const uint32_t half = (q >> 1) * kPfHalfBytes;
+#pragma unroll
+                    for (int ks = 0; ks < 2; ++ks) {
+                        const uint32_t koff = ((q & 1) * 2 + ks) * 32;
+                        pf_mma_i8(tmem_base + buf * kPfBN, pf_smem_desc(a_base + half + koff),
+                                  pf_smem_desc(b_base + half + koff), idesc,
+                                  (group_start && ks == 0) ? 0u : 1u);
+                    }
+                    if ((slice_idx + 1) % dps == 0) {
+                        pf_mma_commit(pf_smem_u32(&bar_acc_full[buf]));
+                        ++buf_uses[buf];
+                        buf ^= 1;
+                    }
+                }
+                pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
+            }
+        }
+    } else if (warp < 4) {
+        // ===== unpack warps: packed words -> int8 lanes, K-major, 128-byte swizzle =====
+        const int ut = (warp - 2) * 32 + lane;      // 0..63
+        for (int it = 0; it < nstages_total; ++it) {
+            const int s = it % kPfStages, round = it / kPfStages;
+            // request this stage's words before waiting for the buffer
+            uint4 w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int u = ut + 64 * i;          // unit index: row = u / 4, quarter t = u % 4
+                const int r = u >> 2, t = u & 3;
+                w[i] = __ldg(reinterpret_cast<const uint4 *>(p.packed + (size_t)(n0 + r) * p.words_per_row +
+                                                             16 * it + 4 * t));
+            }
+            if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
+            unsigned char *a_stage = smem_gen + s * kPfStageBytes;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int u = ut + 64 * i;
+                const int r = u >> 2, t = u & 3;
+                const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) {    // slice sl: k = 64 sl + 16 t .. + 15 of this block
+                    uint4 v;
+                    v.x = lane_codes(ws[sl], 0); v.y = lane_codes(ws[sl], 1);
+                    v.z = lane_codes(ws[sl], 2); v.w = lane_codes(ws[sl], 3);
+                    const int chunk = (4 * (sl & 1) + t) ^ (r & 7);
+                    *reinterpret_cast<uint4 *>(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16) = v;
+                }
+            }
+            pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
+            __syncwarp();
+            if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full_a[s]));
+        }
+    } else {
+        // ===== drain warps: TMEM -> registers, fp32 accumulate with the group scale ======
+        const int q4 = warp & 3;                    // TMEM lane quarter this warp may access
+        const int ch = q4 * 32 + lane;              // channel inside the tile = TMEM lane
+        const int n = n0 + ch;
+        float acc[kPfBN];
+#pragma unroll
+        for (int j = 0; j < kPfBN; ++j) acc[j] = 0.f;
+        const int ngroups = (p.K / 64) / dps;
+        int buf = 0, uses[2] = {0, 0};
+        bool ok = true;
+        for (int gi = 0; gi < ngroups && ok; ++gi) {
+            float sc = 0.f;
+            if (!PARTIALS) sc = __ldg(p.w_scale + (size_t)n * p.G + gi);
+            ok = pf_wait(pf_smem_u32(&bar_acc_full[buf]), uses[buf] & 1, abort_flag);
+            if (!ok) break;
+            pf_tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < kPfBN / 32; ++c) {
+                int v[32];
+                pf_tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + buf * kPfBN + c * 32, v);
+                pf_tmem_ld_wait();
+                if (c == kPfBN / 32 - 1) {
+                    // all of this buffer has been read: hand it back to the MMA warp
+                    pf_tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[buf]));
+                }
+                if (PARTIALS) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int m = m0 + c * 32 + j;
+                        if (m < p.M) p.partials[((size_t)m * p.N + n) * p.G + gi] = v[j] >> 6;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[c * 32 + j] = fmaf(sc, (float)v[j], acc[c * 32 + j]);
+                }
+            }
+            ++uses[buf];
+            buf ^= 1;
+        }
+        if (!PARTIALS && ok) {
+#pragma unroll
+            for (int j = 0; j < kPfBN; ++j) {
+                const int m = m0 + j;
+                if (m < p.M) p.y[(size_t)m * p.N + n] = acc[j] * a_scale_s[j];
+            }
+        }
+    }
+
+    // ---- wind down ---------------------------------------------------------------------
+    pf_tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, W2A8_ERR_TIMEOUT);
+    if (warp == 1) {
+        pf_tc_fence_after();
+        pf_tmem_dealloc(tmem_base, kPfTmemCols);
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+bool prefill_supported(int M, int N, int K, int group) {
+    if (M < 64) return false;
+    if (N % kPfBM != 0 || K % kPfBK != 0) return false;
+    if (!(group == 64 || group == 128 || group % 256 == 0)) return false;   // group == K implies K % 256 == 0 here
+    if ((long long)64 * 254 * group >= (1ll << 31)) return false;           // int32 accumulator range
+    return true;
+}
+
+// Enqueue the prefill kernel.  `partials` != nullptr selects the parity export.
+int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const float *w_scale,
+                   float *y, int32_t *partials, int M, int N, int K, int group, int *status,
+                   cudaStream_t st) {
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return W2A8_ERR_CUDA;
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)K};                 // bytes between tokens
+    const cuuint32_t box[2] = {128u, (cuuint32_t)kPfBN};          // 128 k x 128 tokens
+    const cuuint32_t estr[2] = {1u, 1u};
+    if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(a), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return W2A8_ERR_CUDA;
+    PrefillParams p;
+    p.packed = packed; p.w_scale = w_scale; p.a_scale = a_scale; p.y = y; p.partials = partials;
+    p.status = status;
+    p.M = M; p.N = N; p.K = K; p.G = K / group; p.group = group;
+    p.words_per_row = K / 16;
+    p.slices_per_group = group / 64;
+    const size_t smem = (size_t)kPfStages * kPfStageBytes + 1024;
+    dim3 grid(N / kPfBM, (M + kPfBN - 1) / kPfBN);
+    static bool configured[2] = {false, false};
+    cudaError_t e;
+    if (partials) {
+        if (!configured[1]) {
+            e = cudaFuncSetAttribute(w2a8_prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return W2A8_ERR_CUDA;
+            configured[1] = true;
+        }
+        w2a8_prefill_kernel<true><<<grid, kPfThreads, smem, st>>>(map, p);
+    } else {
+        if (!configured[0]) {
+            e = cudaFuncSetAttribute(w2a8_prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return W2A8_ERR_CUDA;
+            configured[0] = true;
+        }
+        w2a8_prefill_kernel<false><<<grid, kPfThreads, smem, st>>>(map, p);
+    }
+    return cudaGetLastError() == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
+}
+
+}  // namespace w2a8
