@@ -506,6 +506,9 @@ def run_ours(args):
         big = max(range(len(cfg["shapes"])), key=lambda i: cfg["shapes"][i][1] * cfg["shapes"][i][2])
         for M in cfg["Ms"]:
             probes.append(kernel_probe(rep, M, big))
+    prefill = None
+    if rank == 0 and not args.no_prefill:
+        prefill = prefill_probe(device, peaks)
     e2e_ms, h2d, d2h, _ = e2e_measure(rep, max(args.steps // 10, 10), 3)
     e2e_steps = max(args.steps // 10, 10)
     e2e_ms_all, e2e_units = aggregate(e2e_ms, step_bytes(cfg) * e2e_steps, device)
@@ -540,8 +543,67 @@ def run_ours(args):
         "clocks": clocks, "e2e": e2e,
         "gpu_launches": args.steps * len(cfg["Ms"]) * rep.kernels_per_pass,
         "roofline": roofline, "cpu_baseline": cpu, "per_m": per_m, "kernel_probes": probes,
+        "prefill": prefill,
     }
     print(json.dumps(out))
+
+
+def prefill_probe(device, peaks, Ms=(512, 2048, 8192), reps=5):
+    """Tensor-core path on the prefill configuration: Llama-3-8B gate/up (K=4096, N=14336)
+    and down (K=14336, N=4096), group 64.  int8 TOPS = 2*M*N*K / time, GEMM alone and
+    with the a8_quantize pass; CUDA events on the launching stream."""
+    import torch
+    from paper_2508_06753_b200 import binding as b
+    cfg = synth.CONFIGS[4]
+    int8_peak_burst = 2.0 * peaks["bf16_tflops"]            # nominal int8 : bf16 ratio is 2
+    int8_peak_sustained = 2.0 * peaks["bf16_tflops_sustained"]
+    rows = []
+    for idx, (name, K, N) in enumerate(cfg["shapes"]):
+        g = synth.config_group(cfg, K)
+        codes, s_w = synth.make_linear(synth.shape_seed(cfg, idx), K, N, g)
+        packed = b.w2_pack(torch.from_numpy(codes).to(device))
+        s_w_d = torch.from_numpy(s_w).to(device)
+        del codes
+        for M in Ms:
+            bits = synth.activations_bf16(cfg["seed"] + 7 + M, M, K)
+            x = torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+            a, s_a = b.a8_quantize(x)
+            y = torch.empty((M, N), dtype=torch.float32, device=device)
+            ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g), device=device)
+
+            def gemm():
+                b.w2a8_gemm(a, s_a, packed, s_w_d, g, ws, y)
+
+            def both():
+                b.a8_quantize(x, a, s_a)
+                b.w2a8_gemm(a, s_a, packed, s_w_d, g, ws, y)
+            out = {}
+            for label, fn in (("gemm", gemm), ("quantize+gemm", both)):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                out[label] = e0.elapsed_time(e1) / reps
+            ops = 2.0 * M * N * K
+            tops = ops / (out["gemm"] * 1e-3) / 1e12
+            rows.append({"shape": f"{K}x{N}", "M": M, "group": g, "ms_gemm": out["gemm"],
+                         "ms_quantize_gemm": out["quantize+gemm"], "tops": tops,
+                         "tops_with_quantize": ops / (out["quantize+gemm"] * 1e-3) / 1e12,
+                         "frac_of_measured_int8_burst": tops / int8_peak_burst,
+                         "frac_of_measured_int8_sustained": tops / int8_peak_sustained,
+                         "frac_of_nominal_4500": tops / 4500.0,
+                         "status": b.w2a8_workspace_status(ws)})
+            del x, a, y, ws
+        del packed
+    return {"unit": "int8 TOPS", "peak_measured_burst": int8_peak_burst,
+            "peak_measured_sustained": int8_peak_sustained,
+            "peak_note": "measured cuBLAS bf16 peak x 2 (nominal int8 : bf16 ratio); nominal dense int8 4500",
+            "rows": rows}
 
 
 def run_kernel_profile(args):
@@ -602,6 +664,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the tensor-core prefill probe")
+    ap.add_argument("--only-prefill", action="store_true", help="run only the prefill probe")
     ap.add_argument("--only-headline", action="store_true",
                     help="time the steps only (no per-M breakdown, kernel probe, e2e or CPU baseline); "
                          "short command for profilers")
@@ -612,6 +676,12 @@ def main():
     args = ap.parse_args()
     if args.profile_shape:
         run_kernel_profile(args)
+        return
+    if args.only_prefill:
+        import torch
+        from paper_2508_06753_b200 import build
+        build.build()
+        print(json.dumps(prefill_probe(torch.device("cuda", 0), load_peaks())))
         return
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
