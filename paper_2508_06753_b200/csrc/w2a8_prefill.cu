@@ -16,9 +16,9 @@
 //   D: int32 in tensor memory, lane = channel, column = token.  Because a lane is
 //     a channel, a drain thread needs one weight scale per group, not one per value.
 // Per 64-k group (or whatever the scale group is) the MMA warp issues K = 32
-// steps into one of two accumulator buffers; four "drain" warps read the other
+// steps into one of two accumulator buffers; the "drain" warps read the other
 // buffer with tcgen05.ld, convert to fp32 and accumulate scale * value in
-// registers (128 fp32 per thread).  Every wait on an mbarrier is bounded; a wait
+// registers (eight drain warps: two per TMEM lane quarter, 64 token columns each).  Every wait on an mbarrier is bounded; a wait
 // that gives up sets the status word of the workspace and the CTA winds down.
 #include <cuda.h>
 
@@ -26,14 +26,17 @@
 
 namespace w2a8 {
 
-constexpr int kPfThreads = 256;          // 8 warps: TMA, MMA, 2 unpack, 4 drain
+constexpr int kPfUnpackWarps = 2;
+constexpr int kPfThreads = 32 * (2 + kPfUnpackWarps + 8);   // warps: TMA, MMA, unpack, 8 drain
+constexpr int kPfDrainCols = 64;         // token columns per drain warp (two warps share a lane quarter)
 constexpr int kPfBM = 128;               // channels per tile (UMMA M)
 constexpr int kPfBN = 128;               // tokens per tile (UMMA N)
 constexpr int kPfBK = 256;               // k per stage = one W2P block
 constexpr int kPfStages = 3;
 constexpr int kPfHalfBytes = 128 * 128;  // one [128 rows][128 B] swizzled sub-tile
 constexpr int kPfStageBytes = 4 * kPfHalfBytes;   // A: 2 halves, B: 2 halves
-constexpr int kPfTmemCols = 2 * kPfBN;   // two accumulator buffers
+constexpr int kPfAccBufs = 4;             // accumulator buffers in tensor memory (groups in flight)
+constexpr int kPfTmemCols = kPfAccBufs * kPfBN;   // 512 columns: all of tensor memory
 constexpr unsigned kPfWaitPolls = 1u << 20;
 
 struct PrefillParams {
@@ -79,6 +82,13 @@ __device__ __forceinline__ bool pf_wait(uint32_t bar, unsigned parity, volatile 
     *abort_flag = 1;
     return false;
 }
+// Whole-warp wait: only lane 0 polls the barrier (32 lanes polling one shared-memory
+// word would compete with the tensor core for shared-memory bandwidth).
+__device__ __forceinline__ bool pf_wait_warp(uint32_t bar, unsigned parity, volatile int *abort_flag) {
+    int ok = 0;
+    if ((threadIdx.x & 31) == 0) ok = pf_wait(bar, parity, abort_flag) ? 1 : 0;
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+}
 __device__ __forceinline__ void pf_tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -116,6 +126,16 @@ __device__ __forceinline__ void pf_tmem_ld32(uint32_t taddr, int (&v)[32]) {
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
 }
+// (acc0, acc1) += (x0, x1) * sc as one packed fp32 instruction (one issue slot for two FMAs)
+__device__ __forceinline__ void pf_fma2(float &acc0, float &acc1, float x0, float x1, float sc) {
+    asm("{\n\t.reg .b64 a, b, c;\n\t"
+        "mov.b64 a, {%2, %3};\n\t"
+        "mov.b64 b, {%4, %4};\n\t"
+        "mov.b64 c, {%0, %1};\n\t"
+        "fma.rn.f32x2 c, a, b, c;\n\t"
+        "mov.b64 {%0, %1}, c;\n\t}"
+        : "+f"(acc0), "+f"(acc1) : "f"(x0), "f"(x1), "f"(sc));
+}
 __device__ __forceinline__ void pf_tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major [rows][128 B] tile stored with the
@@ -139,12 +159,33 @@ __host__ __device__ constexpr uint32_t pf_instr_desc(int m, int n) {
          | ((uint32_t)(m >> 4) << 24);    // M / 16
 }
 
+// Optional timeline trace (build with -DW2A8_TRACE): CTA (0,0) records the global
+// timer per role and iteration: slot = role * 4096 + index * 4 + point.
+#ifdef W2A8_TRACE
+__device__ unsigned long long *g_pf_trace = nullptr;   // 5 roles x 4096 slots
+__device__ __forceinline__ void pf_trace(int role, int idx, int point) {
+    if (g_pf_trace && blockIdx.x == 0 && blockIdx.y == 0 && idx < 1024) {
+        unsigned long long v;
+        if (role >= 3) v = (unsigned long long)clock64();      // SM cycles for the drain and MMA-group roles
+        else asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(v));
+        g_pf_trace[role * 4096 + idx * 4 + point] = v;
+    }
+}
+extern "C" int w2a8_debug_set_prefill_trace(void *buffer) {
+    unsigned long long *b = reinterpret_cast<unsigned long long *>(buffer);
+    return cudaMemcpyToSymbol(g_pf_trace, &b, sizeof(b)) == cudaSuccess ? 0 : W2A8_ERR_CUDA;
+}
+#define PF_TRACE(role, idx, point) pf_trace(role, idx, point)
+#else
+#define PF_TRACE(role, idx, point) do { } while (0)
+#endif
+
 template <bool PARTIALS>
 __global__ void __launch_bounds__(kPfThreads, 1)
 w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillParams p) {
     extern __shared__ unsigned char pf_smem_raw[];
     __shared__ __align__(8) unsigned long long bar_full_a[kPfStages], bar_full_b[kPfStages], bar_empty[kPfStages];
-    __shared__ __align__(8) unsigned long long bar_acc_full[2], bar_acc_empty[2];
+    __shared__ __align__(8) unsigned long long bar_acc_full[kPfAccBufs], bar_acc_empty[kPfAccBufs];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     __shared__ float a_scale_s[kPfBN];
@@ -162,13 +203,13 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         for (int s = 0; s < kPfStages; ++s) {
-            pf_mbar_init(pf_smem_u32(&bar_full_a[s]), 2);     // one arrive per unpack warp
+            pf_mbar_init(pf_smem_u32(&bar_full_a[s]), kPfUnpackWarps);   // one arrive per unpack warp
             pf_mbar_init(pf_smem_u32(&bar_full_b[s]), 1);     // TMA producer + transaction bytes
             pf_mbar_init(pf_smem_u32(&bar_empty[s]), 1);      // tcgen05.commit
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kPfAccBufs; ++b) {
             pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);   // tcgen05.commit
-            pf_mbar_init(pf_smem_u32(&bar_acc_empty[b]), 4);  // one arrive per drain warp
+            pf_mbar_init(pf_smem_u32(&bar_acc_empty[b]), 8);  // one arrive per drain warp
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         pf_fence_proxy_async();
@@ -194,67 +235,87 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
                 pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
                 pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
+                PF_TRACE(0, it, 0);
             }
         }
     } else if (warp == 1) {
         // ===== MMA issuer (one thread) ================================================
+        // A single thread runs this loop, so its scalar work is kept minimal: descriptors
+        // are a base plus compile-time offsets, group bookkeeping uses counters (no
+        // division), and the four slices of a stage are unrolled.
         if (lane == 0) {
             constexpr uint32_t idesc = pf_instr_desc(kPfBM, kPfBN);
-            int slice_idx = 0;          // 64-k slices issued so far
-            int buf = 0, buf_uses[2] = {0, 0};
+            const uint64_t a_desc0 = pf_smem_desc(smem_base);
+            const uint64_t b_desc0 = pf_smem_desc(smem_base + 2 * kPfHalfBytes);
+            int pos = 0;                    // 64-k slices already issued in the current group
+            int group_idx = 0;              // scale groups committed so far
+            int buf = 0;                    // accumulator buffer of the current group
+            uint32_t empty_parity = 0;      // bit b: parity to wait for on bar_acc_empty[b]
+            int s = 0;
+            uint32_t full_parity = 0;
             bool ok = true;
             for (int it = 0; it < nstages_total && ok; ++it) {
-                const int s = it % kPfStages, round = it / kPfStages;
-                ok = pf_wait(pf_smem_u32(&bar_full_a[s]), round & 1, abort_flag) &&
-                     pf_wait(pf_smem_u32(&bar_full_b[s]), round & 1, abort_flag);
+                ok = pf_wait(pf_smem_u32(&bar_full_a[s]), full_parity, abort_flag) &&
+                     pf_wait(pf_smem_u32(&bar_full_b[s]), full_parity, abort_flag);
                 if (!ok) break;
+                PF_TRACE(1, it, 0);
                 pf_tc_fence_after();
-                const uint32_t a_base = smem_base + s * kPfStageBytes;
-                const uint32_t b_base = a_base + 2 * kPfHalfBytes;
-                for (int q = 0; q < 4 && ok; ++q, ++slice_idx) {
-                    const bool group_start = (slice_idx % dps) == 0;
-                    if (group_start && buf_uses[buf] > 0) {
+                const uint64_t stage_off = (uint64_t)((uint32_t)(s * kPfStageBytes) >> 4);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (pos == 0 && group_idx >= kPfAccBufs) {
                         // the drain warps must have emptied this buffer's previous group
-                        ok = pf_wait(pf_smem_u32(&bar_acc_empty[buf]), (buf_uses[buf] - 1) & 1, abort_flag);
+                        ok = pf_wait(pf_smem_u32(&bar_acc_empty[buf]), (empty_parity >> buf) & 1u, abort_flag);
                         if (!ok) break;
+                        empty_parity ^= 1u << buf;
                         pf_tc_fence_after();
                     }
-                    const uint32_t half = (q >> 1) * kPfHalfBytes;
 #pragma unroll
                     for (int ks = 0; ks < 2; ++ks) {
-                        const uint32_t koff = ((q & 1) * 2 + ks) * 32;
-                        pf_mma_i8(tmem_base + buf * kPfBN, pf_smem_desc(a_base + half + koff),
-                                  pf_smem_desc(b_base + half + koff), idesc,
-                                  (group_start && ks == 0) ? 0u : 1u);
+                        constexpr int kHalf16 = kPfHalfBytes >> 4;
+                        const uint64_t off = stage_off + (uint64_t)((q >> 1) * kHalf16 + ((q & 1) * 2 + ks) * 2);
+                        pf_mma_i8(tmem_base + buf * kPfBN, a_desc0 + off, b_desc0 + off, idesc,
+                                  (pos == 0 && ks == 0) ? 0u : 1u);
                     }
-                    if ((slice_idx + 1) % dps == 0) {
+                    if (++pos == dps) {
                         pf_mma_commit(pf_smem_u32(&bar_acc_full[buf]));
-                        ++buf_uses[buf];
-                        buf ^= 1;
+                        pos = 0;
+                        ++group_idx;
+                        buf = (buf + 1) & (kPfAccBufs - 1);
                     }
                 }
                 pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
+                PF_TRACE(1, it, 1);
+                if (++s == kPfStages) { s = 0; full_parity ^= 1u; }
             }
         }
-    } else if (warp < 4) {
+    } else if (warp < 2 + kPfUnpackWarps) {
         // ===== unpack warps: packed words -> int8 lanes, K-major, 128-byte swizzle =====
-        const int ut = (warp - 2) * 32 + lane;      // 0..63
-        for (int it = 0; it < nstages_total; ++it) {
-            const int s = it % kPfStages, round = it / kPfStages;
-            // request this stage's words before waiting for the buffer
-            uint4 w[8];
+        constexpr int kUnits = 512 / (32 * kPfUnpackWarps);   // 16-byte units per thread and stage
+        const int ut = (warp - 2) * 32 + lane;
+        auto request = [&](uint4 (&w)[kUnits], int it) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int u = ut + 64 * i;          // unit index: row = u / 4, quarter t = u % 4
+            for (int i = 0; i < kUnits; ++i) {
+                const int u = ut + 32 * kPfUnpackWarps * i;   // unit: row = u / 4, quarter t = u % 4
                 const int r = u >> 2, t = u & 3;
                 w[i] = __ldg(reinterpret_cast<const uint4 *>(p.packed + (size_t)(n0 + r) * p.words_per_row +
                                                              16 * it + 4 * t));
             }
-            if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
+        };
+        uint4 w_nxt[kUnits];
+        request(w_nxt, 0);
+        for (int it = 0; it < nstages_total; ++it) {
+            const int s = it % kPfStages, round = it / kPfStages;
+            uint4 w[kUnits];
+#pragma unroll
+            for (int i = 0; i < kUnits; ++i) w[i] = w_nxt[i];
+            if (it + 1 < nstages_total) request(w_nxt, it + 1);   // next stage's words in flight
+            if (round > 0 && !pf_wait_warp(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
+            if (warp == 2 && lane == 0) PF_TRACE(2, it, 0);
             unsigned char *a_stage = smem_gen + s * kPfStageBytes;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int u = ut + 64 * i;
+            for (int i = 0; i < kUnits; ++i) {
+                const int u = ut + 32 * kPfUnpackWarps * i;
                 const int r = u >> 2, t = u & 3;
                 const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
 #pragma unroll
@@ -263,60 +324,99 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     v.x = lane_codes(ws[sl], 0); v.y = lane_codes(ws[sl], 1);
                     v.z = lane_codes(ws[sl], 2); v.w = lane_codes(ws[sl], 3);
                     const int chunk = (4 * (sl & 1) + t) ^ (r & 7);
+#ifdef W2A8_EXP_NOSTS
+                    if (v.x == 0x12345678u)
+#endif
                     *reinterpret_cast<uint4 *>(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16) = v;
                 }
             }
             pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
             __syncwarp();
             if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full_a[s]));
+            if (warp == 2 && lane == 0) PF_TRACE(2, it, 1);
         }
     } else {
         // ===== drain warps: TMEM -> registers, fp32 accumulate with the group scale ======
         const int q4 = warp & 3;                    // TMEM lane quarter this warp may access
+        const int col0 = ((warp - 2 - kPfUnpackWarps) >> 2) * kPfDrainCols;   // first token column of this warp
         const int ch = q4 * 32 + lane;              // channel inside the tile = TMEM lane
         const int n = n0 + ch;
-        float acc[kPfBN];
+        float acc[kPfDrainCols];
 #pragma unroll
-        for (int j = 0; j < kPfBN; ++j) acc[j] = 0.f;
+        for (int j = 0; j < kPfDrainCols; ++j) acc[j] = 0.f;
         const int ngroups = (p.K / 64) / dps;
-        int buf = 0, uses[2] = {0, 0};
-        bool ok = true;
-        for (int gi = 0; gi < ngroups && ok; ++gi) {
-            float sc = 0.f;
-            if (!PARTIALS) sc = __ldg(p.w_scale + (size_t)n * p.G + gi);
-            ok = pf_wait(pf_smem_u32(&bar_acc_full[buf]), uses[buf] & 1, abort_flag);
-            if (!ok) break;
-            pf_tc_fence_after();
+        // Scales are fetched eight groups ahead (a drain takes a few hundred cycles, a
+        // global load several hundred): a ring of eight, refilled once per eight groups.
+        const float *sc_row = PARTIALS ? nullptr : p.w_scale + (size_t)n * p.G;
+        float sc_nxt[8];
 #pragma unroll
-            for (int c = 0; c < kPfBN / 32; ++c) {
-                int v[32];
-                pf_tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + buf * kPfBN + c * 32, v);
-                pf_tmem_ld_wait();
-                if (c == kPfBN / 32 - 1) {
-                    // all of this buffer has been read: hand it back to the MMA warp
-                    pf_tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[buf]));
+        for (int u = 0; u < 8; ++u) sc_nxt[u] = (!PARTIALS && u < ngroups) ? __ldg(sc_row + u) : 0.f;
+        bool ok = true;
+        // Software pipeline over 32-column halves: while one half is converted and
+        // accumulated, the next half (possibly of the next group) is on its way from TMEM.
+        int v0[32], v1[32];                         // first / second half of the current group
+        const uint32_t tlane = tmem_base + ((uint32_t)(q4 * 32) << 16) + col0;
+        ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[0]), 0, abort_flag);
+        if (ok) { pf_tc_fence_after(); pf_tmem_ld32(tlane, v0); }
+        for (int g0 = 0; g0 < ngroups && ok; g0 += 8) {
+            float sc_cur[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                sc_cur[u] = sc_nxt[u];
+                sc_nxt[u] = (!PARTIALS && g0 + 8 + u < ngroups) ? __ldg(sc_row + g0 + 8 + u) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int gi = g0 + u;
+                if (gi >= ngroups || !ok) break;
+                const int buf = u % kPfAccBufs;        // group g lives in buffer g % kPfAccBufs (g0 is a multiple of 8)
+                const float sc = sc_cur[u];
+                pf_tmem_ld_wait();                     // first half of group gi is in v0
+                if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, gi, 0);
+                pf_tmem_ld32(tlane + buf * kPfBN + 32, v1);
+                if (PARTIALS) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int m = m0 + col0 + j;
+                        if (m < p.M) p.partials[((size_t)m * p.N + n) * p.G + gi] = v0[j] >> 6;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) pf_fma2(acc[j], acc[j + 1], (float)v0[j], (float)v0[j + 1], sc);
+                }
+                pf_tmem_ld_wait();                     // second half is in v1
+                // all of this warp's share of the buffer has been read: hand it back
+                pf_tc_fence_before();
+                __syncwarp();
+                if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[buf]));
+                if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, gi, 1);
+                if (gi + 1 < ngroups) {                // request the first half of the next group
+                    const int nbuf = (u + 1) % kPfAccBufs;
+                    ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[nbuf]), ((gi + 1) / kPfAccBufs) & 1, abort_flag);
+                    if (!ok) break;
+                    pf_tc_fence_after();
+                    pf_tmem_ld32(tlane + nbuf * kPfBN, v0);
                 }
                 if (PARTIALS) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        const int m = m0 + c * 32 + j;
-                        if (m < p.M) p.partials[((size_t)m * p.N + n) * p.G + gi] = v[j] >> 6;
+                        const int m = m0 + col0 + 32 + j;
+                        if (m < p.M) p.partials[((size_t)m * p.N + n) * p.G + gi] = v1[j] >> 6;
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[c * 32 + j] = fmaf(sc, (float)v[j], acc[c * 32 + j]);
+                    for (int j = 0; j < 32; j += 2)
+                        pf_fma2(acc[32 + j], acc[32 + j + 1], (float)v1[j], (float)v1[j + 1], sc);
                 }
+                if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, gi, 2);
             }
-            ++uses[buf];
-            buf ^= 1;
         }
+        pf_tmem_ld_wait();
         if (!PARTIALS && ok) {
 #pragma unroll
-            for (int j = 0; j < kPfBN; ++j) {
-                const int m = m0 + j;
-                if (m < p.M) p.y[(size_t)m * p.N + n] = acc[j] * a_scale_s[j];
+            for (int j = 0; j < kPfDrainCols; ++j) {
+                const int m = m0 + col0 + j;
+                if (m < p.M) p.y[(size_t)m * p.N + n] = acc[j] * a_scale_s[col0 + j];
             }
         }
     }
