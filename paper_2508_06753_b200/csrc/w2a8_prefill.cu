@@ -6,20 +6,22 @@
 // up-convert of Sec. II-C done into shared memory because the tensor core has
 // no 2-bit operand type.
 //
-// One CTA computes a 128-channel x 128-token tile of y.
+// One CTA (12 warps) computes a 128-channel x 128-token tile of y.
 //   A operand (UMMA M = 128): weights.  Two "unpack" warps read the packed words
 //     of 128 channels x one 256-k block, expand them to int8 lanes (value
 //     64 * (code - 2): one shift + one LOP3 per four weights) and store them
 //     K-major with the 128-byte swizzle the tensor core expects.
 //   B operand (UMMA N = 128): int8 activations, 128 tokens x 256 k, brought by TMA
-//     with the same swizzle.
+//     (issued by one lane of an unpack warp) with the same swizzle.
 //   D: int32 in tensor memory, lane = channel, column = token.  Because a lane is
 //     a channel, a drain thread needs one weight scale per group, not one per value.
-// Per 64-k group (or whatever the scale group is) the MMA warp issues K = 32
-// steps into one of two accumulator buffers; the "drain" warps read the other
-// buffer with tcgen05.ld, convert to fp32 and accumulate scale * value in
-// registers (eight drain warps: two per TMEM lane quarter, 64 token columns each).  Every wait on an mbarrier is bounded; a wait
-// that gives up sets the status word of the workspace and the CTA winds down.
+// Per 64-k group (or whatever the scale group is) an MMA thread issues K = 32 steps
+// into one of four accumulator buffers (all 512 TMEM columns); two threads share
+// the issuing, alternating groups.  Eight "drain" warps (two per TMEM lane quarter,
+// 64 token columns each) read finished buffers with tcgen05.ld, software-pipelined
+// in 32-column halves, convert to fp32 and accumulate scale * value in registers
+// with packed fp32 FMAs.  Every wait on an mbarrier is bounded; a wait that gives
+// up sets the status word of the workspace and the CTA winds down.
 #include <cuda.h>
 
 #include "w2a8_common.cuh"
@@ -27,7 +29,7 @@
 namespace w2a8 {
 
 constexpr int kPfUnpackWarps = 2;
-constexpr int kPfThreads = 32 * (2 + kPfUnpackWarps + 8);   // warps: TMA, MMA, unpack, 8 drain
+constexpr int kPfThreads = 32 * (2 + kPfUnpackWarps + 8);   // warps: 2 MMA issuers, unpack (+TMA), 8 drain
 constexpr int kPfDrainCols = 64;         // token columns per drain warp (two warps share a lane quarter)
 constexpr int kPfBM = 128;               // channels per tile (UMMA M)
 constexpr int kPfBN = 128;               // tokens per tile (UMMA N)
@@ -37,7 +39,7 @@ constexpr int kPfHalfBytes = 128 * 128;  // one [128 rows][128 B] swizzled sub-t
 constexpr int kPfStageBytes = 4 * kPfHalfBytes;   // A: 2 halves, B: 2 halves
 constexpr int kPfAccBufs = 4;             // accumulator buffers in tensor memory (groups in flight)
 constexpr int kPfTmemCols = kPfAccBufs * kPfBN;   // 512 columns: all of tensor memory
-constexpr unsigned kPfWaitPolls = 1u << 20;
+constexpr unsigned kPfWaitPolls = 1u << 20;   // bound of every barrier wait (polls)
 
 struct PrefillParams {
     const uint32_t *packed;
@@ -205,7 +207,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         for (int s = 0; s < kPfStages; ++s) {
             pf_mbar_init(pf_smem_u32(&bar_full_a[s]), kPfUnpackWarps);   // one arrive per unpack warp
             pf_mbar_init(pf_smem_u32(&bar_full_b[s]), 1);     // TMA producer + transaction bytes
-            pf_mbar_init(pf_smem_u32(&bar_empty[s]), 1);      // tcgen05.commit
+            pf_mbar_init(pf_smem_u32(&bar_empty[s]), 2);      // one tcgen05.commit per MMA-issuing thread
         }
         for (int b = 0; b < kPfAccBufs; ++b) {
             pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);   // tcgen05.commit
@@ -224,26 +226,16 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     pf_tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp == 0) {
-        // ===== TMA producer: activations, 128 tokens x 256 k per stage ==============
+    if (warp < 2) {
+        // ===== MMA issuers (one thread in each of warps 0 and 1) =========================
+        // Issuing is scalar work of a single thread and costs several hundred cycles per
+        // group, so two threads share it: thread `mma_id` takes the scale groups with
+        // group index = mma_id (mod 2), i.e. accumulator buffers mma_id and mma_id + 2.
+        // Groups are independent (different buffers), so no order between the two
+        // threads is needed.  Descriptors are a base plus compile-time offsets, group
+        // bookkeeping uses counters (no division), the four slices of a stage are unrolled.
         if (lane == 0) {
-            for (int it = 0; it < nstages_total; ++it) {
-                const int s = it % kPfStages, round = it / kPfStages;
-                if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
-                const uint32_t bar = pf_smem_u32(&bar_full_b[s]);
-                const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
-                pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
-                pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
-                pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
-                PF_TRACE(0, it, 0);
-            }
-        }
-    } else if (warp == 1) {
-        // ===== MMA issuer (one thread) ================================================
-        // A single thread runs this loop, so its scalar work is kept minimal: descriptors
-        // are a base plus compile-time offsets, group bookkeeping uses counters (no
-        // division), and the four slices of a stage are unrolled.
-        if (lane == 0) {
+            const int mma_id = warp;
             constexpr uint32_t idesc = pf_instr_desc(kPfBM, kPfBN);
             const uint64_t a_desc0 = pf_smem_desc(smem_base);
             const uint64_t b_desc0 = pf_smem_desc(smem_base + 2 * kPfHalfBytes);
@@ -258,34 +250,37 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 ok = pf_wait(pf_smem_u32(&bar_full_a[s]), full_parity, abort_flag) &&
                      pf_wait(pf_smem_u32(&bar_full_b[s]), full_parity, abort_flag);
                 if (!ok) break;
-                PF_TRACE(1, it, 0);
+                if (mma_id == 1) PF_TRACE(1, it, 0);
                 pf_tc_fence_after();
                 const uint64_t stage_off = (uint64_t)((uint32_t)(s * kPfStageBytes) >> 4);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    if (pos == 0 && group_idx >= kPfAccBufs) {
+                    const bool mine = (group_idx & 1) == mma_id;
+                    if (mine && pos == 0 && group_idx >= kPfAccBufs) {
                         // the drain warps must have emptied this buffer's previous group
                         ok = pf_wait(pf_smem_u32(&bar_acc_empty[buf]), (empty_parity >> buf) & 1u, abort_flag);
                         if (!ok) break;
                         empty_parity ^= 1u << buf;
                         pf_tc_fence_after();
                     }
+                    if (mine) {
 #pragma unroll
-                    for (int ks = 0; ks < 2; ++ks) {
-                        constexpr int kHalf16 = kPfHalfBytes >> 4;
-                        const uint64_t off = stage_off + (uint64_t)((q >> 1) * kHalf16 + ((q & 1) * 2 + ks) * 2);
-                        pf_mma_i8(tmem_base + buf * kPfBN, a_desc0 + off, b_desc0 + off, idesc,
-                                  (pos == 0 && ks == 0) ? 0u : 1u);
+                        for (int ks = 0; ks < 2; ++ks) {
+                            constexpr int kHalf16 = kPfHalfBytes >> 4;
+                            const uint64_t off = stage_off + (uint64_t)((q >> 1) * kHalf16 + ((q & 1) * 2 + ks) * 2);
+                            pf_mma_i8(tmem_base + buf * kPfBN, a_desc0 + off, b_desc0 + off, idesc,
+                                      (pos == 0 && ks == 0) ? 0u : 1u);
+                        }
                     }
                     if (++pos == dps) {
-                        pf_mma_commit(pf_smem_u32(&bar_acc_full[buf]));
+                        if (mine) pf_mma_commit(pf_smem_u32(&bar_acc_full[buf]));
                         pos = 0;
                         ++group_idx;
                         buf = (buf + 1) & (kPfAccBufs - 1);
                     }
                 }
                 pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
-                PF_TRACE(1, it, 1);
+                if (mma_id == 1) PF_TRACE(1, it, 1);
                 if (++s == kPfStages) { s = 0; full_parity ^= 1u; }
             }
         }
@@ -311,7 +306,15 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             for (int i = 0; i < kUnits; ++i) w[i] = w_nxt[i];
             if (it + 1 < nstages_total) request(w_nxt, it + 1);   // next stage's words in flight
             if (round > 0 && !pf_wait_warp(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
-            if (warp == 2 && lane == 0) PF_TRACE(2, it, 0);
+            if (warp == 2 && lane == 0) {
+                // this lane is also the TMA producer: activations, 128 tokens x 256 k per stage
+                const uint32_t bar = pf_smem_u32(&bar_full_b[s]);
+                const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
+                pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
+                pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
+                pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
+                PF_TRACE(2, it, 0);
+            }
             unsigned char *a_stage = smem_gen + s * kPfStageBytes;
 #pragma unroll
             for (int i = 0; i < kUnits; ++i) {
