@@ -32,7 +32,7 @@ __device__ __forceinline__ uint32_t lane_codes(uint32_t word, int j) {
     // j is a compile-time constant after unrolling; (x & mask) ^ flip is one LOP3 (LUT 0x6A)
     const uint32_t x = (j == 3) ? word : (word << (6 - 2 * j));
     uint32_t r;
-    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(r) : "r"(x), "r"(kTopMask), "r"(kSignFlip));
+    asm("lop3.b32 %0, %1, 0xC0C0C0C0, 0x80808080, 0x6A;" : "=r"(r) : "r"(x));
     return r;
 }
 

@@ -35,7 +35,10 @@ constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kActPad = 64;                    // activation row stride = chunk bytes + 64
 constexpr int kSmemBudget = 64 * 1024;         // per CTA: scales + activations
-constexpr int kRound = 4;                      // cells whose weights a lane holds at once
+#ifndef W2A8_MINB
+#define W2A8_MINB(MT) ((MT) == 1 ? 7 : ((MT) == 2 ? 5 : 4))
+#endif
+constexpr int kRound = 4;                      // cells a lane keeps in flight (ring depth, power of 2)
 
 struct DecodeParams {
     const int8_t *a;
@@ -54,6 +57,7 @@ struct DecodeParams {
     int act_stride;       // bytes per staged token row
     int s_vec;            // scale rows can be copied in 16-byte units
     int off_a;            // byte offset of the activation area in shared memory
+    int off_ring;         // byte offset of the per-lane weight rings
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------
@@ -76,6 +80,8 @@ __device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // Optional timeline trace (build with -DW2A8_TRACE): every warp records the
 // global timer at a few points of the kernel into a caller-provided buffer.
@@ -99,15 +105,21 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // One cell: 4 slices x (unpack, 2 MMAs per token slab, promotion at group ends).
 // w0s/w1s: this lane's four words (one per slice) of channels n0+gq and n0+gq+8;
 // srow0/srow1: staged scale rows of the same channels.
-template <int MT, int SPP, bool ONE, bool PARTIALS>
+template <int MT, int SPP, bool ONE, bool PARTIALS, bool FULL>
 __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32_t (&w0s)[4],
                                              const uint32_t (&w1s)[4], const unsigned char *srow0,
                                              const unsigned char *srow1,
                                              const unsigned char *const (&brow)[MT], int kl,
                                              int kb, int n0, int m0, int gq, int t,
-                                             float (&acc)[MT][4], int (&D)[MT][4]) {
-    const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
+                                             float (&acc)[MT][4]) {
+    // FULL: the block has all four slices (always, except possibly the last block of K)
+    const int R = FULL ? 4 : p.tail_slices;
     const int magic[4] = {kMagicInt, kMagicInt, kMagicInt, kMagicInt};
+    int D[MT][4];   // int32 accumulators of the current group; a group never outlives a cell
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) D[mt][i] = kMagicInt;
     float s0s[4 / SPP], s1s[4 / SPP];
     if constexpr (!PARTIALS) {
         if constexpr (SPP == 4) {
@@ -129,18 +141,30 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
     for (int s = 0; s < 4; ++s) {
         if (s < R) {
             const uint32_t w0 = w0s[s], w1 = w1s[s];
+#ifdef W2A8_EXP_NOUNPACK
+            const uint32_t a0 = w0, a1 = w1, a2 = w0 + 1, a3 = w1 + 1, a4 = w0 + 2, a5 = w1 + 2, a6 = w0 + 3, a7 = w1 + 3;
+#else
             const uint32_t a0 = lane_codes(w0, 0), a1 = lane_codes(w1, 0);
             const uint32_t a2 = lane_codes(w0, 1), a3 = lane_codes(w1, 1);
             const uint32_t a4 = lane_codes(w0, 2), a5 = lane_codes(w1, 2);
             const uint32_t a6 = lane_codes(w0, 3), a7 = lane_codes(w1, 3);
+#endif
             const bool first = (s % SPP) == 0;
             const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
+#ifdef W2A8_EXP_NOB
+                const uint4 b = make_uint4(w0 ^ 1u, w1 ^ 2u, w0 ^ 3u, w1 ^ 4u);
+#else
                 const uint4 b = *reinterpret_cast<const uint4 *>(brow[mt] + kl * kBlockK + s * kSliceK);
+#endif
+#ifdef W2A8_EXP_NOMMA
+                D[mt][0] += a0 ^ b.x; D[mt][1] += a1 ^ b.y; D[mt][2] += a2 ^ a4 ^ b.z; D[mt][3] += a3 ^ a5 ^ a6 ^ a7 ^ b.w;
+#else
                 if (first) mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, magic);
                 else       mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, D[mt]);
                 mma_s8_16x8x32(D[mt], a4, a5, a6, a7, b.z, b.w, D[mt]);
+#endif
                 if (last) {
                     if constexpr (PARTIALS) {
                         const int gi = (SPP == 1) ? 4 * kb + s
@@ -155,7 +179,11 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
                                           (D[mt][i] - kMagicInt) >> 6);
                         }
                     } else {
+#ifdef W2A8_EXP_NOSCALE
+                        const float s0 = 0.5f, s1 = 0.25f;
+#else
                         const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
+#endif
                         acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
                         acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
                         if constexpr (!ONE) {
@@ -173,7 +201,7 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
 // TG: tiles per CTA (K-lanes per tile = 4 / TG); ONE: a single token (half of
 // each accumulator quad is dead and is not promoted).
 template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
-__global__ void __launch_bounds__(kDecodeThreads, (MT == 1 ? 7 : (MT == 2 ? 5 : 4)))
+__global__ void __launch_bounds__(kDecodeThreads, W2A8_MINB(MT))
 w2a8_decode_kernel(const DecodeParams p) {
     constexpr int KS = kDecodeWarps / TG;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -200,31 +228,32 @@ w2a8_decode_kernel(const DecodeParams p) {
     const int tiles_here = min(TG, p.N / 16 - blockIdx.x * TG);
     const int rows_here = tiles_here * 16;
 
-    // this lane's weight words of up to kRound cells: [cell][channel gq / gq+8][slice]
-    uint32_t wreg[kRound][2][4];
-    auto request_cell = [&](int j, int kl) {
+    // Lane-private ring of kRound cells in shared memory: slot j of this lane holds the two
+    // 16-byte units (channels gq and gq+8) of one cell.  Only this lane writes and reads its
+    // slots, so cp.async.wait_group alone orders them (no warp barrier).
+    unsigned char *ring = smem + p.off_ring + warp * (kRound * 2 * 32 * 16) + lane * 16;
+    auto post_cell = [&](int slot, int kl) {
         const int kb = kb_begin + kl;
         const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             const uint32_t *wp = p.packed + (size_t)(n0 + gq + 8 * r) * p.words_per_row + 16 * kb;
+            unsigned char *dst = ring + (slot * 2 + r) * (32 * 16);
             if (R == 4) {
-                const uint4 v = ld_stream_v4(wp + 4 * t);
-                wreg[j][r][0] = v.x; wreg[j][r][1] = v.y; wreg[j][r][2] = v.z; wreg[j][r][3] = v.w;
+                cp_async16(smem_u32(dst), wp + 4 * t);
             } else {   // trailing block with fewer slices: words t*R .. t*R+R-1
-#pragma unroll
-                for (int s2 = 0; s2 < 4; ++s2) wreg[j][r][s2] = (s2 < R) ? __ldg(wp + t * R + s2) : 0u;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                v.x = __ldg(wp + t * R);
+                if (R > 1) v.y = __ldg(wp + t * R + 1);
+                if (R > 2) v.z = __ldg(wp + t * R + 2);
+                *reinterpret_cast<uint4 *>(dst) = v;
             }
         }
     };
+    const int my_cells = tile_ok ? (nb - ks + KS - 1) / KS : 0;   // cells of this warp: kl = ks + c * KS
 
-    // ---- first half of the first round, and the scales of the whole chunk (all
-    //      independent of the previous kernel) ------------------------------------
-    if (tile_ok) {
-#pragma unroll
-        for (int j = 0; j < kRound / 2; ++j)
-            if (ks + j * KS < nb) request_cell(j, ks + j * KS);
-    }
+    // ---- group 0: scales of the whole chunk + cell 0; group 1: cell 1 (all independent
+    //      of the previous kernel) -------------------------------------------------------
     if constexpr (!PARTIALS) {
         const int nsc = sc_end - sc_begin;
         const float *sbase = p.w_scale + (size_t)blockIdx.x * TG * 16 * p.G + sc_begin;
@@ -239,13 +268,17 @@ w2a8_decode_kernel(const DecodeParams p) {
                     cp_async4(smem_u32(sm_s + r * p.s_stride + 4 * j), sbase + (size_t)r * p.G + j);
         }
     }
+    if (0 < my_cells) post_cell(0, ks);
+    cp_async_commit();
+    if (1 < my_cells) post_cell(1, ks + KS);
+    cp_async_commit();
     W2A8_TRACE_POINT(1);
     pdl_launch_dependents();
     pdl_wait();
     W2A8_TRACE_POINT(2);
 
-    // ---- request the activations of this chunk: [mrows + 1][chunk k (+pad)]; the
-    //      extra row is zeros and stands in for tokens beyond M --------------------
+    // ---- group 2: the activations of this chunk: [mrows + 1][chunk k (+pad)]; the extra
+    //      row is zeros and stands in for tokens beyond M ----------------------------------
     {
         const int row_units = nb * (kBlockK / 16);
         const int klen = min(nb * kBlockK, p.K - kb_begin * kBlockK);
@@ -259,22 +292,20 @@ w2a8_decode_kernel(const DecodeParams p) {
         }
         cp_async_commit();
     }
-    // ---- second half of the first round ---------------------------------------------
-    if (tile_ok) {
-#pragma unroll
-        for (int j = kRound / 2; j < kRound; ++j)
-            if (ks + j * KS < nb) request_cell(j, ks + j * KS);
-    }
-    cp_async_wait_all();
-    __syncthreads();   // scales and activations staged
+    // ---- groups 3, 4: cells 2 and 3 ----------------------------------------------------------
+    if (2 < my_cells) post_cell(2, ks + 2 * KS);
+    cp_async_commit();
+    if (3 < my_cells) post_cell(3, ks + 3 * KS);
+    cp_async_commit();
+    cp_async_wait_group<2>();   // scales, cells 0 and 1 and the activations have landed
+    __syncthreads();            // scales and activations are shared by the CTA
     W2A8_TRACE_POINT(3);
 
     float acc[MT][4];
-    int D[MT][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { acc[mt][i] = 0.f; D[mt][i] = kMagicInt; }
+        for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
 
     if (tile_ok) {
         const unsigned char *brow[MT];   // this lane's token row of each slab (or the zero row)
@@ -283,20 +314,27 @@ w2a8_decode_kernel(const DecodeParams p) {
             brow[mt] = acts + ((8 * mt + gq < mrows) ? (8 * mt + gq) : mrows) * p.act_stride + t * 16;
         const unsigned char *srow0 = sm_s + (tl * 16 + gq) * p.s_stride;   // floats from sc_begin on
         const unsigned char *srow1 = srow0 + 8 * p.s_stride;
-        // Software pipeline over rounds: as soon as a cell has been consumed, its
-        // registers take the weights of the same slot of the next round.
-        for (int kl0 = ks; kl0 < nb; kl0 += kRound * KS) {
-#pragma unroll
-            for (int j = 0; j < kRound; ++j) {
-                const int kl = kl0 + j * KS;
-                if (kl < nb) {
-                    compute_cell<MT, SPP, ONE, PARTIALS>(p, wreg[j][0], wreg[j][1], srow0, srow1, brow,
-                                                         kl, kb_begin + kl, n0, m0, gq, t, acc, D);
-                    if (kl + kRound * KS < nb) request_cell(j, kl + kRound * KS);
-                }
-            }
+        // One group is committed per iteration (the cell four ahead, or nothing), so
+        // "at most three groups pending" always means that the current cell has landed.
+        for (int c = 0; c < my_cells; ++c) {
+            cp_async_wait_group<3>();
+            const int slot = c & (kRound - 1);
+            const uint4 wa = *reinterpret_cast<const uint4 *>(ring + (slot * 2 + 0) * (32 * 16));
+            const uint4 wb = *reinterpret_cast<const uint4 *>(ring + (slot * 2 + 1) * (32 * 16));
+            if (c + kRound < my_cells) post_cell(slot, ks + (c + kRound) * KS);
+            cp_async_commit();
+            const uint32_t w0s[4] = {wa.x, wa.y, wa.z, wa.w};
+            const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
+            const int kl = ks + c * KS;
+            if (kb_begin + kl != p.blocks - 1 || p.tail_slices == 4)
+                compute_cell<MT, SPP, ONE, PARTIALS, true>(p, w0s, w1s, srow0, srow1, brow, kl, kb_begin + kl,
+                                                           n0, m0, gq, t, acc);
+            else
+                compute_cell<MT, SPP, ONE, PARTIALS, false>(p, w0s, w1s, srow0, srow1, brow, kl, kb_begin + kl,
+                                                            n0, m0, gq, t, acc);
         }
     }
+    cp_async_wait_all();
     W2A8_TRACE_POINT(5);
 
     if constexpr (!PARTIALS) {
@@ -367,7 +405,7 @@ static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct DecodePlan {
     int mt, tg, chunks, blocks_per_chunk, slabs, groups;
-    int s_stride, act_stride, off_a, s_vec;
+    int s_stride, act_stride, off_a, off_ring, s_vec;
     size_t smem;
 };
 
@@ -381,7 +419,8 @@ static void plan_smem(DecodePlan &pl, int M, int G, int spp, int nb) {
     pl.off_a = round_up(pl.tg * 16 * pl.s_stride, 128);
     const size_t act = (size_t)(mrows + 1) * pl.act_stride;
     const size_t red = (size_t)kDecodeWarps * pl.mt * 4 * 32 * sizeof(float);
-    pl.smem = pl.off_a + (act > red ? act : red);
+    pl.off_ring = round_up(pl.off_a + (int)(act > red ? act : red), 128);
+    pl.smem = pl.off_ring + (size_t)kDecodeWarps * kRound * 2 * 32 * 16;
 }
 
 // Tiles per CTA and K-chunks.  One tile per CTA (4 K-lanes) keeps each warp's
@@ -502,7 +541,7 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
     p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;
     p.s_stride = pl.s_stride; p.act_stride = pl.act_stride;
-    p.off_a = pl.off_a; p.s_vec = pl.s_vec;
+    p.off_a = pl.off_a; p.off_ring = pl.off_ring; p.s_vec = pl.s_vec;
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
     char *base = reinterpret_cast<char *>(workspace);
     p.status = reinterpret_cast<int *>(base);
