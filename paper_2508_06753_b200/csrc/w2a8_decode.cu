@@ -36,7 +36,7 @@ constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kActPad = 64;                    // activation row stride = chunk bytes + 64
 constexpr int kSmemBudget = 64 * 1024;         // per CTA: scales + activations
 #ifndef W2A8_MINB
-#define W2A8_MINB(MT) ((MT) == 1 ? 7 : ((MT) == 2 ? 5 : 4))
+#define W2A8_MINB(MT) ((MT) == 1 ? 7 : 3)
 #endif
 constexpr int kRound = 4;                      // cells a lane keeps in flight (ring depth, power of 2)
 
@@ -53,6 +53,7 @@ struct DecodeParams {
     int M, N, K, G, group;
     int blocks, tail_slices, words_per_row;
     int chunks, blocks_per_chunk;
+    int tiles_per_warp;   // tiles a warp walks when it owns whole tiles (TG == 4)
     int s_stride;         // bytes per staged scale row
     int act_stride;       // bytes per staged token row
     int s_vec;            // scale rows can be copied in 16-byte units
@@ -198,9 +199,16 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
 }
 
 // MT: 8-token slabs per CTA; SPP: 64-k slices per scale group (capped at 4);
-// TG: tiles per CTA (K-lanes per tile = 4 / TG); ONE: a single token (half of
-// each accumulator quad is dead and is not promoted).
-template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
+// TG: tiles the four warps of a CTA work on side by side (K-lanes per tile = 4 / TG);
+// RING: cells a lane keeps in flight; ONE: a single token (half of each accumulator
+// quad is dead and is not promoted).
+//
+// With TG == 4 every warp owns whole tiles: it walks p.tiles_per_warp tiles of the
+// chunk one after the other (tile = (blockIdx.x * tiles_per_warp + i) * 4 + warp),
+// re-using the activations the CTA staged once, and finishes each tile on its own
+// (no CTA barrier after the staging).  With TG < 4 the K-lanes of a tile are summed
+// through shared memory and tiles_per_warp is 1.
+template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS>
 __global__ void __launch_bounds__(kDecodeThreads, W2A8_MINB(MT))
 w2a8_decode_kernel(const DecodeParams p) {
     constexpr int KS = kDecodeWarps / TG;
@@ -209,31 +217,41 @@ w2a8_decode_kernel(const DecodeParams p) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, t = lane & 3;
     const int tl = warp % TG, ks = warp / TG;
-    const int tile = blockIdx.x * TG + tl;
-    const bool tile_ok = tile * 16 < p.N;
-    const int n0 = tile * 16;
+    const int TL = (KS == 1) ? p.tiles_per_warp : 1;
+    const int ntiles = p.N / 16;
+    const int tile0 = blockIdx.x * TL * TG;       // first tile of this CTA
     const int chunk = blockIdx.y;
     const int kb_begin = chunk * p.blocks_per_chunk;
     const int kb_end = min(kb_begin + p.blocks_per_chunk, p.blocks);
     const int nb = kb_end - kb_begin;
     const int m0 = blockIdx.z * (8 * MT);
     const int mrows = min(8 * MT, p.M - m0);
-    unsigned char *sm_s = smem;                 // [TG * 16][s_stride]
+    unsigned char *sm_s = smem;                 // [tiles of the CTA * 16][s_stride]
     unsigned char *acts = smem + p.off_a;       // [mrows + 1][act_stride]
     W2A8_TRACE_POINT(0);
 
     constexpr int SPB = 4 / SPP;                                  // scales per block and channel
     const int sc_begin = (SPP == 4) ? 0 : SPB * kb_begin;
     const int sc_end = (SPP == 4) ? p.G : min(SPB * kb_end, p.G);
-    const int tiles_here = min(TG, p.N / 16 - blockIdx.x * TG);
+    const int tiles_here = min(TG * TL, ntiles - tile0);
     const int rows_here = tiles_here * 16;
 
-    // Lane-private ring of kRound cells in shared memory: slot j of this lane holds the two
+    // This warp's cells, flattened over its tiles: cell c = (tile i = c / nbw, block
+    // kl = ks + (c % nbw) * KS); tiles beyond N are cut off.
+    const int nbw = (nb - ks + KS - 1) / KS;                       // cells per tile for this K-lane
+    int my_tiles = 0;
+    for (int i = 0; i < TL; ++i)
+        if (tile0 + i * TG + tl < ntiles) my_tiles = i + 1;
+    const int my_cells = my_tiles * nbw;
+
+    // Lane-private ring of RING cells in shared memory: slot j of this lane holds the two
     // 16-byte units (channels gq and gq+8) of one cell.  Only this lane writes and reads its
     // slots, so cp.async.wait_group alone orders them (no warp barrier).
-    unsigned char *ring = smem + p.off_ring + warp * (kRound * 2 * 32 * 16) + lane * 16;
-    auto post_cell = [&](int slot, int kl) {
+    unsigned char *ring = smem + p.off_ring + warp * (RING * 2 * 32 * 16) + lane * 16;
+    auto post_cell = [&](int slot, int c) {
+        const int ti = c / nbw, kl = ks + (c - ti * nbw) * KS;
         const int kb = kb_begin + kl;
+        const int n0 = (tile0 + ti * TG + tl) * 16;
         const int R = (kb == p.blocks - 1) ? p.tail_slices : 4;
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
@@ -250,13 +268,12 @@ w2a8_decode_kernel(const DecodeParams p) {
             }
         }
     };
-    const int my_cells = tile_ok ? (nb - ks + KS - 1) / KS : 0;   // cells of this warp: kl = ks + c * KS
 
-    // ---- group 0: scales of the whole chunk + cell 0; group 1: cell 1 (all independent
-    //      of the previous kernel) -------------------------------------------------------
+    // ---- first group: scales of the CTA's tiles for the whole chunk + cell 0; then one
+    //      group per cell up to half the ring (all independent of the previous kernel) ----
     if constexpr (!PARTIALS) {
         const int nsc = sc_end - sc_begin;
-        const float *sbase = p.w_scale + (size_t)blockIdx.x * TG * 16 * p.G + sc_begin;
+        const float *sbase = p.w_scale + (size_t)tile0 * 16 * p.G + sc_begin;
         if (p.s_vec && (nsc % 4 == 0)) {
             const int nu = nsc / 4;
             for (int r = warp; r < rows_here; r += kDecodeWarps)
@@ -268,16 +285,17 @@ w2a8_decode_kernel(const DecodeParams p) {
                     cp_async4(smem_u32(sm_s + r * p.s_stride + 4 * j), sbase + (size_t)r * p.G + j);
         }
     }
-    if (0 < my_cells) post_cell(0, ks);
-    cp_async_commit();
-    if (1 < my_cells) post_cell(1, ks + KS);
-    cp_async_commit();
+#pragma unroll
+    for (int j = 0; j < RING / 2; ++j) {
+        if (j < my_cells) post_cell(j, j);
+        cp_async_commit();
+    }
     W2A8_TRACE_POINT(1);
     pdl_launch_dependents();
     pdl_wait();
     W2A8_TRACE_POINT(2);
 
-    // ---- group 2: the activations of this chunk: [mrows + 1][chunk k (+pad)]; the extra
+    // ---- next group: the activations of this chunk: [mrows + 1][chunk k (+pad)]; the extra
     //      row is zeros and stands in for tokens beyond M ----------------------------------
     {
         const int row_units = nb * (kBlockK / 16);
@@ -292,13 +310,14 @@ w2a8_decode_kernel(const DecodeParams p) {
         }
         cp_async_commit();
     }
-    // ---- groups 3, 4: cells 2 and 3 ----------------------------------------------------------
-    if (2 < my_cells) post_cell(2, ks + 2 * KS);
-    cp_async_commit();
-    if (3 < my_cells) post_cell(3, ks + 3 * KS);
-    cp_async_commit();
-    cp_async_wait_group<2>();   // scales, cells 0 and 1 and the activations have landed
-    __syncthreads();            // scales and activations are shared by the CTA
+    // ---- the second half of the ring ----------------------------------------------------------
+#pragma unroll
+    for (int j = RING / 2; j < RING; ++j) {
+        if (j < my_cells) post_cell(j, j);
+        cp_async_commit();
+    }
+    cp_async_wait_group<RING / 2>();   // scales, the first half of the ring and the activations have landed
+    __syncthreads();                   // scales and activations are shared by the CTA
     W2A8_TRACE_POINT(3);
 
     float acc[MT][4];
@@ -307,37 +326,86 @@ w2a8_decode_kernel(const DecodeParams p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
 
-    if (tile_ok) {
-        const unsigned char *brow[MT];   // this lane's token row of each slab (or the zero row)
+    const unsigned char *brow[MT];   // this lane's token row of each slab (or the zero row)
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-            brow[mt] = acts + ((8 * mt + gq < mrows) ? (8 * mt + gq) : mrows) * p.act_stride + t * 16;
-        const unsigned char *srow0 = sm_s + (tl * 16 + gq) * p.s_stride;   // floats from sc_begin on
+    for (int mt = 0; mt < MT; ++mt)
+        brow[mt] = acts + ((8 * mt + gq < mrows) ? (8 * mt + gq) : mrows) * p.act_stride + t * 16;
+    const size_t MN = (size_t)p.M * p.N;
+
+    // One group is committed per iteration (the cell RING ahead, or nothing), so "at most
+    // RING - 1 groups pending" always means that the current cell has landed.
+    int ti = 0, ci = 0;              // tile of the current cell, cell index inside the tile
+    for (int c = 0; c < my_cells; ++c) {
+        cp_async_wait_group<RING - 1>();
+        const int slot = c & (RING - 1);
+        const uint4 wa = *reinterpret_cast<const uint4 *>(ring + (slot * 2 + 0) * (32 * 16));
+        const uint4 wb = *reinterpret_cast<const uint4 *>(ring + (slot * 2 + 1) * (32 * 16));
+        if (c + RING < my_cells) post_cell(slot, c + RING);
+        cp_async_commit();
+        const uint32_t w0s[4] = {wa.x, wa.y, wa.z, wa.w};
+        const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
+        const int kl = ks + ci * KS;
+        const int n0 = (tile0 + ti * TG + tl) * 16;
+        const unsigned char *srow0 = sm_s + ((ti * TG + tl) * 16 + gq) * p.s_stride;   // floats from sc_begin on
         const unsigned char *srow1 = srow0 + 8 * p.s_stride;
-        // One group is committed per iteration (the cell four ahead, or nothing), so
-        // "at most three groups pending" always means that the current cell has landed.
-        for (int c = 0; c < my_cells; ++c) {
-            cp_async_wait_group<3>();
-            const int slot = c & (kRound - 1);
-            const uint4 wa = *reinterpret_cast<const uint4 *>(ring + (slot * 2 + 0) * (32 * 16));
-            const uint4 wb = *reinterpret_cast<const uint4 *>(ring + (slot * 2 + 1) * (32 * 16));
-            if (c + kRound < my_cells) post_cell(slot, ks + (c + kRound) * KS);
-            cp_async_commit();
-            const uint32_t w0s[4] = {wa.x, wa.y, wa.z, wa.w};
-            const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
-            const int kl = ks + c * KS;
-            if (kb_begin + kl != p.blocks - 1 || p.tail_slices == 4)
-                compute_cell<MT, SPP, ONE, PARTIALS, true>(p, w0s, w1s, srow0, srow1, brow, kl, kb_begin + kl,
-                                                           n0, m0, gq, t, acc);
-            else
-                compute_cell<MT, SPP, ONE, PARTIALS, false>(p, w0s, w1s, srow0, srow1, brow, kl, kb_begin + kl,
-                                                            n0, m0, gq, t, acc);
+        if (kb_begin + kl != p.blocks - 1 || p.tail_slices == 4)
+            compute_cell<MT, SPP, ONE, PARTIALS, true>(p, w0s, w1s, srow0, srow1, brow, kl, kb_begin + kl,
+                                                       n0, m0, gq, t, acc);
+        else
+            compute_cell<MT, SPP, ONE, PARTIALS, false>(p, w0s, w1s, srow0, srow1, brow, kl, kb_begin + kl,
+                                                        n0, m0, gq, t, acc);
+        if (++ci == nbw) {
+            // ---- the tile is complete for this warp --------------------------------------------
+            if constexpr (KS == 1 && !PARTIALS) {
+                // the warp owns the whole tile: lane (gq, t) holds channels n0+gq, n0+gq+8 for
+                // tokens 2t, 2t+1 of each slab
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int mm = m0 + 8 * mt + 2 * t + (i & 1);
+                        const int nn = n0 + gq + 8 * (i >> 1);
+                        if (mm < p.M) {
+                            if (p.chunks == 1) p.y[(size_t)mm * p.N + nn] = acc[mt][i] * (p.a_scale[mm] * (1.0f / kCodeGain));
+                            else __stcg(p.ws + chunk * MN + (size_t)mm * p.N + nn, acc[mt][i]);
+                        }
+                        acc[mt][i] = 0.f;
+                    }
+                if (p.chunks > 1) {
+                    // split-K: the last warp to arrive for this tile and slab sums the chunks in order
+                    __threadfence();
+                    __syncwarp();
+                    unsigned *counter = p.counters + (size_t)blockIdx.z * ntiles + (n0 >> 4);
+                    unsigned ticket = 0;
+                    if (lane == 0) ticket = atomicAdd(counter, 1u);
+                    ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+                    if (ticket == (unsigned)p.chunks - 1u) {
+                        __threadfence();
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int mm = m0 + 8 * mt + 2 * t + (i & 1);
+                                const int nn = n0 + gq + 8 * (i >> 1);
+                                if (mm < p.M) {
+                                    float v = 0.f;
+                                    for (int ch = 0; ch < p.chunks; ++ch)
+                                        v += __ldcg(p.ws + ch * MN + (size_t)mm * p.N + nn);
+                                    p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
+                                }
+                            }
+                        if (lane == 0) *counter = 0u;   // leave the workspace reusable
+                    }
+                }
+            }
+            ci = 0;
+            ++ti;
         }
     }
     cp_async_wait_all();
     W2A8_TRACE_POINT(5);
 
-    if constexpr (!PARTIALS) {
+    if constexpr (!PARTIALS && KS > 1) {
         // ---- sum the K-lanes of each tile in a fixed order -----------------------
         // lane (gq, t) holds channels n0+gq, n0+gq+8 for tokens 2t, 2t+1 of each slab
         float *red = reinterpret_cast<float *>(acts);   // [KS][TG][MT*4][32], reuses the staging area
@@ -348,7 +416,6 @@ w2a8_decode_kernel(const DecodeParams p) {
             for (int i = 0; i < 4; ++i)
                 red[((ks * TG + tl) * (MT * 4) + mt * 4 + i) * 32 + lane] = acc[mt][i];
         __syncthreads();
-        const size_t MN = (size_t)p.M * p.N;
         // element e of the CTA: (tile etl, slab mt, quad register i, lane el)
         for (int e = threadIdx.x; e < TG * MT * 128; e += kDecodeThreads) {
             const int el = e & 31, ei = (e >> 5) % (MT * 4), etl = e / (MT * 128);
@@ -357,7 +424,7 @@ w2a8_decode_kernel(const DecodeParams p) {
 #pragma unroll
             for (int k2 = 0; k2 < KS; ++k2) v += red[((k2 * TG + etl) * (MT * 4) + ei) * 32 + el];
             const int mm = m0 + 8 * mt + 2 * (el & 3) + (i & 1);
-            const int nn = (blockIdx.x * TG + etl) * 16 + (el >> 2) + 8 * (i >> 1);
+            const int nn = (tile0 + etl) * 16 + (el >> 2) + 8 * (i >> 1);
             if (mm < p.M && nn < p.N) {
                 if (p.chunks == 1) p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
                 else __stcg(p.ws + chunk * MN + (size_t)mm * p.N + nn, v);
@@ -369,7 +436,7 @@ w2a8_decode_kernel(const DecodeParams p) {
         // ---- split-K: the last CTA to arrive sums the partial outputs in order ---
         __threadfence();
         __syncthreads();
-        unsigned *counter = p.counters + (size_t)blockIdx.z * gridDim.x + blockIdx.x;
+        unsigned *counter = p.counters + (size_t)blockIdx.z * ntiles + tile0;
         if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) == (unsigned)p.chunks - 1u);
         __syncthreads();
         if (!is_last) return;
@@ -378,7 +445,7 @@ w2a8_decode_kernel(const DecodeParams p) {
             const int el = e & 31, ei = (e >> 5) % (MT * 4), etl = e / (MT * 128);
             const int mt = ei >> 2, i = ei & 3;
             const int mm = m0 + 8 * mt + 2 * (el & 3) + (i & 1);
-            const int nn = (blockIdx.x * TG + etl) * 16 + (el >> 2) + 8 * (i >> 1);
+            const int nn = (tile0 + etl) * 16 + (el >> 2) + 8 * (i >> 1);
             if (mm < p.M && nn < p.N) {
                 float v = 0.f;
                 for (int ch = 0; ch < p.chunks; ++ch) v += __ldcg(p.ws + ch * MN + (size_t)mm * p.N + nn);
@@ -404,67 +471,103 @@ static inline int decode_mt(int M) { return M > 32 ? 4 : (M + 7) / 8; }
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct DecodePlan {
-    int mt, tg, chunks, blocks_per_chunk, slabs, groups;
+    int mt, tg, ring, tl, chunks, blocks_per_chunk, slabs, groups;
     int s_stride, act_stride, off_a, off_ring, s_vec;
     size_t smem;
 };
 
-// Shared-memory footprint of a CTA that stages `nb` blocks of K.
+// Shared-memory footprint of a CTA that stages `nb` blocks of K for tg * tl tiles.
 static void plan_smem(DecodePlan &pl, int M, int G, int spp, int nb) {
     const int mrows = M < 8 * pl.mt ? M : 8 * pl.mt;
-    // scale rows: stride = 16 mod 128 spreads the 8 channels of a warp read over the banks
+    // scale rows: a stride of 16 mod 32 bytes (64 m + 16) spreads the 8 channels of a
+    // warp read over distinct 16-byte bank groups
     const int nsc = spp == 4 ? G : (4 / spp) * nb;
-    pl.s_stride = round_up(nsc * 4, 128) + 16;
+    pl.s_stride = round_up(nsc * 4, 64) + 16;
     pl.act_stride = nb * kBlockK + kActPad;
-    pl.off_a = round_up(pl.tg * 16 * pl.s_stride, 128);
+    pl.off_a = round_up(pl.tg * pl.tl * 16 * pl.s_stride, 128);
     const size_t act = (size_t)(mrows + 1) * pl.act_stride;
     const size_t red = (size_t)kDecodeWarps * pl.mt * 4 * 32 * sizeof(float);
     pl.off_ring = round_up(pl.off_a + (int)(act > red ? act : red), 128);
-    pl.smem = pl.off_ring + (size_t)kDecodeWarps * kRound * 2 * 32 * 16;
+    pl.smem = pl.off_ring + (size_t)kDecodeWarps * pl.ring * 2 * 32 * 16;
 }
 
-// Tiles per CTA and K-chunks.  One tile per CTA (4 K-lanes) keeps each warp's
-// serial work shortest; several tiles per CTA share the staged activations,
-// which matters once there are many tokens.  Chunks are added when the staged
-// data would not fit, or when the grid would leave most SMs idle.
+// Launch plan.  Few tokens (one 8-token slab): one tile per CTA, its four warps take
+// interleaved blocks of K (shortest serial work per warp).  More tokens: two tiles per
+// CTA, two K-lanes each, sharing the staged activations.  Optionally (W2A8_TG=4) every
+// warp owns whole tiles and walks several of them, so that the activations a CTA stages
+// (M x chunk bytes, which rivals the weight stream once M is large) are read from L2
+// once per 4 * tl tiles.  K-chunks are added when the staged data would not fit, when
+// a warp would otherwise hold more cells than its ring, or when the grid would leave
+// most SMs idle.
 static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
     DecodePlan pl;
     pl.mt = decode_mt(M);
     pl.slabs = (M + 8 * pl.mt - 1) / (8 * pl.mt);
+    const int ntiles = N / 16;
     const int forced_tg = env_int("W2A8_TG", 0);
-    pl.tg = (forced_tg == 1 || forced_tg == 2 || forced_tg == 4)
-                ? forced_tg : (pl.mt == 1 ? 1 : (pl.mt == 2 ? 2 : 4));
-    pl.groups = (N / 16 + pl.tg - 1) / pl.tg;
+    // measured on B200: whole-tile warps (tg = 4) lose to K-lanes at every decode shape tried --
+    // the number of independent warps matters more than the activation traffic -- so they
+    // are only taken on request
+    pl.tg = (forced_tg == 1 || forced_tg == 2 || forced_tg == 4) ? forced_tg : (pl.mt == 1 ? 1 : 2);
+    pl.ring = pl.tg == 4 ? 8 : kRound;
+    pl.tl = 1;
     const int ks = kDecodeWarps / pl.tg;
-    int chunks = 1;
-    for (;;) {   // smallest chunk count whose staging fits the budget
-        const int bpc = (si.blocks + chunks - 1) / chunks;
-        plan_smem(pl, M, si.G, si.spp, bpc);
-        if ((int)pl.smem <= kSmemBudget || bpc == 1) break;
-        ++chunks;
-    }
     const int forced = env_int("W2A8_CHUNKS", 0);
-    if (forced > 0) {
+    int chunks = 1;
+    if (pl.tg == 4) {
+        // whole-tile warps: blocks per chunk (= cells per tile) 4, fewer if the grid is small
+        int nb = env_int("W2A8_NB", 4);
+        if (nb < 1) nb = 1;
+        if (nb > si.blocks) nb = si.blocks;
+        auto ctas = [&](int nb_) { return (long long)((ntiles + 3) / 4) * ((si.blocks + nb_ - 1) / nb_) * pl.slabs; };
+        while (forced <= 0 && nb > 1 && ctas(nb) < 200) nb /= 2;
+        chunks = (si.blocks + nb - 1) / nb;
         if (forced > chunks) chunks = forced;
+        if (chunks > si.blocks) chunks = si.blocks;
+        pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
+        pl.chunks = (si.blocks + pl.blocks_per_chunk - 1) / pl.blocks_per_chunk;
+        // tiles per warp: aim at about two CTAs per SM, within the shared-memory budget
+        int tl = env_int("W2A8_TL", 0);
+        if (tl <= 0) tl = (int)(((long long)ntiles * pl.chunks * pl.slabs) / (4 * 296));
+        if (tl < 1) tl = 1;
+        if (tl > 16) tl = 16;
+        for (;; --tl) {
+            pl.tl = tl;
+            plan_smem(pl, M, si.G, si.spp, pl.blocks_per_chunk);
+            if ((int)pl.smem <= kSmemBudget + 16 * 1024 || tl == 1) break;
+        }
+        pl.groups = (ntiles + 4 * pl.tl - 1) / (4 * pl.tl);
     } else {
-        // Measured on B200: a warp should hold all its cells in one round (its later
-        // rounds wait a full memory latency each), and the whole grid should field
-        // about 2000 warps or more so that enough loads are in flight; beyond that
-        // the cross-CTA sum costs more than further splitting gains.
-        const int one_round = (si.blocks + kRound * ks - 1) / (kRound * ks);
-        if (one_round > chunks) chunks = one_round;
-        const int min_warps = env_int("W2A8_MIN_WARPS", 2000);
-        while ((long long)pl.groups * pl.slabs * kDecodeWarps * chunks < min_warps &&
-               (si.blocks / (chunks * 2)) >= ks)
-            chunks *= 2;
+        pl.groups = (ntiles + pl.tg - 1) / pl.tg;
+        for (;;) {   // smallest chunk count whose staging fits the budget
+            const int bpc = (si.blocks + chunks - 1) / chunks;
+            plan_smem(pl, M, si.G, si.spp, bpc);
+            if ((int)pl.smem <= kSmemBudget || bpc == 1) break;
+            ++chunks;
+        }
+        if (forced > 0) {
+            if (forced > chunks) chunks = forced;
+        } else {
+            // Measured on B200: a warp should hold all its cells in its ring (later cells
+            // wait a full memory latency each), and the whole grid should field about 2000
+            // warps or more so that enough loads are in flight; beyond that the cross-CTA
+            // sum costs more than further splitting gains.
+            const int one_round = (si.blocks + pl.ring * ks - 1) / (pl.ring * ks);
+            if (one_round > chunks) chunks = one_round;
+            const int min_warps = env_int("W2A8_MIN_WARPS", 2000);
+            while ((long long)pl.groups * pl.slabs * kDecodeWarps * chunks < min_warps &&
+                   (si.blocks / (chunks * 2)) >= ks)
+                chunks *= 2;
+        }
+        if (chunks > si.blocks) chunks = si.blocks;
+        pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
+        pl.chunks = (si.blocks + pl.blocks_per_chunk - 1) / pl.blocks_per_chunk;
+        plan_smem(pl, M, si.G, si.spp, pl.blocks_per_chunk);
     }
-    if (chunks > si.blocks) chunks = si.blocks;
-    pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
-    pl.chunks = (si.blocks + pl.blocks_per_chunk - 1) / pl.blocks_per_chunk;
-    plan_smem(pl, M, si.G, si.spp, pl.blocks_per_chunk);
     // scale rows can be copied in 16-byte units when row pitch and chunk starts allow
     const int spb = si.spp == 4 ? 0 : 4 / si.spp;
     pl.s_vec = (si.spp != 4) && (si.G % 4 == 0) && ((spb * pl.blocks_per_chunk) % 4 == 0);
+    (void)K;
     return pl;
 }
 
@@ -474,7 +577,9 @@ size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si) {
     const DecodePlan pl = decode_plan(M, N, K, si);
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;   // >= any tile grouping
     // with an environment override in force, size for the finest split
-    const int chunks = (env_int("W2A8_CHUNKS", 0) > 0 || env_int("W2A8_TG", 0) > 0) ? si.blocks : pl.chunks;
+    const bool overridden = env_int("W2A8_CHUNKS", 0) > 0 || env_int("W2A8_TG", 0) > 0 ||
+                            env_int("W2A8_NB", 0) > 0 || env_int("W2A8_TL", 0) > 0;
+    const int chunks = overridden ? si.blocks : pl.chunks;
     size_t part = (size_t)(chunks > 1 ? chunks : 0) * M * N * sizeof(float);
     return kStatusBytes + counters + part;
 }
@@ -488,14 +593,15 @@ size_t decode_workspace_header_bytes(int M, int N, int K, const ShapeInfo &si) {
 
 template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
 static cudaError_t launch_decode_inst(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
+    constexpr int RING = TG == 4 ? 8 : kRound;
     static bool configured = false;   // one attribute call per instantiation and process
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, TG, ONE, PARTIALS>,
+        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, TG, RING, ONE, PARTIALS>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return launch_kernel(w2a8_decode_kernel<MT, SPP, TG, ONE, PARTIALS>, grid, dim3(kDecodeThreads),
+    return launch_kernel(w2a8_decode_kernel<MT, SPP, TG, RING, ONE, PARTIALS>, grid, dim3(kDecodeThreads),
                          smem, st, pdl_enabled(), p);
 }
 
@@ -539,7 +645,7 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
     p.y = y; p.partials = partials;
     p.M = M; p.N = N; p.K = K; p.G = si.G; p.group = group;
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
-    p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;
+    p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk; p.tiles_per_warp = pl.tl;
     p.s_stride = pl.s_stride; p.act_stride = pl.act_stride;
     p.off_a = pl.off_a; p.off_ring = pl.off_ring; p.s_vec = pl.s_vec;
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
