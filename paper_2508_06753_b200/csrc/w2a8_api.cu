@@ -60,10 +60,12 @@ w2_pack_kernel(const uint8_t *__restrict__ codes, uint32_t *__restrict__ packed,
 }
 
 // ---- a8_quantize -----------------------------------------------------------------
-// One CTA per token.  Pass 1: abs-max over the row (bf16 magnitudes order like
-// their bit patterns).  Pass 2: x * (1 / (amax / 127)), round to nearest even,
-// clamp, store 8 int8 per thread and step.  The row is re-read from L1/L2.
+// One CTA per token.  Abs-max over the row (bf16 magnitudes order like their bit
+// patterns), then x * (1 / (amax / 127)), round to nearest even, clamp, store 8
+// int8 per 16-byte vector.  Rows of up to kQuantRegThreads * 4 vectors (K <= 16384)
+// stay in registers between the two steps; longer rows are re-read from L1/L2.
 constexpr int kQuantThreads = 256;
+constexpr int kQuantRegThreads = 512;
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
 
@@ -123,6 +125,68 @@ a8_quantize_kernel(const uint16_t *__restrict__ x, int M, int K, int8_t *__restr
     }
 }
 
+__device__ __forceinline__ float quant_scale(uint32_t amax_bits, float *inv_out) {
+    const float amax = bf16_bits_to_float(amax_bits);
+    const float s = __fdiv_rn(amax, 127.0f);
+    float inv = __fdiv_rn(1.0f, s);
+    const bool dead = !(amax > 0.0f) || !(fabsf(inv) <= 3.402823466e38f);
+    *inv_out = dead ? 0.0f : inv;
+    return dead ? 0.0f : s;
+}
+
+// VPT 16-byte vectors per thread, all loaded before the reduction starts.
+template <int VPT>
+__global__ void __launch_bounds__(kQuantRegThreads)
+a8_quantize_reg_kernel(const uint16_t *__restrict__ x, int M, int K, int8_t *__restrict__ a,
+                       float *__restrict__ a_scale) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int m = blockIdx.x;
+    const uint4 *xr = reinterpret_cast<const uint4 *>(x + (size_t)m * K);
+    const int nvec = K / 8;
+    uint4 v[VPT];
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) {
+        const int i = threadIdx.x + j * kQuantRegThreads;
+        v[j] = i < nvec ? xr[i] : make_uint4(0u, 0u, 0u, 0u);
+    }
+    uint32_t amax_bits = 0;
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) {
+        const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            amax_bits = max(amax_bits, w[q] & 0x7FFFu);
+            amax_bits = max(amax_bits, (w[q] >> 16) & 0x7FFFu);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax_bits = max(amax_bits, __shfl_xor_sync(0xFFFFFFFFu, amax_bits, o));
+    __shared__ uint32_t wmax[kQuantRegThreads / 32];
+    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = amax_bits;
+    __syncthreads();
+    amax_bits = wmax[threadIdx.x & (kQuantRegThreads / 32 - 1)];
+#pragma unroll
+    for (int o = kQuantRegThreads / 64; o > 0; o >>= 1)
+        amax_bits = max(amax_bits, __shfl_xor_sync(0xFFFFFFFFu, amax_bits, o));
+
+    float inv;
+    const float s = quant_scale(amax_bits, &inv);
+    if (threadIdx.x == 0) a_scale[m] = s;
+    uint2 *ar = reinterpret_cast<uint2 *>(a + (size_t)m * K);
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) {
+        const int i = threadIdx.x + j * kQuantRegThreads;
+        if (i < nvec) {
+            uint2 o;
+            o.x = quant4(v[j].x, v[j].y, inv);
+            o.y = quant4(v[j].z, v[j].w, inv);
+            ar[i] = o;
+        }
+    }
+}
+
+
 }  // namespace w2a8
 
 // ====================================================================== C ABI ==
@@ -171,9 +235,22 @@ int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, voi
     if (!aligned16(x_bf16) || !aligned16(a) || (reinterpret_cast<uintptr_t>(a_scale) & 3u))
         return W2A8_ERR_ALIGN;
     if (int st = check_device()) return st;
-    cudaError_t e = launch_kernel(a8_quantize_kernel, dim3(M), dim3(kQuantThreads), 0,
-                                  (cudaStream_t)stream, pdl_enabled(),
-                                  reinterpret_cast<const uint16_t *>(x_bf16), M, K, a, a_scale);
+    const uint16_t *x = reinterpret_cast<const uint16_t *>(x_bf16);
+    cudaStream_t st = (cudaStream_t)stream;
+    const int vpt = (K / 8 + kQuantRegThreads - 1) / kQuantRegThreads;
+    cudaError_t e;
+    if (vpt <= 1)
+        e = launch_kernel(a8_quantize_reg_kernel<1>, dim3(M), dim3(kQuantRegThreads), 0, st,
+                          pdl_enabled(), x, M, K, a, a_scale);
+    else if (vpt <= 2)
+        e = launch_kernel(a8_quantize_reg_kernel<2>, dim3(M), dim3(kQuantRegThreads), 0, st,
+                          pdl_enabled(), x, M, K, a, a_scale);
+    else if (vpt <= 4)
+        e = launch_kernel(a8_quantize_reg_kernel<4>, dim3(M), dim3(kQuantRegThreads), 0, st,
+                          pdl_enabled(), x, M, K, a, a_scale);
+    else
+        e = launch_kernel(a8_quantize_kernel, dim3(M), dim3(kQuantThreads), 0, st,
+                          pdl_enabled(), x, M, K, a, a_scale);
     return e == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
 

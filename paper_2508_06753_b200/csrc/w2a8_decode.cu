@@ -142,30 +142,18 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
     for (int s = 0; s < 4; ++s) {
         if (s < R) {
             const uint32_t w0 = w0s[s], w1 = w1s[s];
-#ifdef W2A8_EXP_NOUNPACK
-            const uint32_t a0 = w0, a1 = w1, a2 = w0 + 1, a3 = w1 + 1, a4 = w0 + 2, a5 = w1 + 2, a6 = w0 + 3, a7 = w1 + 3;
-#else
             const uint32_t a0 = lane_codes(w0, 0), a1 = lane_codes(w1, 0);
             const uint32_t a2 = lane_codes(w0, 1), a3 = lane_codes(w1, 1);
             const uint32_t a4 = lane_codes(w0, 2), a5 = lane_codes(w1, 2);
             const uint32_t a6 = lane_codes(w0, 3), a7 = lane_codes(w1, 3);
-#endif
             const bool first = (s % SPP) == 0;
             const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
-#ifdef W2A8_EXP_NOB
-                const uint4 b = make_uint4(w0 ^ 1u, w1 ^ 2u, w0 ^ 3u, w1 ^ 4u);
-#else
                 const uint4 b = *reinterpret_cast<const uint4 *>(brow[mt] + kl * kBlockK + s * kSliceK);
-#endif
-#ifdef W2A8_EXP_NOMMA
-                D[mt][0] += a0 ^ b.x; D[mt][1] += a1 ^ b.y; D[mt][2] += a2 ^ a4 ^ b.z; D[mt][3] += a3 ^ a5 ^ a6 ^ a7 ^ b.w;
-#else
                 if (first) mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, magic);
                 else       mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, D[mt]);
                 mma_s8_16x8x32(D[mt], a4, a5, a6, a7, b.z, b.w, D[mt]);
-#endif
                 if (last) {
                     if constexpr (PARTIALS) {
                         const int gi = (SPP == 1) ? 4 * kb + s
@@ -180,11 +168,7 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
                                           (D[mt][i] - kMagicInt) >> 6);
                         }
                     } else {
-#ifdef W2A8_EXP_NOSCALE
-                        const float s0 = 0.5f, s1 = 0.25f;
-#else
                         const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
-#endif
                         acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
                         acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
                         if constexpr (!ONE) {

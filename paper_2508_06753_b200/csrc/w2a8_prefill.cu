@@ -327,9 +327,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     v.x = lane_codes(ws[sl], 0); v.y = lane_codes(ws[sl], 1);
                     v.z = lane_codes(ws[sl], 2); v.w = lane_codes(ws[sl], 3);
                     const int chunk = (4 * (sl & 1) + t) ^ (r & 7);
-#ifdef W2A8_EXP_NOSTS
-                    if (v.x == 0x12345678u)
-#endif
                     *reinterpret_cast<uint4 *>(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16) = v;
                 }
             }
