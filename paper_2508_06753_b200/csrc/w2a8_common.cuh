@@ -36,6 +36,20 @@ __device__ __forceinline__ uint32_t lane_codes(uint32_t word, int j) {
     return r;
 }
 
+// (acc0, acc1) += sc * (float(d0), float(d1)) for two accumulators in the magic-number form:
+// one packed subtract and one packed fused multiply-add (two issue slots for two values).
+__device__ __forceinline__ void promote2(float &acc0, float &acc1, int d0, int d1, float sc) {
+    asm("{\n\t.reg .b64 a, b, c, m;\n\t"
+        "mov.b64 a, {%2, %3};\n\t"
+        "mov.b64 m, {%5, %5};\n\t"
+        "add.rn.f32x2 a, a, m;\n\t"
+        "mov.b64 b, {%4, %4};\n\t"
+        "mov.b64 c, {%0, %1};\n\t"
+        "fma.rn.f32x2 c, a, b, c;\n\t"
+        "mov.b64 {%0, %1}, c;\n\t}"
+        : "+f"(acc0), "+f"(acc1) : "r"(d0), "r"(d1), "f"(sc), "f"(-kMagicFloat));
+}
+
 // Programmatic dependent launch: wait until the previous kernel of the stream
 // has completed and its writes are visible / let the next kernel start early.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -35,8 +35,6 @@ namespace w2a8 {
 
 constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kActPad = 64;                    // activation row stride = chunk bytes + 64
-constexpr int kSmemBudget = 64 * 1024;         // per CTA: scales + activations
 #ifndef W2A8_MINB
 #define W2A8_MINB(MT) ((MT) == 1 ? 7 : 3)
 #endif
@@ -55,11 +53,8 @@ struct DecodeParams {
     int M, N, K, G, group;
     int blocks, tail_slices, words_per_row;
     int chunks, blocks_per_chunk;
-    int s_stride;         // bytes per staged scale row
-    int act_stride;       // bytes per staged token row
-    int s_vec;            // scale rows can be copied in 16-byte units
-    int off_a;            // byte offset of the activation area in shared memory
-    int off_ring;         // byte offset of the per-lane weight rings
+    int blocks_per_group; // 256-k blocks per scale group (groups of 256 and more)
+    int s_vec;            // the scales of a cell and channel can be copied as one 16- or 8-byte unit
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------
@@ -77,6 +72,9 @@ __device__ __forceinline__ uint4 ld_stream_v4(const uint32_t *p) {
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -90,7 +88,11 @@ __device__ __forceinline__ void cp_async_wait_pending(int n) {
         case 0: cp_async_wait_group<0>(); break;
         case 1: cp_async_wait_group<1>(); break;
         case 2: cp_async_wait_group<2>(); break;
-        default: cp_async_wait_group<3>(); break;
+        case 3: cp_async_wait_group<3>(); break;
+        case 4: cp_async_wait_group<4>(); break;
+        case 5: cp_async_wait_group<5>(); break;
+        case 6: cp_async_wait_group<6>(); break;
+        default: cp_async_wait_group<7>(); break;
     }
 }
 
@@ -118,16 +120,26 @@ __device__ __forceinline__ unsigned long long global_ns() {
 #define W2A8_TRACE_POINT(i) do { } while (0)
 #endif
 
+__device__ __forceinline__ uint4 ld_act16(const int8_t *p) {
+    // plain (L1-allocating) load: the activations are written by the previous kernel of the
+    // stream and are only read after the wait for it, so the read-only path is not used
+    uint4 v;
+    asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
 // One cell: 4 slices x (unpack, 2 MMAs per token slab, promotion at group ends).
 // w0s/w1s: this lane's four words (one per slice) of channels n0+gq and n0+gq+8;
-// srow0/srow1: staged scale rows of the same channels.
+// sc0/sc1: the cell's scales of the same channels (shared memory, 16 bytes each);
+// brow[mt]: this lane's 16 activation bytes of slice 0 of the cell, token row of slab mt.
 template <int MT, int SPP, bool ONE, bool PARTIALS, bool FULL>
 __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32_t (&w0s)[4],
-                                             const uint32_t (&w1s)[4], const unsigned char *srow0,
-                                             const unsigned char *srow1,
-                                             const unsigned char *const (&brow)[MT], int kl,
-                                             int kb, int n0, int m0, int gq, int t,
-                                             float (&acc)[MT][4]) {
+                                             const uint32_t (&w1s)[4], const unsigned char *sc0,
+                                             const unsigned char *sc1,
+                                             const int8_t *const (&brow)[MT], int kb, int n0, int m0,
+                                             int gq, int t, float (&acc)[MT][4]) {
     // FULL: the block has all four slices (always, except possibly the last block of K)
     const int R = FULL ? 4 : p.tail_slices;
     const int magic[4] = {kMagicInt, kMagicInt, kMagicInt, kMagicInt};
@@ -139,16 +151,15 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
     float s0s[4 / SPP], s1s[4 / SPP];
     if constexpr (!PARTIALS) {
         if constexpr (SPP == 4) {
-            const int gi = (int)(((long long)kb * kBlockK) / p.group);
-            s0s[0] = reinterpret_cast<const float *>(srow0)[gi];
-            s1s[0] = reinterpret_cast<const float *>(srow1)[gi];
-        } else if constexpr (SPP == 2) {   // staged rows are 16-byte aligned: 8-byte loads are fine
-            const float2 v0 = reinterpret_cast<const float2 *>(srow0)[kl];
-            const float2 v1 = reinterpret_cast<const float2 *>(srow1)[kl];
+            s0s[0] = *reinterpret_cast<const float *>(sc0);
+            s1s[0] = *reinterpret_cast<const float *>(sc1);
+        } else if constexpr (SPP == 2) {
+            const float2 v0 = *reinterpret_cast<const float2 *>(sc0);
+            const float2 v1 = *reinterpret_cast<const float2 *>(sc1);
             s0s[0] = v0.x; s0s[1] = v0.y; s1s[0] = v1.x; s1s[1] = v1.y;
         } else {
-            const float4 v0 = reinterpret_cast<const float4 *>(srow0)[kl];
-            const float4 v1 = reinterpret_cast<const float4 *>(srow1)[kl];
+            const float4 v0 = *reinterpret_cast<const float4 *>(sc0);
+            const float4 v1 = *reinterpret_cast<const float4 *>(sc1);
             s0s[0] = v0.x; s0s[1] = v0.y; s0s[2] = v0.z; s0s[3] = v0.w;
             s1s[0] = v1.x; s1s[1] = v1.y; s1s[2] = v1.z; s1s[3] = v1.w;
         }
@@ -165,7 +176,7 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
             const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
-                const uint4 b = *reinterpret_cast<const uint4 *>(brow[mt] + kl * kBlockK + s * kSliceK);
+                const uint4 b = ld_act16(brow[mt] + s * kSliceK);
                 if (first) mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, magic);
                 else       mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, D[mt]);
                 mma_s8_16x8x32(D[mt], a4, a5, a6, a7, b.z, b.w, D[mt]);
@@ -184,10 +195,17 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
                         }
                     } else {
                         const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
-                        acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
-                        acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
-                        if constexpr (!ONE) {
+                        if constexpr (ONE) {
+                            acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
+                            acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
+                        } else if constexpr (MT == 1) {
+                            // packed fp32 pairs: measured faster for one slab, slower for more
+                            promote2(acc[mt][0], acc[mt][1], D[mt][0], D[mt][1], s0);
+                            promote2(acc[mt][2], acc[mt][3], D[mt][2], D[mt][3], s1);
+                        } else {
+                            acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
                             acc[mt][1] = fmaf(s0, __int_as_float(D[mt][1]) - kMagicFloat, acc[mt][1]);
+                            acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
                             acc[mt][3] = fmaf(s1, __int_as_float(D[mt][3]) - kMagicFloat, acc[mt][3]);
                         }
                     }
@@ -205,13 +223,16 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
 // A warp handles only a handful of cells, so the code around the cells is kept
 // short: one weight pointer per lane with cell c at a fixed stride from it, a
 // fully unrolled cell loop (slot and operand offsets are immediates), no
-// divisions and no 64-bit multiplies per cell.
+// divisions and no 64-bit multiplies per cell.  Warps do not meet before the
+// final sum over the K-lanes.
 template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS>
 __global__ void __launch_bounds__(kDecodeThreads, W2A8_MINB(MT))
 w2a8_decode_kernel(const DecodeParams p) {
     constexpr int KS = kDecodeWarps / TG;
-    constexpr int kSlotBytes = 2 * 32 * 16;     // one cell of one warp: two channels x 32 lanes x 16 B
-    constexpr int kWarpBytes = RING * kSlotBytes;
+    constexpr int kSlotBytes = 2 * 32 * 16;     // weights of one cell: two channels x 32 lanes x 16 B
+    constexpr int kScaleBytes = 16 * 16;        // scales of one cell: 16 channels x 16 B
+    constexpr int kWarpBytes = RING * (kSlotBytes + kScaleBytes);
+    constexpr int SPB = 4 / SPP;                // scales per block and channel
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -225,86 +246,66 @@ w2a8_decode_kernel(const DecodeParams p) {
     const int nb = kb_end - kb_begin;
     const int m0 = blockIdx.z * (8 * MT);
     const int mrows = min(8 * MT, p.M - m0);
-    unsigned char *sm_s = smem;                 // [tiles of the CTA * 16][s_stride]
-    unsigned char *acts = smem + p.off_a;       // [mrows][act_stride]
     W2A8_TRACE_POINT(0);
 
-    constexpr int SPB = 4 / SPP;                                  // scales per block and channel
-    const int sc_begin = (SPP == 4) ? 0 : SPB * kb_begin;
-    const int sc_end = (SPP == 4) ? p.G : min(SPB * kb_end, p.G);
-    const int rows_here = min(TG, ntiles - tile0) * 16;
-
-    // This warp's cells: cell c is block kb_begin + ks + c * KS of tile tile0 + tl
-    // (at most RING of them).
+    // This warp's cells: cell c is block kb0 + c * KS of tile tile0 + tl (at most RING of them).
     const int n0 = (tile0 + tl) * 16;
+    const int kb0 = kb_begin + ks;
     const int my_cells = (tile0 + tl < ntiles) ? (int)((unsigned)(nb - ks + KS - 1) / KS) : 0;
     // only the last block of K can have fewer than four slices
     const bool tail_cta = (kb_end == p.blocks) && (p.tail_slices != 4);
     const bool tail_mine = tail_cta && (nb - 1 - ks) >= 0 && (nb - 1 - ks) % KS == 0;   // ... and it is this warp's
     const int tail_cell = tail_mine ? (nb - 1 - ks) / KS : -1;
-
-    // Lane-private landing slots in shared memory: slot c of this lane holds the two 16-byte
-    // units (channels gq and gq+8) of cell c.  Only this lane writes and reads its slots, so
-    // cp.async.wait_group alone orders them (no warp barrier).
-    unsigned char *slots = smem + p.off_ring + warp * kWarpBytes + lane * 16;
-    const uint32_t slots_u32 = smem_u32(slots);
-    // word 4t of block kb_begin + ks in rows n0 + gq and n0 + gq + 8; cell c is 16 * KS words on
-    const uint32_t *wrow0 = p.packed + (size_t)(n0 + gq) * p.words_per_row + 16 * (kb_begin + ks) + 4 * t;
-    const uint32_t *wrow1 = wrow0 + (size_t)8 * p.words_per_row;
     const int full_cells = my_cells - (tail_mine ? 1 : 0);
+
+    // Landing slots of this warp in shared memory.  Weights: slot c of a lane holds its two
+    // 16-byte units (channels gq and gq+8) of cell c; only this lane writes and reads them.
+    // Scales: 16 bytes per channel and cell, copied by lanes 0..15 (one channel each) and read
+    // by the whole warp after a warp barrier.
+    unsigned char *wslots = smem + warp * kWarpBytes + lane * 16;
+    unsigned char *sslots = smem + warp * kWarpBytes + RING * kSlotBytes;
+    const uint32_t wslots_u32 = smem_u32(wslots);
+    const uint32_t sslot_u32 = smem_u32(sslots) + (lane & 15) * 16;
+    // word 4t of block kb0 in rows n0 + gq and n0 + gq + 8; cell c is 16 * KS words on
+    const uint32_t *wrow0 = p.packed + (size_t)(n0 + gq) * p.words_per_row + 16 * kb0 + 4 * t;
+    const uint32_t *wrow1 = wrow0 + (size_t)8 * p.words_per_row;
+    // first scale of block kb0 in row n0 + (lane & 15)
+    const float *srow = nullptr;
+    if constexpr (!PARTIALS) {
+        srow = p.w_scale + (size_t)(n0 + (lane & 15)) * p.G;
+        if constexpr (SPP != 4) srow += SPB * kb0;
+    }
     auto post_cell = [&](int c) {   // c is a constant after unrolling
-        cp_async16(slots_u32 + c * kSlotBytes, wrow0 + c * (16 * KS));
-        cp_async16(slots_u32 + c * kSlotBytes + 32 * 16, wrow1 + c * (16 * KS));
+        cp_async16(wslots_u32 + c * kSlotBytes, wrow0 + c * (16 * KS));
+        cp_async16(wslots_u32 + c * kSlotBytes + 32 * 16, wrow1 + c * (16 * KS));
+        if constexpr (!PARTIALS) {
+            if (lane < 16) {
+                if constexpr (SPP == 4) {
+                    const int kb = kb0 + c * KS;
+                    const int gi = p.blocks_per_group >= p.blocks ? 0 : kb / p.blocks_per_group;
+                    cp_async4(sslot_u32 + c * kScaleBytes, srow + gi);
+                } else if (p.s_vec) {
+                    if constexpr (SPP == 1) cp_async16(sslot_u32 + c * kScaleBytes, srow + c * (SPB * KS));
+                    else                    cp_async8(sslot_u32 + c * kScaleBytes, srow + c * (SPB * KS));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < SPB; ++i)
+                        cp_async4(sslot_u32 + c * kScaleBytes + 4 * i, srow + c * (SPB * KS) + i);
+                }
+            }
+        }
     };
 
-    // ---- the scales of the CTA's tiles for the whole chunk and all weights of this warp: none
-    //      of it depends on the previous kernel of the stream, so it is requested before the
-    //      wait for that kernel ------------------------------------------------------------
-    if constexpr (!PARTIALS) {
-        const int nsc = sc_end - sc_begin;
-        const float *src = p.w_scale + ((size_t)tile0 * 16 + warp) * p.G + sc_begin;
-        uint32_t dst = smem_u32(sm_s + warp * p.s_stride);
-        const size_t src_step = (size_t)kDecodeWarps * p.G;
-        const uint32_t dst_step = kDecodeWarps * p.s_stride;
-        if (p.s_vec && (nsc % 4 == 0)) {
-            const int nu = nsc / 4;
-#pragma unroll 1
-            for (int r = warp; r < rows_here; r += kDecodeWarps, src += src_step, dst += dst_step) {
-#pragma unroll 1
-                for (int j = lane; j < nu; j += 32) cp_async16(dst + 16 * j, src + 4 * j);
-            }
-        } else {
-#pragma unroll 1
-            for (int r = warp; r < rows_here; r += kDecodeWarps, src += src_step, dst += dst_step) {
-#pragma unroll 1
-                for (int j = lane; j < nsc; j += 32) cp_async4(dst + 4 * j, src + j);
-            }
-        }
-    }
+    // ---- weights and scales of all full cells: none of it depends on the previous kernel of
+    //      the stream, so it is requested before the wait for that kernel; one group per cell --
 #pragma unroll
-    for (int j = 0; j < RING; ++j)
+    for (int j = 0; j < RING; ++j) {
         if (j < full_cells) post_cell(j);
-    cp_async_commit();
-    W2A8_TRACE_POINT(1);
-    pdl_launch_dependents();
-    pdl_wait();
-    W2A8_TRACE_POINT(2);
-
-    // ---- next group: the activations of this chunk, [mrows][chunk k (+pad)] ---------------
-    {
-        const int kunits = min(nb * kBlockK, p.K - kb_begin * kBlockK) / 16;
-        const int8_t *src = p.a + (size_t)m0 * p.K + (size_t)kb_begin * kBlockK + threadIdx.x * 16;
-        uint32_t dst = smem_u32(acts) + threadIdx.x * 16;
-#pragma unroll 1
-        for (int r = 0; r < mrows; ++r, src += p.K, dst += p.act_stride) {
-#pragma unroll 1
-            for (int cu = threadIdx.x; cu < kunits; cu += kDecodeThreads)
-                cp_async16(dst + (cu - threadIdx.x) * 16, src + (cu - threadIdx.x) * 16);
-        }
         cp_async_commit();
     }
     if (tail_mine) {
-        // trailing block of K with R < 4 slices: this lane's words are t*R .. t*R+R-1 of the block
+        // trailing block of K with R < 4 slices: this lane's words are t*R .. t*R+R-1 of the
+        // block; it has R (SPP 1), (R+1)/2 (SPP 2) or one scale per channel
         const int R = p.tail_slices;
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
@@ -313,12 +314,25 @@ w2a8_decode_kernel(const DecodeParams p) {
             v.x = __ldg(wp);
             if (R > 1) v.y = __ldg(wp + 1);
             if (R > 2) v.z = __ldg(wp + 2);
-            *reinterpret_cast<uint4 *>(slots + tail_cell * kSlotBytes + r * (32 * 16)) = v;
+            *reinterpret_cast<uint4 *>(wslots + tail_cell * kSlotBytes + r * (32 * 16)) = v;
+        }
+        if constexpr (!PARTIALS) {
+            if (lane < 16) {
+                float *dst = reinterpret_cast<float *>(sslots + tail_cell * kScaleBytes + lane * 16);
+                if constexpr (SPP == 4) {
+                    const int kb = kb0 + tail_cell * KS;
+                    dst[0] = __ldg(srow + (p.blocks_per_group >= p.blocks ? 0 : kb / p.blocks_per_group));
+                } else {
+                    const int nsc = (R + SPP - 1) / SPP;
+                    for (int i = 0; i < nsc; ++i) dst[i] = __ldg(srow + tail_cell * (SPB * KS) + i);
+                }
+            }
         }
     }
-    cp_async_wait_all();
-    __syncthreads();                   // scales and activations are shared by the CTA
-    W2A8_TRACE_POINT(3);
+    W2A8_TRACE_POINT(1);
+    pdl_launch_dependents();
+    pdl_wait();
+    W2A8_TRACE_POINT(2);
 
     float acc[MT][4];
 #pragma unroll
@@ -326,35 +340,43 @@ w2a8_decode_kernel(const DecodeParams p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
 
-    // This lane's token row of each slab.  Token columns of an MMA are independent, and
-    // columns beyond M are never stored, so they may read any staged row: the last one.
-    const unsigned char *brow[MT];
+    // This lane's activation bytes of block kb0: token row of each slab.  Token columns of an
+    // MMA are independent, and columns beyond M are never stored, so they may read any row:
+    // the last one.  The activations are read through L1, which all CTAs of an SM share.
+    const int8_t *brow[MT];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
-        brow[mt] = acts + min(8 * mt + gq, mrows - 1) * p.act_stride + t * 16;
+        brow[mt] = p.a + (size_t)(m0 + min(8 * mt + gq, mrows - 1)) * p.K + (size_t)kb0 * kBlockK + t * 16;
     const size_t MN = (size_t)p.M * p.N;
-    const unsigned char *srow0 = sm_s + (tl * 16 + gq) * p.s_stride;   // floats from sc_begin on
-    const unsigned char *srow1 = srow0 + 8 * p.s_stride;
+    const unsigned char *sc0 = sslots + gq * 16, *sc1 = sc0 + 8 * 16;
 
 #pragma unroll
     for (int c = 0; c < RING; ++c) {
         if (c < full_cells) {                                 // warp-uniform
-            const uint4 wa = *reinterpret_cast<const uint4 *>(slots + c * kSlotBytes);
-            const uint4 wb = *reinterpret_cast<const uint4 *>(slots + c * kSlotBytes + 32 * 16);
+            cp_async_wait_pending(RING - 1 - c);
+            __syncwarp();                                     // the scales were copied by other lanes
+            const uint4 wa = *reinterpret_cast<const uint4 *>(wslots + c * kSlotBytes);
+            const uint4 wb = *reinterpret_cast<const uint4 *>(wslots + c * kSlotBytes + 32 * 16);
             const uint32_t w0s[4] = {wa.x, wa.y, wa.z, wa.w};
             const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
-            const int kl = ks + c * KS;
-            compute_cell<MT, SPP, ONE, PARTIALS, true>(p, w0s, w1s, srow0, srow1, brow, kl, kb_begin + kl,
-                                                       n0, m0, gq, t, acc);
+            const int8_t *bc[MT];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + c * (KS * kBlockK);
+            compute_cell<MT, SPP, ONE, PARTIALS, true>(p, w0s, w1s, sc0 + c * kScaleBytes, sc1 + c * kScaleBytes,
+                                                       bc, kb0 + c * KS, n0, m0, gq, t, acc);
         }
     }
-    if (tail_mine) {   // the trailing block is this warp's last cell; its words were stored directly
-        const uint4 wa = *reinterpret_cast<const uint4 *>(slots + tail_cell * kSlotBytes);
-        const uint4 wb = *reinterpret_cast<const uint4 *>(slots + tail_cell * kSlotBytes + 32 * 16);
+    if (tail_mine) {   // the trailing block is this warp's last cell; its words and scales were stored directly
+        __syncwarp();
+        const uint4 wa = *reinterpret_cast<const uint4 *>(wslots + tail_cell * kSlotBytes);
+        const uint4 wb = *reinterpret_cast<const uint4 *>(wslots + tail_cell * kSlotBytes + 32 * 16);
         const uint32_t w0s[4] = {wa.x, wa.y, wa.z, wa.w};
         const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
-        const int kl = ks + tail_cell * KS;
-        compute_cell<MT, SPP, ONE, PARTIALS, false>(p, w0s, w1s, srow0, srow1, brow, kl, kb_begin + kl,
+        const int8_t *bc[MT];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + (size_t)tail_cell * (KS * kBlockK);
+        compute_cell<MT, SPP, ONE, PARTIALS, false>(p, w0s, w1s, sc0 + tail_cell * kScaleBytes,
+                                                    sc1 + tail_cell * kScaleBytes, bc, kb0 + tail_cell * KS,
                                                     n0, m0, gq, t, acc);
     }
     W2A8_TRACE_POINT(5);
@@ -362,9 +384,9 @@ w2a8_decode_kernel(const DecodeParams p) {
     if constexpr (!PARTIALS) {
         // ---- sum the K-lanes of each tile in a fixed order -----------------------
         // Lane (gq, t) holds channels n0+gq, n0+gq+8 for tokens 2t, 2t+1 of each slab.  Each
-        // warp parks its sums in its own (now idle) landing slots.
-        float *red = reinterpret_cast<float *>(smem + p.off_ring + warp * kWarpBytes);
-        const float *red0 = reinterpret_cast<const float *>(smem + p.off_ring);
+        // warp parks its sums in its own (now idle) weight slots.
+        float *red = reinterpret_cast<float *>(smem + warp * kWarpBytes);
+        const float *red0 = reinterpret_cast<const float *>(smem);
         constexpr int kWarpFloats = kWarpBytes / 4;
         __syncwarp();      // every lane has read its slots
         if constexpr (ONE) {
@@ -461,52 +483,30 @@ extern "C" int w2a8_debug_set_trace(void *buffer, const float *y0, unsigned long
 int env_int(const char *name, int dflt);
 
 static inline int decode_mt(int M) { return M > 32 ? 4 : (M + 7) / 8; }
-static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct DecodePlan {
-    int mt, tg, ring, chunks, blocks_per_chunk, slabs, groups;
-    int s_stride, act_stride, off_a, off_ring, s_vec;
+    int mt, tg, ring, chunks, blocks_per_chunk, slabs, groups, s_vec;
     size_t smem;
 };
 
-// Shared-memory footprint of a CTA that stages `nb` blocks of K for tg tiles.
-static void plan_smem(DecodePlan &pl, int M, int G, int spp, int nb) {
-    const int mrows = M < 8 * pl.mt ? M : 8 * pl.mt;
-    // scale rows: a stride of 16 mod 32 bytes (64 m + 16) spreads the 8 channels of a
-    // warp read over distinct 16-byte bank groups
-    const int nsc = spp == 4 ? G : (4 / spp) * nb;
-    pl.s_stride = round_up(nsc * 4, 64) + 16;
-    pl.act_stride = nb * kBlockK + kActPad;
-    pl.off_a = round_up(pl.tg * 16 * pl.s_stride, 128);
-    pl.off_ring = round_up(pl.off_a + mrows * pl.act_stride, 128);
-    // landing slots of the four warps; afterwards each warp parks its MT * 4 * 32 partial
-    // sums (at most 2 KB) in its own slots for the K-lane sum
-    pl.smem = pl.off_ring + (size_t)kDecodeWarps * pl.ring * 2 * 32 * 16;
-}
-
 // Launch plan.  Few tokens (one 8-token slab): one tile per CTA, its four warps take
 // interleaved blocks of K (shortest serial work per warp).  More tokens: two tiles per
-// CTA, two K-lanes each, sharing the staged activations.  K-chunks are added when the
-// staged data would not fit, when a warp would otherwise hold more cells than its ring,
-// or when the grid would leave most SMs idle.
+// CTA, two K-lanes each.  K-chunks are added when a warp would otherwise have more cells
+// than landing slots, or when the grid would leave most SMs idle.
 static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
     DecodePlan pl;
     pl.mt = decode_mt(M);
     pl.slabs = (M + 8 * pl.mt - 1) / (8 * pl.mt);
     const int ntiles = N / 16;
     const int forced_tg = env_int("W2A8_TG", 0);
-    pl.tg = (forced_tg == 1 || forced_tg == 2) ? forced_tg : (pl.mt == 1 ? 1 : 2);
-    pl.ring = kRound;
+    pl.tg = (forced_tg == 1 || forced_tg == 2) ? forced_tg : 1;
+    { const int r = env_int("W2A8_RING", 0); pl.ring = (r == 4 || r == 8) ? r : kRound; }
     const int ks = kDecodeWarps / pl.tg;
     const int forced = env_int("W2A8_CHUNKS", 0);
     int chunks = 1;
     pl.groups = (ntiles + pl.tg - 1) / pl.tg;
-    for (;;) {   // smallest chunk count whose staging fits the budget
-        const int bpc = (si.blocks + chunks - 1) / chunks;
-        plan_smem(pl, M, si.G, si.spp, bpc);
-        if ((int)pl.smem <= kSmemBudget || bpc == 1) break;
-        ++chunks;
-    }
+    // landing slots: 1 KB of weights and 256 B of scales per cell and warp
+    pl.smem = (size_t)kDecodeWarps * pl.ring * (2 * 32 * 16 + 16 * 16);
     // a warp holds all its cells at once: at most ring * ks blocks per chunk
     const int one_round = (si.blocks + pl.ring * ks - 1) / (pl.ring * ks);
     if (one_round > chunks) chunks = one_round;
@@ -524,10 +524,8 @@ static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
     if (chunks > si.blocks) chunks = si.blocks;
     pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
     pl.chunks = (si.blocks + pl.blocks_per_chunk - 1) / pl.blocks_per_chunk;
-    plan_smem(pl, M, si.G, si.spp, pl.blocks_per_chunk);
-    // scale rows can be copied in 16-byte units when row pitch and chunk starts allow
-    const int spb = si.spp == 4 ? 0 : 4 / si.spp;
-    pl.s_vec = (si.spp != 4) && (si.G % 4 == 0) && ((spb * pl.blocks_per_chunk) % 4 == 0);
+    pl.s_vec = (si.spp == 1 && si.G % 4 == 0) || (si.spp == 2 && si.G % 2 == 0);
+    (void)M;
     (void)K;
     return pl;
 }
@@ -538,7 +536,8 @@ size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si) {
     const DecodePlan pl = decode_plan(M, N, K, si);
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;   // >= any tile grouping
     // with an environment override in force, size for the finest split
-    const bool overridden = env_int("W2A8_CHUNKS", 0) > 0 || env_int("W2A8_TG", 0) > 0;
+    const bool overridden = env_int("W2A8_CHUNKS", 0) > 0 || env_int("W2A8_TG", 0) > 0 ||
+                            env_int("W2A8_RING", 0) > 0;
     const int chunks = overridden ? si.blocks : pl.chunks;
     size_t part = (size_t)(chunks > 1 ? chunks : 0) * M * N * sizeof(float);
     return kStatusBytes + counters + part;
@@ -551,9 +550,8 @@ size_t decode_workspace_header_bytes(int M, int N, int K, const ShapeInfo &si) {
     return kStatusBytes + ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
 }
 
-template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
-static cudaError_t launch_decode_inst(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
-    constexpr int RING = kRound;
+template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS>
+static cudaError_t launch_decode_ring(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
     static bool configured = false;   // one attribute call per instantiation and process
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, TG, RING, ONE, PARTIALS>,
@@ -565,20 +563,26 @@ static cudaError_t launch_decode_inst(const DecodeParams &p, dim3 grid, size_t s
                          smem, st, pdl_enabled(), p);
 }
 
+template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
+static cudaError_t launch_decode_inst(const DecodeParams &p, int ring, dim3 grid, size_t smem, cudaStream_t st) {
+    if (ring == 8) return launch_decode_ring<MT, SPP, TG, 8, ONE, PARTIALS>(p, grid, smem, st);
+    return launch_decode_ring<MT, SPP, TG, kRound, ONE, PARTIALS>(p, grid, smem, st);
+}
+
 template <int MT, int SPP, int TG>
-static cudaError_t launch_decode_tg(const DecodeParams &p, bool want_partials, dim3 grid, size_t smem,
+static cudaError_t launch_decode_tg(const DecodeParams &p, int ring, bool want_partials, dim3 grid, size_t smem,
                                     cudaStream_t st) {
-    if (want_partials) return launch_decode_inst<MT, SPP, TG, false, true>(p, grid, smem, st);
-    if (MT == 1 && p.M == 1) return launch_decode_inst<1, SPP, TG, true, false>(p, grid, smem, st);
-    return launch_decode_inst<MT, SPP, TG, false, false>(p, grid, smem, st);
+    if (want_partials) return launch_decode_inst<MT, SPP, TG, false, true>(p, ring, grid, smem, st);
+    if (MT == 1 && p.M == 1) return launch_decode_inst<1, SPP, TG, true, false>(p, ring, grid, smem, st);
+    return launch_decode_inst<MT, SPP, TG, false, false>(p, ring, grid, smem, st);
 }
 
 template <int MT, int SPP>
 static cudaError_t launch_decode_mt(const DecodeParams &p, const DecodePlan &pl, bool want_partials,
                                     cudaStream_t st) {
     dim3 grid(pl.groups, pl.chunks, pl.slabs);
-    if (pl.tg == 1) return launch_decode_tg<MT, SPP, 1>(p, want_partials, grid, pl.smem, st);
-    return launch_decode_tg<MT, SPP, 2>(p, want_partials, grid, pl.smem, st);
+    if (pl.tg == 1) return launch_decode_tg<MT, SPP, 1>(p, pl.ring, want_partials, grid, pl.smem, st);
+    return launch_decode_tg<MT, SPP, 2>(p, pl.ring, want_partials, grid, pl.smem, st);
 }
 
 template <int SPP>
@@ -603,8 +607,7 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
     p.M = M; p.N = N; p.K = K; p.G = si.G; p.group = group;
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
     p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;
-    p.s_stride = pl.s_stride; p.act_stride = pl.act_stride;
-    p.off_a = pl.off_a; p.off_ring = pl.off_ring; p.s_vec = pl.s_vec;
+    p.blocks_per_group = (group + kBlockK - 1) / kBlockK; p.s_vec = pl.s_vec;
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
     char *base = reinterpret_cast<char *>(workspace);
     p.status = reinterpret_cast<int *>(base);
