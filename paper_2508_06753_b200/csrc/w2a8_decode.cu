@@ -35,8 +35,11 @@ namespace w2a8 {
 
 constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
+// Resident CTAs per SM the compiler must allow.  One slab: 8 (64 registers), which also lets
+// every 4-CTA cluster of a split-K launch be resident at once (clusters are placed inside one
+// GPC; with 7 per SM the last few clusters of a 1024-CTA grid waited for a second round).
 #ifndef W2A8_MINB
-#define W2A8_MINB(MT) ((MT) == 1 ? 7 : 3)
+#define W2A8_MINB(MT) ((MT) == 1 ? 8 : 3)
 #endif
 constexpr int kRound = 4;                      // cells a lane keeps in flight (ring depth, power of 2)
 
@@ -53,6 +56,7 @@ struct DecodeParams {
     int M, N, K, G, group;
     int blocks, tail_slices, words_per_row;
     int chunks, blocks_per_chunk;
+    int cluster;          // chunks > 1 and the chunks of a tile form one thread-block cluster
     int blocks_per_group; // 256-k blocks per scale group (groups of 256 and more)
     int s_vec;            // the scales of a cell and channel can be copied as one 16- or 8-byte unit
 };
@@ -398,53 +402,72 @@ w2a8_decode_kernel(const DecodeParams p) {
                 for (int i = 0; i < 4; ++i) red[(mt * 4 + i) * 32 + lane] = acc[mt][i];
         }
         __syncthreads();
-        if constexpr (ONE) {
-            // one token: 16 outputs per tile
-            const int etl = threadIdx.x >> 4, nn = (tile0 + etl) * 16 + (threadIdx.x & 15);
-            const bool mine = threadIdx.x < TG * 16 && nn < p.N;
-            if (mine) {
-                float v = 0.f;
-#pragma unroll
-                for (int k2 = 0; k2 < KS; ++k2) v += red0[(k2 * TG + etl) * kWarpFloats + (threadIdx.x & 15)];
-                if (p.chunks == 1) p.y[nn] = v * (p.a_scale[0] * (1.0f / kCodeGain));
-                else __stcg(p.ws + chunk * MN + nn, v);
-            }
-            W2A8_TRACE_POINT(6);
-            if (p.chunks == 1) return;
-            // ---- split-K: the last CTA to arrive sums the partial outputs in order ---
-            __threadfence();
-            __syncthreads();
-            unsigned *counter = p.counters + tile0;
-            if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) == (unsigned)p.chunks - 1u);
-            __syncthreads();
-            if (!is_last) return;
-            __threadfence();
-            if (mine) {
-                float v = 0.f;
-                for (int ch = 0; ch < p.chunks; ++ch) v += __ldcg(p.ws + ch * MN + nn);
-                p.y[nn] = v * (p.a_scale[0] * (1.0f / kCodeGain));
-            }
-            if (threadIdx.x == 0) *counter = 0u;   // leave the workspace reusable
-            W2A8_TRACE_POINT(7);
-        } else {
-            // element e of the CTA: (tile etl, slab mt, quad register i, lane el)
-            for (int e = threadIdx.x; e < TG * MT * 128; e += kDecodeThreads) {
+
+        // Outputs of the CTA as a flat list: element e = (tile etl, slab mt, quad register i,
+        // lane el); with one token only channel (e & 15) of tile (e >> 4) for e < 16 * TG.
+        constexpr int kElems = ONE ? TG * 16 : TG * MT * 128;
+        auto locate = [&](int e, int &mm, int &nn) -> bool {
+            if constexpr (ONE) {
+                mm = 0;
+                nn = (tile0 + (e >> 4)) * 16 + (e & 15);
+            } else {
                 const int el = e & 31, ei = (e >> 5) % (MT * 4), etl = e / (MT * 128);
-                const int mt = ei >> 2, i = ei & 3;
-                float v = 0.f;
+                mm = m0 + 8 * (ei >> 2) + 2 * (el & 3) + (ei & 1);
+                nn = (tile0 + etl) * 16 + (el >> 2) + 8 * ((ei & 3) >> 1);
+            }
+            return mm < p.M && nn < p.N;
+        };
+        auto cta_sum = [&](int e) -> float {
+            float v = 0.f;
+            if constexpr (ONE) {
+#pragma unroll
+                for (int k2 = 0; k2 < KS; ++k2) v += red0[(k2 * TG + (e >> 4)) * kWarpFloats + (e & 15)];
+            } else {
+                const int el = e & 31, ei = (e >> 5) % (MT * 4), etl = e / (MT * 128);
 #pragma unroll
                 for (int k2 = 0; k2 < KS; ++k2) v += red0[(k2 * TG + etl) * kWarpFloats + ei * 32 + el];
-                const int mm = m0 + 8 * mt + 2 * (el & 3) + (i & 1);
-                const int nn = (tile0 + etl) * 16 + (el >> 2) + 8 * (i >> 1);
-                if (mm < p.M && nn < p.N) {
-                    if (p.chunks == 1) p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
-                    else __stcg(p.ws + chunk * MN + (size_t)mm * p.N + nn, v);
-                }
+            }
+            return v;
+        };
+
+        if (p.chunks == 1) {
+            for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
+                int mm, nn;
+                if (locate(e, mm, nn))
+                    p.y[(size_t)mm * p.N + nn] = cta_sum(e) * (p.a_scale[mm] * (1.0f / kCodeGain));
             }
             W2A8_TRACE_POINT(6);
-            if (p.chunks == 1) return;
-
-            // ---- split-K: the last CTA to arrive sums the partial outputs in order ---
+        } else if (p.cluster) {
+            // ---- split-K inside a thread-block cluster: the chunks of a tile are the CTAs of one
+            //      cluster.  Every CTA writes its sums into the receive buffer of rank 0 (remote
+            //      shared memory); after one cluster barrier rank 0 adds them chunk by chunk. ----
+            const uint32_t recv_u32 = smem_u32(smem + kDecodeWarps * kWarpBytes);
+            const float *recv = reinterpret_cast<const float *>(smem + kDecodeWarps * kWarpBytes);
+            const uint32_t rank = cluster_ctarank();
+            for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
+                int mm, nn;
+                if (locate(e, mm, nn)) st_cluster_f32(recv_u32 + (rank * kElems + e) * 4, 0, cta_sum(e));
+            }
+            cluster_sync();
+            W2A8_TRACE_POINT(6);
+            if (rank != 0) return;
+            for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
+                int mm, nn;
+                if (locate(e, mm, nn)) {
+                    float v = 0.f;
+                    for (int ch = 0; ch < p.chunks; ++ch) v += recv[ch * kElems + e];
+                    p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
+                }
+            }
+            W2A8_TRACE_POINT(7);
+        } else {
+            // ---- split-K through the workspace: the last CTA to arrive sums the partial outputs
+            //      chunk by chunk ------------------------------------------------------------------
+            for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
+                int mm, nn;
+                if (locate(e, mm, nn)) __stcg(p.ws + chunk * MN + (size_t)mm * p.N + nn, cta_sum(e));
+            }
+            W2A8_TRACE_POINT(6);
             __threadfence();
             __syncthreads();
             unsigned *counter = p.counters + (size_t)blockIdx.z * ntiles + tile0;
@@ -452,12 +475,9 @@ w2a8_decode_kernel(const DecodeParams p) {
             __syncthreads();
             if (!is_last) return;
             __threadfence();
-            for (int e = threadIdx.x; e < TG * MT * 128; e += kDecodeThreads) {
-                const int el = e & 31, ei = (e >> 5) % (MT * 4), etl = e / (MT * 128);
-                const int mt = ei >> 2, i = ei & 3;
-                const int mm = m0 + 8 * mt + 2 * (el & 3) + (i & 1);
-                const int nn = (tile0 + etl) * 16 + (el >> 2) + 8 * (i >> 1);
-                if (mm < p.M && nn < p.N) {
+            for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
+                int mm, nn;
+                if (locate(e, mm, nn)) {
                     float v = 0.f;
                     for (int ch = 0; ch < p.chunks; ++ch) v += __ldcg(p.ws + ch * MN + (size_t)mm * p.N + nn);
                     p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
@@ -485,7 +505,7 @@ int env_int(const char *name, int dflt);
 static inline int decode_mt(int M) { return M > 32 ? 4 : (M + 7) / 8; }
 
 struct DecodePlan {
-    int mt, tg, ring, chunks, blocks_per_chunk, slabs, groups, s_vec;
+    int mt, tg, ring, chunks, blocks_per_chunk, slabs, groups, s_vec, cluster;
     size_t smem;
 };
 
@@ -525,6 +545,10 @@ static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
     pl.blocks_per_chunk = (si.blocks + chunks - 1) / chunks;
     pl.chunks = (si.blocks + pl.blocks_per_chunk - 1) / pl.blocks_per_chunk;
     pl.s_vec = (si.spp == 1 && si.G % 4 == 0) || (si.spp == 2 && si.G % 2 == 0);
+    // up to 8 chunks (the portable cluster size) are summed inside a thread-block cluster;
+    // rank 0 receives one partial output per chunk and element of the CTA
+    pl.cluster = pl.chunks > 1 && pl.chunks <= 8 && env_int("W2A8_CLUSTER", 1) != 0;
+    if (pl.cluster) pl.smem += (size_t)pl.chunks * pl.tg * pl.mt * 128 * sizeof(float);
     (void)M;
     (void)K;
     return pl;
@@ -559,8 +583,9 @@ static cudaError_t launch_decode_ring(const DecodeParams &p, dim3 grid, size_t s
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return launch_kernel(w2a8_decode_kernel<MT, SPP, TG, RING, ONE, PARTIALS>, grid, dim3(kDecodeThreads),
-                         smem, st, pdl_enabled(), p);
+    return launch_kernel_cluster(w2a8_decode_kernel<MT, SPP, TG, RING, ONE, PARTIALS>, grid,
+                                 dim3(kDecodeThreads), smem, st, pdl_enabled(),
+                                 p.cluster ? (unsigned)p.chunks : 1u, p);
 }
 
 template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
@@ -608,6 +633,7 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
     p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;
     p.blocks_per_group = (group + kBlockK - 1) / kBlockK; p.s_vec = pl.s_vec;
+    p.cluster = (pl.cluster && partials == nullptr) ? 1 : 0;
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;
     char *base = reinterpret_cast<char *>(workspace);
     p.status = reinterpret_cast<int *>(base);
