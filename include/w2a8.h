@@ -92,7 +92,7 @@ int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, voi
 
 /*
  * Workspace size in bytes that w2a8_gemm / w2a8_gemm_partials need for this
- * problem (split-K partial outputs and their arrival counters).  Returns 0 for
+ * problem (status word, split-K arrival counters and partial outputs).  Returns 0 for
  * shapes that violate the shape rules.  The workspace must be zero-filled once
  * (w2a8_workspace_init) before its first use; the kernels leave it reusable.
  * One workspace serves any sequence of calls on one stream as long as it is at
@@ -125,8 +125,9 @@ int w2a8_workspace_status(const void *workspace, void *stream);
  *   packed  [N][K/16] uint32 (from w2_pack)        w_scale [N][K/group] fp32
  *   y       [M][N] fp32, row-major, fully overwritten
  *   workspace / workspace_bytes: see w2a8_workspace_bytes.
- * M <= 32 takes the memory-bound decode kernel (weights streamed once); larger
- * M takes the tensor-core prefill path.
+ * M >= 64 with N % 128 == 0 and K % 256 == 0 takes the tensor-core kernel
+ * (tcgen05, 128 x 128 output tiles); everything else takes the memory-bound
+ * streaming kernel (weights read once per slab of up to 32 tokens).
  */
 int w2a8_gemm(const int8_t *a, const float *a_scale, const uint32_t *packed,
               const float *w_scale, float *y, int M, int N, int K, int group,

@@ -8,23 +8,28 @@
 // Work split.  A "cell" is one 16-channel tile x one 256-k block: 1 KB of packed
 // weights plus its scales.  A CTA of 4 warps owns TG tiles and one chunk of the
 // contraction; its warps are arranged TG tiles x KS = 4 / TG K-lanes, and the
-// K-lanes take interleaved blocks of the chunk.  The K-lanes of a tile are
-// summed through shared memory in a fixed order; chunks (grid.y, only used when
-// the shape would otherwise leave SMs idle or the data would not fit in shared
-// memory) are summed through the workspace by the last CTA to arrive, also in a
-// fixed order.  grid.z walks 8*MT-token slabs.
+// K-lanes take interleaved blocks of the chunk, at most RING cells each.  The
+// K-lanes of a tile are summed through shared memory in a fixed order.  Chunks
+// (grid.y; used when K has more blocks than the K-lanes can hold, or when the
+// grid would leave SMs idle) are summed in chunk order: inside a thread-block
+// cluster when there are at most 8 of them (every CTA writes its sums into the
+// shared memory of the cluster's first CTA, one cluster barrier, no trip through
+// global memory), else through the workspace by the last CTA to arrive.
+// grid.z walks 8*MT-token slabs.
 //
-// Pipeline.  Every lane owns a small ring of 16-byte slots in shared memory and
-// fills it with per-thread asynchronous copies (cp.async), two per cell (its two
-// channels).  By default a warp's cells all fit its ring, so the whole weight
-// stream of the CTA is in flight at once.  The scales and the first half of the
-// ring are requested before the kernel waits for the previous kernel of the
-// stream (weights and scales are frozen; only activations depend on it), so
-// under programmatic dependent launch the weight stream of this kernel overlaps
-// the tail of the previous one.  The activations of the chunk are requested
-// right behind that first half (so that they do not queue behind the whole
-// weight stream), then the second half.  Scales and activations are staged once
-// per CTA in shared memory.
+// Data movement.  Nothing is staged per CTA, and the warps of a CTA do not meet
+// before the final sum.  Weights: every lane owns 16-byte landing slots in
+// shared memory and fills them with per-thread asynchronous copies (cp.async,
+// L1 bypass), two per cell (its two channels); all cells of a warp are
+// requested at once, so the whole weight stream of the CTA is in flight from
+// the start.  Scales: lanes 0..15 copy the 16 bytes per channel and cell into
+// per-warp slots the same way.  Both are frozen data, so they are requested
+// before the kernel waits for the previous kernel of the stream; under
+// programmatic dependent launch the weight stream of this kernel therefore
+// overlaps the tail of the previous one.  Activations (the only input that can
+// depend on the previous kernel) are read after that wait, straight from global
+// memory through L1: all CTAs of an SM share them there, which keeps the L2
+// traffic at one copy per SM instead of one per CTA.
 //
 // One 128-bit unit per lane and channel holds word t of each of the four 64-k
 // slices of a block -- exactly what the four lanes of an MMA quad must supply
@@ -41,7 +46,7 @@ constexpr int kDecodeThreads = kDecodeWarps * 32;
 #ifndef W2A8_MINB
 #define W2A8_MINB(MT) ((MT) == 1 ? 8 : 3)
 #endif
-constexpr int kRound = 4;                      // cells a lane keeps in flight (ring depth, power of 2)
+constexpr int kRound = 4;                      // landing slots (cells) per warp
 
 struct DecodeParams {
     const int8_t *a;
@@ -65,14 +70,7 @@ struct DecodeParams {
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ uint4 ld_stream_v4(const uint32_t *p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-// per-thread asynchronous copies (activations, and scales that bulk copies cannot take)
+// per-thread asynchronous copies into shared memory
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
