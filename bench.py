@@ -36,7 +36,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode kernel on the
 # 4096x14336, M=1, group-64 GEMM (ncu capture summarised in profiles/decode_gate_m1_ncu.md);
 # the algorithmic bytes of that launch are 18,411,524.
-NCU_TRAFFIC_BYTES_GATE_M1 = 18_397_440
+NCU_TRAFFIC_BYTES_GATE_M1 = 18_378_752
 
 
 # --------------------------------------------------------------------- accounting
@@ -320,6 +320,70 @@ def kernel_probe(rep, M, shape_idx, reps=30):
                 distinct_weight_bytes=distinct, launches=reps * len(mats))
 
 
+def concat_probe(rep, reps=200):
+    """Extra row (not the headline): the same layer with q|k|v and gate|up concatenated along N,
+    i.e. 4 GEMMs + 4 a8_quantize per pass instead of 7 + 4.  Packed rows are independent, so the
+    concatenated matrix is the row-wise concatenation of the packed matrices.  Reported with the
+    headline's byte count so that the two are comparable."""
+    torch, b, cfg = rep.torch, rep.b, rep.cfg
+    names = [n for n, _, _ in rep.shapes]
+    if not all(n in names for n in ("q", "k", "v", "o", "gate", "up", "down")):
+        return None
+    ix = {n: names.index(n) for n in names}
+    fused = []
+    for mats in rep.copies:
+        def cat(group):
+            return (torch.cat([mats[ix[n]][0] for n in group], 0).contiguous(),
+                    torch.cat([mats[ix[n]][1] for n in group], 0).contiguous(), mats[ix[group[0]]][2])
+        fused.append({"qkv": cat(("q", "k", "v")), "o": mats[ix["o"]], "gateup": cat(("gate", "up")),
+                      "down": mats[ix["down"]]})
+    out = {}
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        for M in cfg["Ms"]:
+            bufs = rep.per_m[M]
+            ys = {k: torch.empty((M, v[0].shape[0]), dtype=torch.float32, device=v[0].device)
+                  for k, v in fused[0].items()}
+            ws = b.new_workspace(max(b.w2a8_workspace_bytes(M, v[0].shape[0], v[0].shape[1] * 16, v[2])
+                                     for v in fused[0].values()), device=ys["o"].device)
+            plan = (("attn_in", "qkv"), ("o_in", "o"), ("mlp_in", "gateup"), ("down_in", "down"))
+
+            def one_pass(c):
+                for inp, key in plan:
+                    b.a8_quantize(bufs["x"][inp], bufs["a"][inp], bufs["s"][inp])
+                    packed, s_w, g = fused[c][key]
+                    b.w2a8_gemm(bufs["a"][inp], bufs["s"][inp], packed, s_w, g, ws, ys[key])
+            for c in range(len(fused)):
+                one_pass(c)
+            torch.cuda.synchronize()
+            try:
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=stream):
+                    for c in range(len(fused)):
+                        one_pass(c)
+                run = gr.replay
+            except Exception:
+                def run():
+                    for c in range(len(fused)):
+                        one_pass(c)
+            for _ in range(3):
+                run()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = max(reps // len(fused), 3)
+            e0.record()
+            for _ in range(n):
+                run()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / (n * len(fused))
+            out[str(M)] = {"us_per_layer": ms * 1e3, "gbs": layer_bytes(cfg, M) / (ms * 1e-3) / 1e9}
+    torch.cuda.current_stream().wait_stream(stream)
+    return {"what": "q|k|v and gate|up concatenated along N: 4 GEMMs + 4 a8_quantize per layer pass; "
+                    "GB/s uses the byte count of the 7-GEMM layer", "per_m": out}
+
+
 def e2e_measure(rep, steps, warmup):
     """Same workload through w2a8_linear_host: pinned host activations in, host
     outputs back, copies inside the timed region."""
@@ -506,6 +570,7 @@ def run_ours(args):
         big = max(range(len(cfg["shapes"])), key=lambda i: cfg["shapes"][i][1] * cfg["shapes"][i][2])
         for M in cfg["Ms"]:
             probes.append(kernel_probe(rep, M, big))
+    concat = concat_probe(rep) if rank == 0 else None
     prefill = None
     if rank == 0 and not args.no_prefill:
         prefill = prefill_probe(device, peaks)
@@ -524,9 +589,13 @@ def run_ours(args):
     roofline = {"bound": "hbm", "achieved": dom["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": dom["gbs"] / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES_GATE_M1,
                 "peak_source": peaks["source"],
-                "kernel": "w2a8_decode_kernel<MT=1,SPP=1> on gate/up 4096x14336, M=1",
+                "kernel": "w2a8_decode_kernel<MT=1,SPP=1,TG=1,RING=4,ONE> on gate/up 4096x14336, M=1 "
+                          "(largest GEMV of the layer; the M=4 and M=16 instances are in roofline_by_m)",
                 "bytes_per_launch": dom["bytes_per_launch"], "us_per_launch": dom["us_per_launch"],
                 "frac_of_nominal_8TBs": dom["gbs"] / NOMINAL_HBM_GBS}
+    roofline_by_m = [{"M": pr["M"], "shape": pr["shape"], "achieved": pr["gbs"], "unit": "GB/s",
+                      "frac": pr["gbs"] / peaks["hbm_gbs"], "us_per_launch": pr["us_per_launch"]}
+                     for pr in probes]
     out = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_all / args.steps, "higher_is_better": True,
@@ -542,7 +611,8 @@ def run_ours(args):
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "clocks": clocks, "e2e": e2e,
         "gpu_launches": args.steps * len(cfg["Ms"]) * rep.kernels_per_pass,
-        "roofline": roofline, "cpu_baseline": cpu, "per_m": per_m, "kernel_probes": probes,
+        "roofline": roofline, "roofline_by_m": roofline_by_m, "cpu_baseline": cpu, "per_m": per_m,
+        "kernel_probes": probes, "concatenated_qkv_gateup": concat,
         "prefill": prefill,
     }
     print(json.dumps(out))
