@@ -500,20 +500,17 @@ extern "C" int w2a8_debug_set_trace(void *buffer, const float *y0, unsigned long
 // ---- host side -----------------------------------------------------------------
 int env_int(const char *name, int dflt);
 
-static inline int decode_mt(int M) { return M > 32 ? 4 : (M + 7) / 8; }
-
 struct DecodePlan {
     int mt, tg, ring, chunks, blocks_per_chunk, slabs, groups, s_vec, cluster;
     size_t smem;
 };
 
-// Launch plan.  Few tokens (one 8-token slab): one tile per CTA, its four warps take
-// interleaved blocks of K (shortest serial work per warp).  More tokens: two tiles per
-// CTA, two K-lanes each.  K-chunks are added when a warp would otherwise have more cells
-// than landing slots, or when the grid would leave most SMs idle.
-static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
+// Launch plan for slabs of 8 * mt tokens.  One tile per CTA, its four warps take interleaved
+// blocks of K (shortest serial work per warp).  K-chunks are added when a warp would
+// otherwise have more cells than landing slots, or when the grid would leave most SMs idle.
+static DecodePlan decode_plan_mt(int M, int N, int K, const ShapeInfo &si, int mt) {
     DecodePlan pl;
-    pl.mt = decode_mt(M);
+    pl.mt = mt;
     pl.slabs = (M + 8 * pl.mt - 1) / (8 * pl.mt);
     const int ntiles = N / 16;
     const int forced_tg = env_int("W2A8_TG", 0);
@@ -547,9 +544,24 @@ static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
     // rank 0 receives one partial output per chunk and element of the CTA
     pl.cluster = pl.chunks > 1 && pl.chunks <= 8 && env_int("W2A8_CLUSTER", 1) != 0;
     if (pl.cluster) pl.smem += (size_t)pl.chunks * pl.tg * pl.mt * 128 * sizeof(float);
-    (void)M;
     (void)K;
     return pl;
+}
+
+// Tokens per slab.  Up to 8 tokens: one slab.  More: slabs of 8 tokens (the weights are then
+// streamed once per slab, the later slabs from L2) as long as the whole grid is resident at
+// once (8 CTAs per SM) -- measured faster on the small matrices of a layer (k/v, q/o), whose
+// grids are far from filling the GPU with wider slabs; otherwise the widest slab that covers M,
+// up to 32 tokens.  W2A8_MT forces a width.
+static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
+    const int forced = env_int("W2A8_MT", 0);
+    if (forced >= 1 && forced <= 4) return decode_plan_mt(M, N, K, si, forced);
+    const int widest = M > 32 ? 4 : (M + 7) / 8;
+    if (widest == 1) return decode_plan_mt(M, N, K, si, 1);
+    constexpr long long kResidentCtas = 148 * 8;
+    const DecodePlan narrow = decode_plan_mt(M, N, K, si, 1);
+    if ((long long)narrow.groups * narrow.chunks * narrow.slabs <= kResidentCtas) return narrow;
+    return decode_plan_mt(M, N, K, si, widest);
 }
 
 constexpr size_t kStatusBytes = 256;   // workspace header: status word
@@ -559,7 +571,7 @@ size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si) {
     size_t counters = ((size_t)4 * (N / 16) * pl.slabs + 255) / 256 * 256;   // >= any tile grouping
     // with an environment override in force, size for the finest split
     const bool overridden = env_int("W2A8_CHUNKS", 0) > 0 || env_int("W2A8_TG", 0) > 0 ||
-                            env_int("W2A8_RING", 0) > 0;
+                            env_int("W2A8_RING", 0) > 0 || env_int("W2A8_MT", 0) > 0;
     const int chunks = overridden ? si.blocks : pl.chunks;
     size_t part = (size_t)(chunks > 1 ? chunks : 0) * M * N * sizeof(float);
     return kStatusBytes + counters + part;

@@ -179,6 +179,21 @@ def test_forced_chunking(gpu, oracle, chunks, tg, M, group, monkeypatch):
     assert ok, f"worst error / bound = {worst}"
 
 
+@pytest.mark.parametrize("switch", [("W2A8_CLUSTER", "0"), ("W2A8_MT", "1"), ("W2A8_MT", "3"),
+                                    ("W2A8_RING", "8"), ("W2A8_MIN_WARPS", "100000")])
+@pytest.mark.parametrize("M,N,K,group", [(20, 80, 14336 + 256 * 3, 64), (1, 4096, 4096, 64), (9, 1024, 4096, 128)])
+def test_plan_switches(gpu, oracle, switch, M, N, K, group, monkeypatch):
+    """The alternatives of the decode launch plan (split-K through the workspace instead of a
+    cluster, slab widths, deeper landing slots, finer split-K) give the same exact sums."""
+    torch, b = gpu
+    monkeypatch.setenv(*switch)
+    codes, s_w, bits, g = _problem(7 + M, M, N, K, group)
+    a, s_a, y, P = _run_gpu(torch, b, codes, s_w, bits, g)
+    assert np.array_equal(P, oracle.partials(a, codes, g))
+    ok, worst = _row_err_ok(y, oracle.gemm(a, s_a, codes, s_w, g))
+    assert ok, f"worst error / bound = {worst}"
+
+
 def test_extreme_magnitudes_no_overflow(gpu, oracle):
     torch, b = gpu
     M, N, K = 2, 16, 28672
