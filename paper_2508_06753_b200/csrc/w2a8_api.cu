@@ -321,6 +321,20 @@ size_t w2a8_linear_host_workspace_bytes(int M, int N, int K, int group) {
            up256((size_t)M * N * 4);
 }
 
+constexpr int kDecodeMaxZeroCopyTokens = 32;
+
+// Device-side address of a page-locked, mapped host allocation; nullptr for pageable memory
+// (or anything else the device cannot address directly).
+static void *mapped_device_pointer(const void *host) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
+        cudaGetLastError();   // pageable memory is reported as an error by older drivers
+        return nullptr;
+    }
+    if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) return nullptr;
+    return attr.devicePointer;
+}
+
 int w2a8_linear_host(const void *x_host, int M, int K, const uint32_t *packed,
                      const float *w_scale, int N, int group, float *y_host, void *workspace,
                      size_t workspace_bytes, void *stream) {
@@ -336,6 +350,18 @@ int w2a8_linear_host(const void *x_host, int M, int K, const uint32_t *packed,
     int8_t *a = (int8_t *)p;          p += up256((size_t)M * K);
     float *a_scale = (float *)p;      p += up256((size_t)M * 4);
     float *y_dev = (float *)p;
+    // Few tokens: the transfers are a few KB, and a copy-engine operation costs more in launch
+    // latency than it moves.  If both host buffers are page-locked and mapped (so the device can
+    // address them), the quantiser reads x over the bus itself and the GEMM stores y straight to
+    // the host buffer.  Otherwise, and for many tokens, staged copies.
+    static const int zero_copy_max = env_int("W2A8_ZEROCOPY_MAX", kDecodeMaxZeroCopyTokens);
+    const void *x_map = (M <= zero_copy_max) ? mapped_device_pointer(x_host) : nullptr;
+    void *y_map = (M <= zero_copy_max) ? mapped_device_pointer(y_host) : nullptr;
+    if (x_map && y_map && aligned16(x_map) && aligned16(y_map)) {
+        if (int s = a8_quantize(x_map, M, K, a, a_scale, stream)) return s;
+        return w2a8_gemm(a, a_scale, packed, w_scale, reinterpret_cast<float *>(y_map), M, N, K, group, ws,
+                         gemm_ws, stream);
+    }
     if (cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return W2A8_ERR_CUDA;
     if (int s = a8_quantize(x_dev, M, K, a, a_scale, stream)) return s;

@@ -227,14 +227,19 @@ def test_zero_token_row_and_zero_weights(gpu, oracle):
     assert ok, worst
 
 
-def test_linear_host_end_to_end(gpu, oracle):
+@pytest.mark.parametrize("M,pinned", [(4, True), (4, False), (1, True), (40, True)])
+def test_linear_host_end_to_end(gpu, oracle, M, pinned):
+    """Host buffers in, host buffers out: page-locked buffers with few tokens are read and
+    written by the kernels directly, everything else goes through staged copies."""
     torch, b = gpu
-    M, N, K, g = 4, 1024, 4096, 64
+    N, K, g = 1024, 4096, 64
     codes, s_w, bits, g = _problem(77, M, N, K, g)
     packed = b.w2_pack(_dev(torch, codes))
     s_w_d = _dev(torch, s_w)
-    x_host = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).pin_memory()
-    y_host = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    x_host = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+    y_host = torch.empty((M, N), dtype=torch.float32)
+    if pinned:
+        x_host, y_host = x_host.pin_memory(), y_host.pin_memory()
     ws = b.new_workspace(b.w2a8_linear_host_workspace_bytes(M, N, K, g))
     for _ in range(2):
         y_host.zero_()
