@@ -39,6 +39,7 @@ constexpr int kPfHalfBytes = 128 * 128;  // one [128 rows][128 B] swizzled sub-t
 constexpr int kPfStageBytes = 4 * kPfHalfBytes;   // A: 2 halves, B: 2 halves
 constexpr int kPfAccBufs = 4;             // accumulator buffers in tensor memory (groups in flight)
 constexpr int kPfTmemCols = kPfAccBufs * kPfBN;   // 512 columns: all of tensor memory
+constexpr int kPfUnits = kPfAccBufs / 2;  // hand-off unit between MMA and drain: two groups (two buffers)
 constexpr unsigned kPfWaitPolls = 1u << 20;   // bound of every barrier wait (polls)
 
 struct PrefillParams {
@@ -186,8 +187,8 @@ template <bool PARTIALS>
 __global__ void __launch_bounds__(kPfThreads, 1)
 w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillParams p) {
     extern __shared__ unsigned char pf_smem_raw[];
-    __shared__ __align__(8) unsigned long long bar_full_a[kPfStages], bar_full_b[kPfStages], bar_empty[kPfStages];
-    __shared__ __align__(8) unsigned long long bar_acc_full[kPfAccBufs], bar_acc_empty[kPfAccBufs];
+    __shared__ __align__(8) unsigned long long bar_full[kPfStages], bar_empty[kPfStages];
+    __shared__ __align__(8) unsigned long long bar_acc_full[kPfUnits], bar_acc_empty[kPfUnits];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     __shared__ float a_scale_s[kPfBN];
@@ -205,11 +206,11 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         for (int s = 0; s < kPfStages; ++s) {
-            pf_mbar_init(pf_smem_u32(&bar_full_a[s]), kPfUnpackWarps);   // one arrive per unpack warp
-            pf_mbar_init(pf_smem_u32(&bar_full_b[s]), 1);     // TMA producer + transaction bytes
+            // one arrive per unpack warp + the TMA producer's arrive with its transaction bytes
+            pf_mbar_init(pf_smem_u32(&bar_full[s]), kPfUnpackWarps + 1);
             pf_mbar_init(pf_smem_u32(&bar_empty[s]), 2);      // one tcgen05.commit per MMA-issuing thread
         }
-        for (int b = 0; b < kPfAccBufs; ++b) {
+        for (int b = 0; b < kPfUnits; ++b) {
             pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);   // tcgen05.commit
             pf_mbar_init(pf_smem_u32(&bar_acc_empty[b]), 8);  // one arrive per drain warp
         }
@@ -239,28 +240,28 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             constexpr uint32_t idesc = pf_instr_desc(kPfBM, kPfBN);
             const uint64_t a_desc0 = pf_smem_desc(smem_base);
             const uint64_t b_desc0 = pf_smem_desc(smem_base + 2 * kPfHalfBytes);
+            const int ngroups_i = (p.K / 64) / dps;
             int pos = 0;                    // 64-k slices already issued in the current group
-            int group_idx = 0;              // scale groups committed so far
-            int buf = 0;                    // accumulator buffer of the current group
-            uint32_t empty_parity = 0;      // bit b: parity to wait for on bar_acc_empty[b]
+            int group_idx = 0;              // scale groups completed so far; group g uses buffer g % 4
             int s = 0;
             uint32_t full_parity = 0;
             bool ok = true;
             for (int it = 0; it < nstages_total && ok; ++it) {
-                ok = pf_wait(pf_smem_u32(&bar_full_a[s]), full_parity, abort_flag) &&
-                     pf_wait(pf_smem_u32(&bar_full_b[s]), full_parity, abort_flag);
+                ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
                 if (!ok) break;
                 if (mma_id == 1) PF_TRACE(1, it, 0);
                 pf_tc_fence_after();
                 const uint64_t stage_off = (uint64_t)((uint32_t)(s * kPfStageBytes) >> 4);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const bool mine = (group_idx & 1) == mma_id;
-                    if (mine && pos == 0 && group_idx >= kPfAccBufs) {
-                        // the drain warps must have emptied this buffer's previous group
-                        ok = pf_wait(pf_smem_u32(&bar_acc_empty[buf]), (empty_parity >> buf) & 1u, abort_flag);
+                    // hand-off unit u = two consecutive groups = accumulator buffers 2 (u % 2), +1
+                    const int u = group_idx >> 1, slot = u & 1;
+                    const bool mine = slot == mma_id;
+                    const int buf = group_idx & (kPfAccBufs - 1);
+                    if (mine && pos == 0 && (group_idx & 1) == 0 && u >= kPfUnits) {
+                        // the drain warps must have emptied this unit's previous groups
+                        ok = pf_wait(pf_smem_u32(&bar_acc_empty[slot]), ((u >> 1) - 1) & 1, abort_flag);
                         if (!ok) break;
-                        empty_parity ^= 1u << buf;
                         pf_tc_fence_after();
                     }
                     if (mine) {
@@ -273,10 +274,10 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         }
                     }
                     if (++pos == dps) {
-                        if (mine) pf_mma_commit(pf_smem_u32(&bar_acc_full[buf]));
                         pos = 0;
+                        const bool unit_done = (group_idx & 1) == 1 || group_idx == ngroups_i - 1;
+                        if (mine && unit_done) pf_mma_commit(pf_smem_u32(&bar_acc_full[slot]));
                         ++group_idx;
-                        buf = (buf + 1) & (kPfAccBufs - 1);
                     }
                 }
                 pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
@@ -308,7 +309,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             if (round > 0 && !pf_wait_warp(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
             if (warp == 2 && lane == 0) {
                 // this lane is also the TMA producer: activations, 128 tokens x 256 k per stage
-                const uint32_t bar = pf_smem_u32(&bar_full_b[s]);
+                const uint32_t bar = pf_smem_u32(&bar_full[s]);
                 const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
                 pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
                 pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
@@ -332,7 +333,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             }
             pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
             __syncwarp();
-            if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full_a[s]));
+            if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full[s]));
             if (warp == 2 && lane == 0) PF_TRACE(2, it, 1);
         }
     } else {
@@ -385,16 +386,21 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     for (int j = 0; j < 32; j += 2) pf_fma2(acc[j], acc[j + 1], (float)v0[j], (float)v0[j + 1], sc);
                 }
                 pf_tmem_ld_wait();                     // second half is in v1
-                // all of this warp's share of the buffer has been read: hand it back
-                pf_tc_fence_before();
-                __syncwarp();
-                if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[buf]));
+                if ((gi & 1) == 1 || gi == ngroups - 1) {
+                    // all of this warp's share of the unit (two groups) has been read: hand it back
+                    pf_tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[(gi >> 1) & 1]));
+                }
                 if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, gi, 1);
                 if (gi + 1 < ngroups) {                // request the first half of the next group
                     const int nbuf = (u + 1) % kPfAccBufs;
-                    ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[nbuf]), ((gi + 1) / kPfAccBufs) & 1, abort_flag);
-                    if (!ok) break;
-                    pf_tc_fence_after();
+                    if (((gi + 1) & 1) == 0) {         // it opens a new unit: wait for its MMAs
+                        const int nu = (gi + 1) >> 1;
+                        ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[nu & 1]), (nu >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        pf_tc_fence_after();
+                    }
                     pf_tmem_ld32(tlane + nbuf * kPfBN, v0);
                 }
                 if (PARTIALS) {
