@@ -167,7 +167,7 @@ __host__ __device__ constexpr uint32_t pf_instr_desc(int m, int n) {
 #ifdef W2A8_TRACE
 __device__ unsigned long long *g_pf_trace = nullptr;   // 5 roles x 4096 slots
 __device__ __forceinline__ void pf_trace(int role, int idx, int point) {
-    if (g_pf_trace && blockIdx.x == 0 && blockIdx.y == 0 && idx < 1024) {
+    if (g_pf_trace && blockIdx.x == 0 && idx < 1024) {
         unsigned long long v;
         if (role >= 3) v = (unsigned long long)clock64();      // SM cycles for the drain and MMA-group roles
         else asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(v));
@@ -191,14 +191,19 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     __shared__ __align__(8) unsigned long long bar_acc_full[kPfUnits], bar_acc_empty[kPfUnits];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
-    __shared__ float a_scale_s[kPfBN];
     volatile int *abort_flag = &abort_flag_s;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * kPfBM;      // first channel of the tile
-    const int m0 = blockIdx.y * kPfBN;      // first token of the tile
-    const int nstages_total = p.K / kPfBK;
+    const int nstages = p.K / kPfBK;        // stages per tile
     const int dps = p.slices_per_group;     // 64-k slices between two drains
+    const int ngroups = (p.K / 64) / dps;   // scale groups per tile
+    const int units_per_tile = (ngroups + 1) / 2;
+    // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; consecutive tiles share the
+    // channel tile and differ in the token tile, so neighbouring CTAs re-use weights from L2.
+    // Stage slots and accumulator units are numbered across tiles (the pipeline does not drain
+    // between tiles: producers run ahead into the next tile while the drain warps store y).
+    const int tiles_m = (p.M + kPfBN - 1) / kPfBN;
+    const int ntiles = (p.N / kPfBM) * tiles_m;
     // stage buffers, 1024-byte aligned (swizzle atom = 8 rows x 128 B)
     const uint32_t smem_base = (pf_smem_u32(pf_smem_raw) + 1023u) & ~1023u;
     unsigned char *smem_gen = pf_smem_raw + (smem_base - pf_smem_u32(pf_smem_raw));
@@ -218,10 +223,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         pf_fence_proxy_async();
     }
     if (warp == 1) pf_tmem_alloc(pf_smem_u32(&tmem_base_slot), kPfTmemCols);
-    if (threadIdx.x < kPfBN) {
-        const int m = m0 + threadIdx.x;
-        a_scale_s[threadIdx.x] = (!PARTIALS && m < p.M) ? p.a_scale[m] * (1.0f / kCodeGain) : 0.f;
-    }
     pf_tc_fence_before();
     __syncthreads();
     pf_tc_fence_after();
@@ -230,66 +231,71 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     if (warp < 2) {
         // ===== MMA issuers (one thread in each of warps 0 and 1) =========================
         // Issuing is scalar work of a single thread and costs several hundred cycles per
-        // group, so two threads share it: thread `mma_id` takes the scale groups with
-        // group index = mma_id (mod 2), i.e. accumulator buffers mma_id and mma_id + 2.
-        // Groups are independent (different buffers), so no order between the two
-        // threads is needed.  Descriptors are a base plus compile-time offsets, group
-        // bookkeeping uses counters (no division), the four slices of a stage are unrolled.
+        // group, so two threads share it.  The hand-off unit between MMA and drain is two
+        // consecutive scale groups (two accumulator buffers, one barrier pair): a barrier
+        // round trip costs a few hundred cycles, as much as the MMAs of a 64-k group, so
+        // halving their number matters.  Thread `mma_id` owns the units with that parity.
+        // Descriptors are a base plus compile-time offsets, bookkeeping uses counters (no
+        // division), the four slices of a stage are unrolled.
         if (lane == 0) {
             const int mma_id = warp;
             constexpr uint32_t idesc = pf_instr_desc(kPfBM, kPfBN);
             const uint64_t a_desc0 = pf_smem_desc(smem_base);
             const uint64_t b_desc0 = pf_smem_desc(smem_base + 2 * kPfHalfBytes);
-            const int ngroups_i = (p.K / 64) / dps;
-            int pos = 0;                    // 64-k slices already issued in the current group
-            int group_idx = 0;              // scale groups completed so far; group g uses buffer g % 4
             int s = 0;
             uint32_t full_parity = 0;
+            int unit0 = 0;                  // units of the tiles before this one
+            int trace_it = 0;
             bool ok = true;
-            for (int it = 0; it < nstages_total && ok; ++it) {
-                ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
-                if (!ok) break;
-                if (mma_id == 1) PF_TRACE(1, it, 0);
-                pf_tc_fence_after();
-                const uint64_t stage_off = (uint64_t)((uint32_t)(s * kPfStageBytes) >> 4);
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
+                int pos = 0;                // 64-k slices already issued in the current group
+                int group_idx = 0;          // scale groups of this tile completed so far
+                for (int it = 0; it < nstages && ok; ++it, ++trace_it) {
+                    ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
+                    if (!ok) break;
+                    if (mma_id == 1) PF_TRACE(1, trace_it, 0);
+                    pf_tc_fence_after();
+                    const uint64_t stage_off = (uint64_t)((uint32_t)(s * kPfStageBytes) >> 4);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    // hand-off unit u = two consecutive groups = accumulator buffers 2 (u % 2), +1
-                    const int u = group_idx >> 1, slot = u & 1;
-                    const bool mine = slot == mma_id;
-                    const int buf = group_idx & (kPfAccBufs - 1);
-                    if (mine && pos == 0 && (group_idx & 1) == 0 && u >= kPfUnits) {
-                        // the drain warps must have emptied this unit's previous groups
-                        ok = pf_wait(pf_smem_u32(&bar_acc_empty[slot]), ((u >> 1) - 1) & 1, abort_flag);
-                        if (!ok) break;
-                        pf_tc_fence_after();
-                    }
-                    if (mine) {
+                    for (int q = 0; q < 4; ++q) {
+                        // unit u: accumulator buffers 2 (u % 2) and 2 (u % 2) + 1
+                        const int u = unit0 + (group_idx >> 1), slot = u & 1;
+                        const bool mine = slot == mma_id;
+                        const int buf = 2 * slot + (group_idx & 1);
+                        if (mine && pos == 0 && (group_idx & 1) == 0 && u >= kPfUnits) {
+                            // the drain warps must have emptied this unit's previous groups
+                            ok = pf_wait(pf_smem_u32(&bar_acc_empty[slot]), ((u >> 1) - 1) & 1, abort_flag);
+                            if (!ok) break;
+                            pf_tc_fence_after();
+                        }
+                        if (mine) {
 #pragma unroll
-                        for (int ks = 0; ks < 2; ++ks) {
-                            constexpr int kHalf16 = kPfHalfBytes >> 4;
-                            const uint64_t off = stage_off + (uint64_t)((q >> 1) * kHalf16 + ((q & 1) * 2 + ks) * 2);
-                            pf_mma_i8(tmem_base + buf * kPfBN, a_desc0 + off, b_desc0 + off, idesc,
-                                      (pos == 0 && ks == 0) ? 0u : 1u);
+                            for (int ks = 0; ks < 2; ++ks) {
+                                constexpr int kHalf16 = kPfHalfBytes >> 4;
+                                const uint64_t off = stage_off + (uint64_t)((q >> 1) * kHalf16 + ((q & 1) * 2 + ks) * 2);
+                                pf_mma_i8(tmem_base + buf * kPfBN, a_desc0 + off, b_desc0 + off, idesc,
+                                          (pos == 0 && ks == 0) ? 0u : 1u);
+                            }
+                        }
+                        if (++pos == dps) {
+                            pos = 0;
+                            const bool unit_done = (group_idx & 1) == 1 || group_idx == ngroups - 1;
+                            if (mine && unit_done) pf_mma_commit(pf_smem_u32(&bar_acc_full[slot]));
+                            ++group_idx;
                         }
                     }
-                    if (++pos == dps) {
-                        pos = 0;
-                        const bool unit_done = (group_idx & 1) == 1 || group_idx == ngroups_i - 1;
-                        if (mine && unit_done) pf_mma_commit(pf_smem_u32(&bar_acc_full[slot]));
-                        ++group_idx;
-                    }
+                    pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
+                    if (mma_id == 1) PF_TRACE(1, trace_it, 1);
+                    if (++s == kPfStages) { s = 0; full_parity ^= 1u; }
                 }
-                pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
-                if (mma_id == 1) PF_TRACE(1, it, 1);
-                if (++s == kPfStages) { s = 0; full_parity ^= 1u; }
             }
         }
     } else if (warp < 2 + kPfUnpackWarps) {
         // ===== unpack warps: packed words -> int8 lanes, K-major, 128-byte swizzle =====
         constexpr int kUnits = 512 / (32 * kPfUnpackWarps);   // 16-byte units per thread and stage
         const int ut = (warp - 2) * 32 + lane;
-        auto request = [&](uint4 (&w)[kUnits], int it) {
+        auto request = [&](uint4 (&w)[kUnits], int tile, int it) {
+            const int n0 = (tile / tiles_m) * kPfBM;
 #pragma unroll
             for (int i = 0; i < kUnits; ++i) {
                 const int u = ut + 32 * kPfUnpackWarps * i;   // unit: row = u / 4, quarter t = u % 4
@@ -299,130 +305,145 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             }
         };
         uint4 w_nxt[kUnits];
-        request(w_nxt, 0);
-        for (int it = 0; it < nstages_total; ++it) {
-            const int s = it % kPfStages, round = it / kPfStages;
-            uint4 w[kUnits];
+        if ((int)blockIdx.x < ntiles) request(w_nxt, blockIdx.x, 0);
+        int s = 0, round = 0, trace_it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+            const int m0 = (tile % tiles_m) * kPfBN;
+            for (int it = 0; it < nstages; ++it, ++trace_it) {
+                uint4 w[kUnits];
 #pragma unroll
-            for (int i = 0; i < kUnits; ++i) w[i] = w_nxt[i];
-            if (it + 1 < nstages_total) request(w_nxt, it + 1);   // next stage's words in flight
-            if (round > 0 && !pf_wait_warp(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
-            if (warp == 2 && lane == 0) {
-                // this lane is also the TMA producer: activations, 128 tokens x 256 k per stage
-                const uint32_t bar = pf_smem_u32(&bar_full[s]);
-                const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
-                pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
-                pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
-                pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
-                PF_TRACE(2, it, 0);
-            }
-            unsigned char *a_stage = smem_gen + s * kPfStageBytes;
-#pragma unroll
-            for (int i = 0; i < kUnits; ++i) {
-                const int u = ut + 32 * kPfUnpackWarps * i;
-                const int r = u >> 2, t = u & 3;
-                const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
-#pragma unroll
-                for (int sl = 0; sl < 4; ++sl) {    // slice sl: k = 64 sl + 16 t .. + 15 of this block
-                    uint4 v;
-                    v.x = lane_codes(ws[sl], 0); v.y = lane_codes(ws[sl], 1);
-                    v.z = lane_codes(ws[sl], 2); v.w = lane_codes(ws[sl], 3);
-                    const int chunk = (4 * (sl & 1) + t) ^ (r & 7);
-                    *reinterpret_cast<uint4 *>(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16) = v;
+                for (int i = 0; i < kUnits; ++i) w[i] = w_nxt[i];
+                // next stage's words in flight (possibly the first stage of the next tile)
+                if (it + 1 < nstages) request(w_nxt, tile, it + 1);
+                else if (tile + (int)gridDim.x < ntiles) request(w_nxt, tile + gridDim.x, 0);
+                if (round > 0 && !pf_wait_warp(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) {
+                    ok = false;
+                    break;
                 }
+                if (warp == 2 && lane == 0) {
+                    // this lane is also the TMA producer: activations, 128 tokens x 256 k per stage
+                    const uint32_t bar = pf_smem_u32(&bar_full[s]);
+                    const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
+                    pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
+                    pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
+                    pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
+                    PF_TRACE(2, trace_it, 0);
+                }
+                unsigned char *a_stage = smem_gen + s * kPfStageBytes;
+#pragma unroll
+                for (int i = 0; i < kUnits; ++i) {
+                    const int u = ut + 32 * kPfUnpackWarps * i;
+                    const int r = u >> 2, t = u & 3;
+                    const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+#pragma unroll
+                    for (int sl = 0; sl < 4; ++sl) {    // slice sl: k = 64 sl + 16 t .. + 15 of this block
+                        uint4 v;
+                        v.x = lane_codes(ws[sl], 0); v.y = lane_codes(ws[sl], 1);
+                        v.z = lane_codes(ws[sl], 2); v.w = lane_codes(ws[sl], 3);
+                        const int chunk = (4 * (sl & 1) + t) ^ (r & 7);
+                        *reinterpret_cast<uint4 *>(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16) = v;
+                    }
+                }
+                pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
+                __syncwarp();
+                if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full[s]));
+                if (warp == 2 && lane == 0) PF_TRACE(2, trace_it, 1);
+                if (++s == kPfStages) { s = 0; ++round; }
             }
-            pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
-            __syncwarp();
-            if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full[s]));
-            if (warp == 2 && lane == 0) PF_TRACE(2, it, 1);
         }
     } else {
         // ===== drain warps: TMEM -> registers, fp32 accumulate with the group scale ======
         const int q4 = warp & 3;                    // TMEM lane quarter this warp may access
         const int col0 = ((warp - 2 - kPfUnpackWarps) >> 2) * kPfDrainCols;   // first token column of this warp
         const int ch = q4 * 32 + lane;              // channel inside the tile = TMEM lane
-        const int n = n0 + ch;
-        float acc[kPfDrainCols];
-#pragma unroll
-        for (int j = 0; j < kPfDrainCols; ++j) acc[j] = 0.f;
-        const int ngroups = (p.K / 64) / dps;
-        // Scales are fetched eight groups ahead (a drain takes a few hundred cycles, a
-        // global load several hundred): a ring of eight, refilled once per eight groups.
-        const float *sc_row = PARTIALS ? nullptr : p.w_scale + (size_t)n * p.G;
-        float sc_nxt[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) sc_nxt[u] = (!PARTIALS && u < ngroups) ? __ldg(sc_row + u) : 0.f;
-        bool ok = true;
-        // Software pipeline over 32-column halves: while one half is converted and
-        // accumulated, the next half (possibly of the next group) is on its way from TMEM.
-        int v0[32], v1[32];                         // first / second half of the current group
         const uint32_t tlane = tmem_base + ((uint32_t)(q4 * 32) << 16) + col0;
-        ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[0]), 0, abort_flag);
-        if (ok) { pf_tc_fence_after(); pf_tmem_ld32(tlane, v0); }
-        for (int g0 = 0; g0 < ngroups && ok; g0 += 8) {
-            float sc_cur[8];
+        bool ok = true;
+        int unit0 = 0;                              // units of the tiles before this one
+        int trace_g = 0;
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
+            const int n = (tile / tiles_m) * kPfBM + ch;
+            const int m0 = (tile % tiles_m) * kPfBN;
+            float acc[kPfDrainCols];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                sc_cur[u] = sc_nxt[u];
-                sc_nxt[u] = (!PARTIALS && g0 + 8 + u < ngroups) ? __ldg(sc_row + g0 + 8 + u) : 0.f;
+            for (int j = 0; j < kPfDrainCols; ++j) acc[j] = 0.f;
+            // Scales are fetched eight groups ahead (a drain takes a few hundred cycles, a
+            // global load several hundred): a ring of eight, refilled once per eight groups.
+            const float *sc_row = PARTIALS ? nullptr : p.w_scale + (size_t)n * p.G;
+            float sc_nxt[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) sc_nxt[u] = (!PARTIALS && u < ngroups) ? __ldg(sc_row + u) : 0.f;
+            // Software pipeline over 32-column halves: while one half is converted and
+            // accumulated, the next half (possibly of the next group) is on its way from TMEM.
+            int v0[32], v1[32];                         // first / second half of the current group
+            ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[unit0 & 1]), (unit0 >> 1) & 1, abort_flag);
+            if (ok) { pf_tc_fence_after(); pf_tmem_ld32(tlane + (2 * (unit0 & 1)) * kPfBN, v0); }
+            for (int g0 = 0; g0 < ngroups && ok; g0 += 8) {
+                float sc_cur[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    sc_cur[u] = sc_nxt[u];
+                    sc_nxt[u] = (!PARTIALS && g0 + 8 + u < ngroups) ? __ldg(sc_row + g0 + 8 + u) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int gi = g0 + u;
+                    if (gi >= ngroups || !ok) break;
+                    const int unit = unit0 + (gi >> 1);            // group gi lives in buffer 2 (unit % 2) + gi % 2
+                    const int buf = 2 * (unit & 1) + (gi & 1);
+                    const float sc = sc_cur[u];
+                    pf_tmem_ld_wait();                     // first half of group gi is in v0
+                    if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, trace_g + gi, 0);
+                    pf_tmem_ld32(tlane + buf * kPfBN + 32, v1);
+                    if (PARTIALS) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int m = m0 + col0 + j;
+                            if (m < p.M) p.partials[((size_t)m * p.N + n) * p.G + gi] = v0[j] >> 6;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) pf_fma2(acc[j], acc[j + 1], (float)v0[j], (float)v0[j + 1], sc);
+                    }
+                    pf_tmem_ld_wait();                     // second half is in v1
+                    if ((gi & 1) == 1 || gi == ngroups - 1) {
+                        // all of this warp's share of the unit (two groups) has been read: hand it back
+                        pf_tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[unit & 1]));
+                    }
+                    if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, trace_g + gi, 1);
+                    if (gi + 1 < ngroups) {                // request the first half of the next group
+                        const int nunit = unit0 + ((gi + 1) >> 1);
+                        if (((gi + 1) & 1) == 0) {         // it opens a new unit: wait for its MMAs
+                            ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[nunit & 1]), (nunit >> 1) & 1, abort_flag);
+                            if (!ok) break;
+                            pf_tc_fence_after();
+                        }
+                        pf_tmem_ld32(tlane + (2 * (nunit & 1) + ((gi + 1) & 1)) * kPfBN, v0);
+                    }
+                    if (PARTIALS) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int m = m0 + col0 + 32 + j;
+                            if (m < p.M) p.partials[((size_t)m * p.N + n) * p.G + gi] = v1[j] >> 6;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2)
+                            pf_fma2(acc[32 + j], acc[32 + j + 1], (float)v1[j], (float)v1[j + 1], sc);
+                    }
+                    if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, trace_g + gi, 2);
+                }
             }
+            pf_tmem_ld_wait();
+            trace_g += ngroups;
+            if (!PARTIALS && ok) {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int gi = g0 + u;
-                if (gi >= ngroups || !ok) break;
-                const int buf = u % kPfAccBufs;        // group g lives in buffer g % kPfAccBufs (g0 is a multiple of 8)
-                const float sc = sc_cur[u];
-                pf_tmem_ld_wait();                     // first half of group gi is in v0
-                if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, gi, 0);
-                pf_tmem_ld32(tlane + buf * kPfBN + 32, v1);
-                if (PARTIALS) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int m = m0 + col0 + j;
-                        if (m < p.M) p.partials[((size_t)m * p.N + n) * p.G + gi] = v0[j] >> 6;
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) pf_fma2(acc[j], acc[j + 1], (float)v0[j], (float)v0[j + 1], sc);
+                for (int j = 0; j < kPfDrainCols; ++j) {
+                    const int m = m0 + col0 + j;
+                    if (m < p.M) p.y[(size_t)m * p.N + n] = acc[j] * (__ldg(p.a_scale + m) * (1.0f / kCodeGain));
                 }
-                pf_tmem_ld_wait();                     // second half is in v1
-                if ((gi & 1) == 1 || gi == ngroups - 1) {
-                    // all of this warp's share of the unit (two groups) has been read: hand it back
-                    pf_tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[(gi >> 1) & 1]));
-                }
-                if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, gi, 1);
-                if (gi + 1 < ngroups) {                // request the first half of the next group
-                    const int nbuf = (u + 1) % kPfAccBufs;
-                    if (((gi + 1) & 1) == 0) {         // it opens a new unit: wait for its MMAs
-                        const int nu = (gi + 1) >> 1;
-                        ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[nu & 1]), (nu >> 1) & 1, abort_flag);
-                        if (!ok) break;
-                        pf_tc_fence_after();
-                    }
-                    pf_tmem_ld32(tlane + nbuf * kPfBN, v0);
-                }
-                if (PARTIALS) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int m = m0 + col0 + 32 + j;
-                        if (m < p.M) p.partials[((size_t)m * p.N + n) * p.G + gi] = v1[j] >> 6;
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2)
-                        pf_fma2(acc[32 + j], acc[32 + j + 1], (float)v1[j], (float)v1[j + 1], sc);
-                }
-                if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, gi, 2);
-            }
-        }
-        pf_tmem_ld_wait();
-        if (!PARTIALS && ok) {
-#pragma unroll
-            for (int j = 0; j < kPfDrainCols; ++j) {
-                const int m = m0 + col0 + j;
-                if (m < p.M) p.y[(size_t)m * p.N + n] = acc[j] * a_scale_s[col0 + j];
             }
         }
     }
@@ -485,7 +506,15 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
     p.words_per_row = K / 16;
     p.slices_per_group = group / 64;
     const size_t smem = (size_t)kPfStages * kPfStageBytes + 1024;
-    dim3 grid(N / kPfBM, (M + kPfBN - 1) / kPfBN);
+    static int sm_count = 0;
+    if (sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
+            sm_count = 148;
+    }
+    const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
+    dim3 grid((unsigned)(tiles < sm_count ? tiles : sm_count));   // persistent CTAs, one per SM
     static bool configured[2] = {false, false};
     cudaError_t e;
     if (partials) {
