@@ -6,7 +6,7 @@
 // up-convert of Sec. II-C done into shared memory because the tensor core has
 // no 2-bit operand type.
 //
-// One CTA (12 warps) computes a 128-channel x 128-token tile of y.
+// Persistent CTAs (12 warps, one CTA per SM) walk 128-channel x 128-token tiles of y.
 //   A operand (UMMA M = 128): weights.  Two "unpack" warps read the packed words
 //     of 128 channels x one 256-k block, expand them to int8 lanes (value
 //     64 * (code - 2): one shift + one LOP3 per four weights) and store them
@@ -16,12 +16,15 @@
 //   D: int32 in tensor memory, lane = channel, column = token.  Because a lane is
 //     a channel, a drain thread needs one weight scale per group, not one per value.
 // Per 64-k group (or whatever the scale group is) an MMA thread issues K = 32 steps
-// into one of four accumulator buffers (all 512 TMEM columns); two threads share
-// the issuing, alternating groups.  Eight "drain" warps (two per TMEM lane quarter,
-// 64 token columns each) read finished buffers with tcgen05.ld, software-pipelined
-// in 32-column halves, convert to fp32 and accumulate scale * value in registers
-// with packed fp32 FMAs.  Every wait on an mbarrier is bounded; a wait that gives
-// up sets the status word of the workspace and the CTA winds down.
+// into one of four accumulator buffers (all 512 TMEM columns).  MMA and drain hand
+// buffers over in units of two consecutive groups (a barrier round trip costs as much
+// as the MMAs of a 64-k group); two threads share the issuing, one unit slot each.
+// Eight "drain" warps (two per TMEM lane quarter, 64 token columns each) read finished
+// buffers with tcgen05.ld, software-pipelined in 32-column halves, convert to fp32 and
+// accumulate scale * value in registers with packed fp32 FMAs.  Stage slots and units
+// are numbered across tiles, so the producers run ahead into the next tile while the
+// drain warps store y.  Every wait on an mbarrier is bounded; a wait that gives up
+// sets the status word of the workspace and the CTA winds down.
 #include <cuda.h>
 
 #include "w2a8_common.cuh"
