@@ -34,6 +34,9 @@ CASES = [
     (200, 256, 1536, 512),      # a scale group spans two stages
     (257, 128, 1280, 0),        # one scale per channel
     (512, 512, 4096, 64),       # configuration-4-like slice: K of gate/up
+    (640, 4096, 512, 64),       # 160 tiles: more than one tile per persistent CTA
+    (384, 6400, 768, 256),      # 150 tiles, three groups per tile (the last hand-off unit has one group)
+    (200, 19200, 256, 128),     # 300 tiles of a single stage each, ragged token tiles
 ]
 
 
@@ -73,3 +76,28 @@ def test_prefill_matches_streaming_path(gpu, monkeypatch):
     monkeypatch.setenv("W2A8_PREFILL", "0")
     y_st = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws).cpu().numpy()
     assert np.abs(y_tc - y_st).max() <= TOL * np.abs(y_st).max()
+
+
+@pytest.mark.parametrize("K,N", [(4096, 14336), (14336, 4096)])
+def test_prefill_full_size_sampled_rows(gpu, oracle, K, N):
+    """Prefill configuration at full size (M = 2048, group 64): every channel of a sample of
+    token rows -- first and last row of the first, a middle and the last token tile, plus a few
+    seeded ones -- against the reference."""
+    torch, b = gpu
+    M, g = 2048, 64
+    codes, s_w = synth.make_linear(4000 + K, K, N, g)
+    bits = synth.activations_bf16(4000 + N, M, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    rows = sorted(set([0, 127, 1024, 1151, M - 128, M - 1] +
+                      [int(r) for r in np.random.default_rng(K).integers(0, M, size=6)]))
+    a_ref, s_ref = oracle.quantize(bits[rows])
+    assert np.array_equal(a.cpu().numpy()[rows], a_ref)
+    y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+    got = y.cpu().numpy()[rows].astype(np.float64)
+    err = np.abs(got - y_ref).max(axis=1)
+    assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), float((err / np.abs(y_ref).max(axis=1)).max())
