@@ -670,10 +670,60 @@ def prefill_probe(device, peaks, Ms=(512, 2048, 8192), reps=5):
                          "status": b.w2a8_workspace_status(ws)})
             del x, a, y, ws
         del packed
+    # the same kernel with coarser scale groups on gate/up at M = 2048: the per-group drain halves
+    # (group 128), quarters (256) and all but vanishes (one scale per channel)
+    by_group = []
+    name, K, N = cfg["shapes"][0]
+    M = 2048
+    bits = synth.activations_bf16(cfg["seed"] + 7 + M, M, K)
+    x = torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+    a, s_a = b.a8_quantize(x)
+    y = torch.empty((M, N), dtype=torch.float32, device=device)
+    for g in (64, 128, 256, K):
+        codes, s_w = synth.make_linear(synth.shape_seed(cfg, 0) + g, K, N, g)
+        packed = b.w2_pack(torch.from_numpy(codes).to(device))
+        s_w_d = torch.from_numpy(s_w).to(device)
+        del codes
+        ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g), device=device)
+        for _ in range(3):
+            b.w2a8_gemm(a, s_a, packed, s_w_d, g, ws, y)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            b.w2a8_gemm(a, s_a, packed, s_w_d, g, ws, y)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        tops = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+        by_group.append({"shape": f"{K}x{N}", "M": M, "group": g, "ms_gemm": ms, "tops": tops,
+                         "frac_of_measured_int8_sustained": tops / int8_peak_sustained,
+                         "status": b.w2a8_workspace_status(ws)})
+        del packed, s_w_d, ws
+    # library int8 GEMM on the same device as a second, directly measured denominator
+    lib_int8 = None
+    try:
+        n = 8192
+        ai = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=device)
+        bi = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=device)
+        for _ in range(3):
+            torch._int_mm(ai, bi)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(10):
+            torch._int_mm(ai, bi)
+        e1.record()
+        torch.cuda.synchronize()
+        lib_int8 = {"what": "torch._int_mm 8192^3 (library int8 GEMM), 10 back-to-back calls",
+                    "tops": 2.0 * n ** 3 / (e0.elapsed_time(e1) / 10 * 1e-3) / 1e12}
+        del ai, bi
+    except Exception as exc:      # not available in this torch build: report, do not fail the bench
+        lib_int8 = {"what": "torch._int_mm 8192^3", "unavailable": str(exc)[:200]}
     return {"unit": "int8 TOPS", "peak_measured_burst": int8_peak_burst,
             "peak_measured_sustained": int8_peak_sustained,
             "peak_note": "measured cuBLAS bf16 peak x 2 (nominal int8 : bf16 ratio); nominal dense int8 4500",
-            "rows": rows}
+            "library_int8_gemm": lib_int8, "rows": rows, "by_group_m2048": by_group}
 
 
 def run_kernel_profile(args):
