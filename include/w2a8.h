@@ -143,6 +143,27 @@ int w2a8_gemm_partials(const int8_t *a, const uint32_t *packed, int32_t *partial
                        void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * w2a8_linear -- a8_quantize and w2a8_gemm in one call: y = W2A8(x) for bf16
+ * activations in device memory (the fused "bf16 in, scaled output" operator of
+ * Sec. II-D, where computing the abs-max scales inside the GEMM pays off for
+ * GEMV-sized problems and not for large GEMMs).
+ *   x_bf16  [M][K] bf16 bit patterns, DEVICE
+ *   a, a_scale   caller-provided DEVICE buffers ([M][K] int8, [M] fp32) that
+ *           receive exactly what a8_quantize would write; they stay valid, so
+ *           later w2a8_gemm calls on other weight matrices can reuse them (the
+ *           k and v projections after q, up after gate)
+ *   the rest as for w2a8_gemm (same workspace size).
+ * This enqueues the two kernels, chained by programmatic dependent launch: on
+ * B200 that measured faster than a single launch with quantiser CTAs inside the
+ * GEMM grid (see the implementation), so the fusion is one of interface, not of
+ * kernels.
+ * a, a_scale and y are bitwise what a8_quantize + w2a8_gemm produce.
+ */
+int w2a8_linear(const void *x_bf16, int8_t *a, float *a_scale, const uint32_t *packed,
+                const float *w_scale, float *y, int M, int N, int K, int group,
+                void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Workspace size for w2a8_linear_host: staging for x, a, a_scale and y plus
  * the GEMM workspace.  Zero-fill once with w2a8_workspace_init.
  */

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libw2a8.so")
 EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
-    "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
+    "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
 ]
 
 _lib = None
@@ -53,12 +53,13 @@ def lib() -> ctypes.CDLL:
         L.w2a8_workspace_status.argtypes = [vp, vp]
         L.w2a8_gemm.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_partials.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
+        L.w2a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear_host_workspace_bytes.restype = sz
         L.w2a8_linear_host_workspace_bytes.argtypes = [i, i, i, i]
         L.w2a8_linear_host.argtypes = [vp, i, i, vp, vp, i, i, vp, vp, sz, vp]
         L.w2a8_gemm_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp]
         for name in ("w2_pack", "a8_quantize", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm",
-                     "w2a8_gemm_partials", "w2a8_linear_host", "w2a8_gemm_static"):
+                     "w2a8_gemm_partials", "w2a8_linear", "w2a8_linear_host", "w2a8_gemm_static"):
             getattr(L, name).restype = i
         _lib = L
     return _lib
@@ -148,6 +149,25 @@ def w2a8_gemm(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor, w_sc
                            group, _ptr(workspace), workspace.numel() * workspace.element_size(),
                            _stream(stream)), "w2a8_gemm")
     return y
+
+
+def w2a8_linear(x: torch.Tensor, packed: torch.Tensor, w_scale: torch.Tensor, group: int,
+                workspace: torch.Tensor, a: torch.Tensor | None = None, a_scale: torch.Tensor | None = None,
+                y: torch.Tensor | None = None, stream=None):
+    """bf16 x [M][K] (device) -> (y fp32 [M][N], a int8 [M][K], a_scale fp32 [M]) in one call; see
+    w2a8_linear in include/w2a8.h.  a / a_scale receive what a8_quantize would write."""
+    M, K = x.shape
+    N = packed.shape[0]
+    if a is None:
+        a = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    if a_scale is None:
+        a_scale = torch.empty((M,), dtype=torch.float32, device=x.device)
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    _check(lib().w2a8_linear(_ptr(x), _ptr(a), _ptr(a_scale), _ptr(packed), _ptr(w_scale), _ptr(y), M, N, K,
+                             group, _ptr(workspace), workspace.numel() * workspace.element_size(),
+                             _stream(stream)), "w2a8_linear")
+    return y, a, a_scale
 
 
 def w2a8_gemm_partials(a: torch.Tensor, packed: torch.Tensor, group: int, workspace: torch.Tensor,

@@ -11,6 +11,7 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st);
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
+
 bool prefill_supported(int M, int N, int K, int group);
 int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const float *w_scale,
                    float *y, int32_t *partials, int M, int N, int K, int group, int *status,
@@ -313,6 +314,28 @@ int w2a8_gemm_partials(const int8_t *a, const uint32_t *packed, int32_t *partial
 }
 
 static inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+
+int w2a8_linear(const void *x_bf16, int8_t *a, float *a_scale, const uint32_t *packed,
+                const float *w_scale, float *y, int M, int N, int K, int group, void *workspace,
+                size_t workspace_bytes, void *stream) {
+    if (!x_bf16 || !a || !a_scale || !packed || !w_scale || !y) return W2A8_ERR_NULL;
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
+    if (!aligned16(x_bf16) || !aligned16(a) || !aligned16(packed) || !aligned16(y) || !aligned16(w_scale) ||
+        (reinterpret_cast<uintptr_t>(a_scale) & 3u))
+        return W2A8_ERR_ALIGN;
+    const size_t need = decode_workspace_bytes(M, N, K, si);
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
+    if (int st = check_device()) return st;
+    // Two launches chained by programmatic dependent launch.  A single-launch form (M extra CTAs
+    // of the GEMM grid quantise one token each and publish the rows through flags in the
+    // workspace; the other CTAs request their weights and then poll) was built and measured on
+    // B200 on the gate/up GEMV, back to back: GEMM alone 5.1 us, quantiser launch + GEMM 6.3 us,
+    // single launch 9.0 us -- handing the rows to the other CTAs costs several global round trips
+    // (fence, flag, poll, fence), more than the dependent launch it replaces -- so it was dropped.
+    if (int st = a8_quantize(x_bf16, M, K, a, a_scale, stream)) return st;
+    return w2a8_gemm(a, a_scale, packed, w_scale, y, M, N, K, group, workspace, workspace_bytes, stream);
+}
 
 size_t w2a8_linear_host_workspace_bytes(int M, int N, int K, int group) {
     const size_t g = w2a8_workspace_bytes(M, N, K, group);

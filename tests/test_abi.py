@@ -85,6 +85,9 @@ def test_argument_errors_are_detected_on_the_host(lib):
     assert lib.w2a8_gemm(p, p, p, p, p, 1, 16, 64, 64, None, 0, None) == WS
     assert lib.w2a8_gemm(p, p, p, p, p, 1, 16, 64, 64, p, 8, None) == WS
     assert lib.w2a8_gemm_partials(p, p, None, 1, 16, 64, 64, p, 1 << 15, None) == NULLP
+    assert lib.w2a8_linear(None, p, p, p, p, p, 1, 16, 64, 64, p, 1 << 15, None) == NULLP
+    assert lib.w2a8_linear(p, p, p, p, p, p, 1, 16, 64, 32, p, 1 << 15, None) == SHAPE
+    assert lib.w2a8_linear(p, p, p, p, p, p, 1, 16, 64, 64, p, 8, None) == WS
     assert lib.w2a8_linear_host(None, 1, 64, p, p, 16, 64, p, p, 1 << 15, None) == NULLP
     assert lib.w2a8_linear_host(p, 1, 64, p, p, 16, 48, p, p, 1 << 15, None) == SHAPE
     assert lib.w2a8_linear_host(p, 1, 64, p, p, 16, 64, p, p, 16, None) == WS

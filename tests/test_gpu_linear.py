@@ -1,0 +1,100 @@
+"""GPU parity of the operator w2a8_linear (bf16 in, scaled output): bitwise equal to
+a8_quantize + w2a8_gemm, and against the CPU reference."""
+import numpy as np
+import pytest
+
+from paper_2508_06753_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2508_06753_b200 import binding, build
+    build.build()
+    binding.lib()
+    return torch, binding
+
+
+def _dev(torch, arr):
+    return torch.from_numpy(np.ascontiguousarray(arr)).cuda()
+
+
+CASES = [
+    # M, N, K, group (0 = K)
+    (1, 2048, 2048, 64),        # one token, one chunk
+    (1, 256, 14336, 64),        # split-K inside a cluster
+    (4, 1024, 4096, 128),
+    (8, 4096, 4096, 64),
+    (16, 512, 4096, 64),        # two slabs of eight tokens
+    (20, 80, 14336 + 768, 64),  # ragged slabs, ragged last chunk, few tiles
+    (32, 1024, 8192, 0),        # one scale per channel
+    (3, 1600, 1600, 64),        # K not a multiple of 256
+    (40, 256, 1024, 64),        # several 32-token slabs
+    (96, 256, 1024, 64),        # tensor-core shape
+]
+
+
+@pytest.mark.parametrize("M,N,K,group", CASES)
+def test_linear_matches_two_calls_and_reference(gpu, oracle, M, N, K, group):
+    torch, b = gpu
+    g = K if group == 0 else group
+    codes, s_w = synth.make_linear(11 * M + N + K, K, N, g)
+    bits = synth.activations_bf16(M + K, M, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    s_w_d = _dev(torch, s_w)
+    x = _dev(torch, bits.view(np.int16)).view(torch.bfloat16)
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    a2, s2 = b.a8_quantize(x)
+    y2 = b.w2a8_gemm(a2, s2, packed, s_w_d, g, ws)
+    for call in range(3):
+        y, a, s = b.w2a8_linear(x, packed, s_w_d, g, ws)
+        torch.cuda.synchronize()
+        assert b.w2a8_workspace_status(ws) == 0
+        assert torch.equal(a, a2) and torch.equal(s, s2), call
+        assert torch.equal(y, y2), call
+    y3 = b.w2a8_gemm(a, s, packed, s_w_d, g, ws)    # a plain call on the same workspace afterwards
+    assert torch.equal(y3, y2)
+    a_ref, s_ref = oracle.quantize(bits)
+    assert np.array_equal(a.cpu().numpy(), a_ref)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+    err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max(axis=1)
+    assert (err <= TOL * np.abs(y_ref).max(axis=1)).all()
+
+
+def test_linear_in_a_graph_with_changing_inputs(gpu, oracle):
+    """Replays of one captured operator with new activations each time."""
+    torch, b = gpu
+    M, N, K, g = 4, 4096, 4096, 64
+    codes, s_w = synth.make_linear(5, K, N, g)
+    packed = b.w2_pack(_dev(torch, codes))
+    s_w_d = _dev(torch, s_w)
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    x = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    a = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    s = torch.empty((M,), dtype=torch.float32, device="cuda")
+    y = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        b.w2a8_linear(x, packed, s_w_d, g, ws, a, s, y)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            b.w2a8_linear(x, packed, s_w_d, g, ws, a, s, y)
+            b.w2a8_linear(x, packed, s_w_d, g, ws, a, s, y)      # back to back on one workspace
+        for rep in range(4):
+            bits = synth.activations_bf16(100 + rep, M, K)
+            x.copy_(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
+            graph.replay()
+            torch.cuda.synchronize()
+            assert b.w2a8_workspace_status(ws) == 0
+            a_ref, s_ref = oracle.quantize(bits)
+            assert np.array_equal(a.cpu().numpy(), a_ref), rep
+            y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+            err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max(axis=1)
+            assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), rep
