@@ -98,3 +98,44 @@ def test_linear_in_a_graph_with_changing_inputs(gpu, oracle):
             y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
             err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max(axis=1)
             assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), rep
+
+
+@pytest.mark.parametrize("M", [1, 8, 16])
+def test_back_to_back_launches_reusing_one_activation_buffer(gpu, oracle, M):
+    """quantise(x1 -> a), gemm(a), quantise(x2 -> a), gemm(a), ... in one stream with programmatic
+    dependent launch: a GEMM CTA can be resident while the previous GEMM (which read the old
+    contents of `a` through L1) is still running on the same SM; it must still read the new
+    contents after its dependency wait."""
+    torch, b = gpu
+    N, K, g = 14336, 4096, 64
+    codes, s_w = synth.make_linear(21, K, N, g)
+    packed = b.w2_pack(_dev(torch, codes))
+    s_w_d = _dev(torch, s_w)
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    rounds = 6
+    all_bits = [synth.activations_bf16(300 + r, M, K) for r in range(rounds)]
+    xs = [_dev(torch, bits.view(np.int16)).view(torch.bfloat16) for bits in all_bits]
+    a = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    s = torch.empty((M,), dtype=torch.float32, device="cuda")
+    ys = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _ in range(rounds)]
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        def body():
+            for r in range(rounds):
+                b.a8_quantize(xs[r], a, s)
+                b.w2a8_gemm(a, s, packed, s_w_d, g, ws, ys[r])
+        body()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            body()
+        for y in ys:
+            y.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    for r in range(rounds):
+        a_ref, s_ref = oracle.quantize(all_bits[r])
+        y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+        err = np.abs(ys[r].cpu().numpy().astype(np.float64) - y_ref).max(axis=1)
+        assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), r
