@@ -529,10 +529,13 @@ static DecodePlan decode_plan_mt(int M, int N, int K, const ShapeInfo &si, int m
         if (forced > chunks) chunks = forced;
     } else {
         // Measured on B200: the whole grid should field about 2000 warps or more so that
-        // enough loads are in flight; beyond that the cross-CTA sum costs more than
-        // further splitting gains.
+        // enough loads are in flight, and it pays to go on splitting (down to one cell per
+        // warp) as long as all CTAs are still resident at once (8 per SM for one slab, 4 for
+        // wider slabs); beyond that the extra round of CTAs costs more than the split gains.
         const int min_warps = env_int("W2A8_MIN_WARPS", 2000);
-        while ((long long)pl.groups * pl.slabs * kDecodeWarps * chunks < min_warps &&
+        const long long resident = 148ll * (mt == 1 ? 8 : 4);
+        auto ctas = [&](int c) { return (long long)pl.groups * pl.slabs * c; };
+        while ((ctas(chunks) * kDecodeWarps < min_warps || ctas(chunks * 2) <= resident) &&
                (si.blocks / (chunks * 2)) >= ks)
             chunks *= 2;
     }
