@@ -25,10 +25,21 @@ _lib = None
 
 def build(force: bool = False) -> str:
     """Compile the C reference into ``libw2a8_ref.so`` next to its source."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        cmd = ["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-shared",
-               "-fPIC", "-o", _LIB, _SRC, "-lm"]
-        subprocess.run(cmd, check=True)
+    def stale():
+        return not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale():
+        import fcntl
+        with open(_LIB + ".lock", "w") as lock:        # several test or bench processes may race here
+            fcntl.flock(lock, fcntl.LOCK_EX)
+            try:
+                if force or stale():
+                    tmp = _LIB + f".tmp{os.getpid()}"
+                    cmd = ["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-shared",
+                           "-fPIC", "-o", tmp, _SRC, "-lm"]
+                    subprocess.run(cmd, check=True)
+                    os.replace(tmp, _LIB)
+            finally:
+                fcntl.flock(lock, fcntl.LOCK_UN)
     return _LIB
 
 

@@ -38,15 +38,26 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
-    cmd = [_nvcc(), "-std=c++17", "-O3", "-lineinfo",
-           "-gencode", "arch=compute_100a,code=sm_100a",
-           "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
-           "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB] + sources()
-    if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    subprocess.run(cmd, check=True)
+    # several processes (one per GPU) may get here at once: one builds, the others wait for it
+    import fcntl
+    with open(LIB + ".lock", "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if not force and not _stale():
+                return LIB
+            tmp = LIB + f".tmp{os.getpid()}"
+            cmd = [_nvcc(), "-std=c++17", "-O3", "-lineinfo",
+                   "-gencode", "arch=compute_100a,code=sm_100a",
+                   "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
+                   "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+                   "-o", tmp] + sources()
+            if verbose:
+                cmd.insert(1, "-Xptxas")
+                cmd.insert(2, "-v")
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, LIB)        # atomic: nobody ever loads a half-written library
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
     return LIB
 
 
