@@ -304,6 +304,10 @@ w2a8_decode_kernel(const DecodeParams p) {
     for (int j = 0; j < RING; ++j) {
         if (j < full_cells) post_cell(j);
         cp_async_commit();
+        // Let the next kernel of the stream start once the first cell is requested (measured: a
+        // little better than at kernel entry or after all requests; the request instructions
+        // themselves queue for microseconds while the memory system is busy).
+        if (j == 0) pdl_launch_dependents();
     }
     if (tail_mine) {
         // trailing block of K with R < 4 slices: this lane's words are t*R .. t*R+R-1 of the
@@ -332,7 +336,6 @@ w2a8_decode_kernel(const DecodeParams p) {
         }
     }
     W2A8_TRACE_POINT(1);
-    pdl_launch_dependents();
     pdl_wait();
     W2A8_TRACE_POINT(2);
 
