@@ -8,7 +8,8 @@
 // Work split.  A "cell" is one 16-channel tile x one 256-k block: 1 KB of packed
 // weights plus its scales.  A CTA of 4 warps owns TG tiles and one chunk of the
 // contraction; its warps are arranged TG tiles x KS = 4 / TG K-lanes, and the
-// K-lanes take interleaved blocks of the chunk, at most RING cells each.  The
+// K-lanes take runs of consecutive blocks of the chunk, at most RING cells each
+// (consecutive, so that the scale pieces a warp requests are neighbours).  The
 // K-lanes of a tile are summed through shared memory in a fixed order.  Chunks
 // (grid.y; used when K has more blocks than the K-lanes can hold, or when the
 // grid would leave SMs idle) are summed in chunk order: inside a thread-block
@@ -250,14 +251,18 @@ w2a8_decode_kernel(const DecodeParams p) {
     const int mrows = min(8 * MT, p.M - m0);
     W2A8_TRACE_POINT(0);
 
-    // This warp's cells: cell c is block kb0 + c * KS of tile tile0 + tl (at most RING of them).
+    // This warp's cells: the chunk is cut into KS runs of consecutive blocks, one per K-lane; cell c
+    // is block kb0 + c of tile tile0 + tl (at most RING of them).  Consecutive blocks matter for the
+    // scales: the 16-byte pieces a warp asks for, cell after cell, are then neighbours in memory
+    // (64 bytes per channel), which DRAM serves far better than isolated 16-byte pieces.
     const int n0 = (tile0 + tl) * 16;
-    const int kb0 = kb_begin + ks;
-    const int my_cells = (tile0 + tl < ntiles) ? (int)((unsigned)(nb - ks + KS - 1) / KS) : 0;
-    // only the last block of K can have fewer than four slices
+    const int cpw = (int)((unsigned)(nb + KS - 1) / KS);          // cells per K-lane
+    const int kb0 = kb_begin + ks * cpw;
+    const int my_cells = (tile0 + tl < ntiles) ? max(0, min(cpw, nb - ks * cpw)) : 0;
+    // only the last block of K can have fewer than four slices; it is the last cell of its K-lane
     const bool tail_cta = (kb_end == p.blocks) && (p.tail_slices != 4);
-    const bool tail_mine = tail_cta && (nb - 1 - ks) >= 0 && (nb - 1 - ks) % KS == 0;   // ... and it is this warp's
-    const int tail_cell = tail_mine ? (nb - 1 - ks) / KS : -1;
+    const bool tail_mine = tail_cta && my_cells > 0 && ks * cpw + my_cells == nb;
+    const int tail_cell = tail_mine ? my_cells - 1 : -1;
     const int full_cells = my_cells - (tail_mine ? 1 : 0);
 
     // Landing slots of this warp in shared memory.  Weights: slot c of a lane holds its two
@@ -268,7 +273,7 @@ w2a8_decode_kernel(const DecodeParams p) {
     unsigned char *sslots = smem + warp * kWarpBytes + RING * kSlotBytes;
     const uint32_t wslots_u32 = smem_u32(wslots);
     const uint32_t sslot_u32 = smem_u32(sslots) + (lane & 15) * 16;
-    // word 4t of block kb0 in rows n0 + gq and n0 + gq + 8; cell c is 16 * KS words on
+    // word 4t of block kb0 in rows n0 + gq and n0 + gq + 8; cell c is 16 words on
     const uint32_t *wrow0 = p.packed + (size_t)(n0 + gq) * p.words_per_row + 16 * kb0 + 4 * t;
     const uint32_t *wrow1 = wrow0 + (size_t)8 * p.words_per_row;
     // first scale of block kb0 in row n0 + (lane & 15)
@@ -278,21 +283,21 @@ w2a8_decode_kernel(const DecodeParams p) {
         if constexpr (SPP != 4) srow += SPB * kb0;
     }
     auto post_cell = [&](int c) {   // c is a constant after unrolling
-        cp_async16(wslots_u32 + c * kSlotBytes, wrow0 + c * (16 * KS));
-        cp_async16(wslots_u32 + c * kSlotBytes + 32 * 16, wrow1 + c * (16 * KS));
+        cp_async16(wslots_u32 + c * kSlotBytes, wrow0 + c * 16);
+        cp_async16(wslots_u32 + c * kSlotBytes + 32 * 16, wrow1 + c * 16);
         if constexpr (!PARTIALS) {
             if (lane < 16) {
                 if constexpr (SPP == 4) {
-                    const int kb = kb0 + c * KS;
+                    const int kb = kb0 + c;
                     const int gi = p.blocks_per_group >= p.blocks ? 0 : kb / p.blocks_per_group;
                     cp_async4(sslot_u32 + c * kScaleBytes, srow + gi);
                 } else if (p.s_vec) {
-                    if constexpr (SPP == 1) cp_async16(sslot_u32 + c * kScaleBytes, srow + c * (SPB * KS));
-                    else                    cp_async8(sslot_u32 + c * kScaleBytes, srow + c * (SPB * KS));
+                    if constexpr (SPP == 1) cp_async16(sslot_u32 + c * kScaleBytes, srow + c * SPB);
+                    else                    cp_async8(sslot_u32 + c * kScaleBytes, srow + c * SPB);
                 } else {
 #pragma unroll
                     for (int i = 0; i < SPB; ++i)
-                        cp_async4(sslot_u32 + c * kScaleBytes + 4 * i, srow + c * (SPB * KS) + i);
+                        cp_async4(sslot_u32 + c * kScaleBytes + 4 * i, srow + c * SPB + i);
                 }
             }
         }
@@ -315,7 +320,7 @@ w2a8_decode_kernel(const DecodeParams p) {
         const int R = p.tail_slices;
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-            const uint32_t *wp = (r ? wrow1 : wrow0) + tail_cell * (16 * KS) - 4 * t + t * R;
+            const uint32_t *wp = (r ? wrow1 : wrow0) + tail_cell * 16 - 4 * t + t * R;
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             v.x = __ldg(wp);
             if (R > 1) v.y = __ldg(wp + 1);
@@ -326,11 +331,11 @@ w2a8_decode_kernel(const DecodeParams p) {
             if (lane < 16) {
                 float *dst = reinterpret_cast<float *>(sslots + tail_cell * kScaleBytes + lane * 16);
                 if constexpr (SPP == 4) {
-                    const int kb = kb0 + tail_cell * KS;
+                    const int kb = kb0 + tail_cell;
                     dst[0] = __ldg(srow + (p.blocks_per_group >= p.blocks ? 0 : kb / p.blocks_per_group));
                 } else {
                     const int nsc = (R + SPP - 1) / SPP;
-                    for (int i = 0; i < nsc; ++i) dst[i] = __ldg(srow + tail_cell * (SPB * KS) + i);
+                    for (int i = 0; i < nsc; ++i) dst[i] = __ldg(srow + tail_cell * SPB + i);
                 }
             }
         }
@@ -366,9 +371,9 @@ w2a8_decode_kernel(const DecodeParams p) {
             const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
             const int8_t *bc[MT];
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + c * (KS * kBlockK);
+            for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + c * kBlockK;
             compute_cell<MT, SPP, ONE, PARTIALS, true>(p, w0s, w1s, sc0 + c * kScaleBytes, sc1 + c * kScaleBytes,
-                                                       bc, kb0 + c * KS, n0, m0, gq, t, acc);
+                                                       bc, kb0 + c, n0, m0, gq, t, acc);
         }
     }
     if (tail_mine) {   // the trailing block is this warp's last cell; its words and scales were stored directly
@@ -379,9 +384,9 @@ w2a8_decode_kernel(const DecodeParams p) {
         const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
         const int8_t *bc[MT];
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + (size_t)tail_cell * (KS * kBlockK);
+        for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + (size_t)tail_cell * kBlockK;
         compute_cell<MT, SPP, ONE, PARTIALS, false>(p, w0s, w1s, sc0 + tail_cell * kScaleBytes,
-                                                    sc1 + tail_cell * kScaleBytes, bc, kb0 + tail_cell * KS,
+                                                    sc1 + tail_cell * kScaleBytes, bc, kb0 + tail_cell,
                                                     n0, m0, gq, t, acc);
     }
     W2A8_TRACE_POINT(5);
@@ -508,8 +513,8 @@ struct DecodePlan {
     size_t smem;
 };
 
-// Launch plan for slabs of 8 * mt tokens.  One tile per CTA, its four warps take interleaved
-// blocks of K (shortest serial work per warp).  K-chunks are added when a warp would
+// Launch plan for slabs of 8 * mt tokens.  One tile per CTA, its four warps take equal
+// runs of consecutive blocks of K (shortest serial work per warp).  K-chunks are added when a warp would
 // otherwise have more cells than landing slots, or when the grid would leave most SMs idle.
 static DecodePlan decode_plan_mt(int M, int N, int K, const ShapeInfo &si, int mt) {
     DecodePlan pl;
