@@ -48,6 +48,10 @@ def _load():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.ref_num_threads.restype = ctypes.c_int
+        _lib.ref_half_to_float.restype = ctypes.c_float
+        _lib.ref_half_to_float.argtypes = [ctypes.c_uint16]
+        _lib.ref_float_to_bf16.restype = ctypes.c_uint16
+        _lib.ref_float_to_bf16.argtypes = [ctypes.c_float]
     return _lib
 
 
@@ -116,3 +120,33 @@ def gemm(a: np.ndarray, a_scale: np.ndarray, codes: np.ndarray, w_scale: np.ndar
     _load().ref_gemm(_p(a), _p(a_scale), _p(codes), _p(w_scale), ctypes.c_int(M),
                      ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(g), _p(y))
     return y
+
+
+def half_to_float(h: int) -> float:
+    """IEEE binary16 bit pattern -> value (exact)."""
+    return float(_load().ref_half_to_float(int(h) & 0xFFFF))
+
+
+def float_to_bf16(f: float) -> int:
+    """fp32 value -> bf16 bit pattern, round to nearest even."""
+    return int(_load().ref_float_to_bf16(float(np.float32(f))))
+
+
+def gemm_h(a: np.ndarray, a_scale: np.ndarray, codes: np.ndarray, w_scale_h: np.ndarray, g: int):
+    """16-bit recipe: w_scale_h holds binary16 bit patterns uint16 [N][K/g].
+
+    Returns (y fp32 [M][N], the same values rounded to bf16 bit patterns uint16 [M][N]).
+    """
+    a = np.ascontiguousarray(a, dtype=np.int8)
+    a_scale = np.ascontiguousarray(a_scale, dtype=np.float32)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    w_scale_h = np.ascontiguousarray(w_scale_h, dtype=np.uint16)
+    M, K = a.shape
+    N = codes.shape[0]
+    assert codes.shape[1] == K and K % g == 0
+    assert w_scale_h.shape == (N, K // g) and a_scale.shape == (M,)
+    y32 = np.empty((M, N), dtype=np.float32)
+    y16 = np.empty((M, N), dtype=np.uint16)
+    _load().ref_gemm_h(_p(a), _p(a_scale), _p(codes), _p(w_scale_h), ctypes.c_int(M),
+                       ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(g), _p(y32), _p(y16))
+    return y32, y16

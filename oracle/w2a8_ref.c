@@ -29,6 +29,13 @@
  *   ref_gemm : Sec. II-D dequantisation: int32 -> float, times the product
  *       of activation scale and weight scale; with K-groups the weight scale
  *       is applied per group before summing.
+ *   ref_half_to_float / ref_float_to_bf16 / ref_gemm_h : the recipe of the
+ *       end-to-end ternary section (groups of 128 along K, weight scales
+ *       stored in 16 bits; the 16-bit format is read as IEEE binary16, the
+ *       type the direct-conversion listing of Sec. II names for its scale):
+ *       the same sums as ref_gemm with each scale first widened exactly to
+ *       fp32, and an optional bf16 result (round to nearest even of the
+ *       fp32 result).
  *
  * Parity pins: every routine here is pinned by tests that do not reuse this
  * code (hand-written golden words, exhaustive exact-rational evaluation of
@@ -196,5 +203,61 @@ void ref_gemm(const int8_t *a, const float *a_scale, const uint8_t *codes,
                 acc += (double)w_scale[(size_t)n * G + gi] * (double)p;
             }
             y[(size_t)m * N + n] = (float)((double)a_scale[m] * acc);
+        }
+}
+
+/* ------------------------------------------------- 16-bit scales / outputs */
+/*
+ * IEEE binary16 bit pattern -> its value, field by field: 1 sign bit, 5
+ * exponent bits (bias 15), 10 fraction bits; exponent 0 = subnormal
+ * (fraction * 2^-24), exponent 31 = infinity / NaN.  Every binary16 value is
+ * a float, so the result is exact.
+ */
+float ref_half_to_float(uint16_t h) {
+    int sign = (h >> 15) & 1, e = (h >> 10) & 31, frac = h & 1023;
+    double v;
+    if (e == 0)       v = ldexp((double)frac, -24);
+    else if (e == 31) v = frac ? (double)NAN : (double)INFINITY;
+    else              v = ldexp((double)(1024 + frac), e - 25);
+    return (float)(sign ? -v : v);
+}
+
+/*
+ * float -> bf16 bit pattern (the upper 16 bits of a float whose lower 16 bits
+ * are zero), round to nearest, ties to the even 16-bit pattern; overflow goes
+ * to infinity as in IEEE; NaN stays NaN (quiet bit set).  Written as a
+ * comparison of the discarded half with one half unit, not as a bias trick.
+ */
+uint16_t ref_float_to_bf16(float f) {
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t keep = u >> 16, rest = u & 0xffffu;
+    if (rest > 0x8000u || (rest == 0x8000u && (keep & 1u))) keep += 1u;   /* may carry into the exponent */
+    return (uint16_t)keep;
+}
+
+/*
+ * ref_gemm with w_scale given as binary16 bit patterns [N][K/g].  y32 (fp32
+ * [M][N]) is always written; y16 (bf16 bit patterns [M][N]) when not NULL is
+ * the rounding of the same fp32 values.
+ */
+void ref_gemm_h(const int8_t *a, const float *a_scale, const uint8_t *codes,
+                const uint16_t *w_scale_h, int M, int N, int K, int g, float *y32, uint16_t *y16) {
+    int G = K / g;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int m = 0; m < M; ++m) {
+            double acc = 0.0;
+            for (int gi = 0; gi < G; ++gi) {
+                int32_t p = 0;
+                for (int k = gi * g; k < (gi + 1) * g; ++k)
+                    p += (int32_t)a[(size_t)m * K + k] *
+                         ((int32_t)(codes[(size_t)n * K + k] & 3) - 2);
+                acc += (double)ref_half_to_float(w_scale_h[(size_t)n * G + gi]) * (double)p;
+            }
+            float r = (float)((double)a_scale[m] * acc);
+            y32[(size_t)m * N + n] = r;
+            if (y16) y16[(size_t)m * N + n] = ref_float_to_bf16(r);
         }
 }

@@ -65,6 +65,11 @@ def weight_scales(seed: int, N: int, G: int) -> np.ndarray:
     return (0.02 * np.exp(0.5 * z)).astype(np.float32)
 
 
+def weight_scales_h(seed: int, N: int, G: int) -> np.ndarray:
+    """IEEE binary16 bit patterns uint16 [N][G]: the fp32 scales of `weight_scales` stored in 16 bits."""
+    return weight_scales(seed, N, G).astype(np.float16).view(np.uint16)
+
+
 def activations_bf16(seed: int, M: int, K: int, outlier_frac: float = 0.0) -> np.ndarray:
     """bf16 bit patterns uint16 [M][K]; N(0,1), optional +-20 outliers.
 
