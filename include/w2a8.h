@@ -134,6 +134,28 @@ int w2a8_gemm(const int8_t *a, const float *a_scale, const uint32_t *packed,
               void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * w2a8_gemm with the storage recipe of the paper's end-to-end ternary section
+ * (groups of 128 along K, weight scales kept in 16 bits): the weight scales
+ * are IEEE binary16 bit patterns -- the 16-bit type the direct-conversion
+ * listing of Sec. II names for its scale -- and the result is fp32 or bf16.
+ *
+ *   w_scale_h  device, [N][K/group] binary16, row-major, 16-byte aligned
+ *   y          device, [M][N], 16-byte aligned: fp32 when y_is_bf16 == 0,
+ *              else bf16
+ * Everything else (a, a_scale, packed, shapes, group, workspace -- sized by
+ * w2a8_workspace_bytes --, stream, dispatch by M, error codes, asynchronous
+ * completion) is as for w2a8_gemm; any group w2a8_gemm takes is accepted.
+ *
+ * The value computed is that of w2a8_gemm called with every scale widened
+ * (exactly) to fp32; with y_is_bf16 that fp32 value is rounded once to bf16,
+ * to nearest, ties to even.  Scale bytes per weight drop from 32/group bit to
+ * 16/group bit, result bytes from 4 to 2 per element.
+ */
+int w2a8_gemm_h16(const int8_t* a, const float* a_scale, const uint32_t* packed,
+                  const uint16_t* w_scale_h, void* y, int y_is_bf16, int M, int N, int K, int group,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * w2a8_gemm_partials -- parity/debug export of the exact int32 per-group sums
  * P[m][n][gi] computed by the same inner-product code as w2a8_gemm.
  *   partials [M][N][K/group] int32, fully overwritten.

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libw2a8.so")
 EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
-    "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
+    "w2a8_gemm_h16", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
 ]
 
 _lib = None
@@ -52,6 +52,7 @@ def lib() -> ctypes.CDLL:
         L.w2a8_workspace_init.argtypes = [vp, sz, vp]
         L.w2a8_workspace_status.argtypes = [vp, vp]
         L.w2a8_gemm.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+        L.w2a8_gemm_h16.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_partials.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear_host_workspace_bytes.restype = sz
@@ -148,6 +149,26 @@ def w2a8_gemm(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor, w_sc
     _check(lib().w2a8_gemm(_ptr(a), _ptr(a_scale), _ptr(packed), _ptr(w_scale), _ptr(y), M, N, K,
                            group, _ptr(workspace), workspace.numel() * workspace.element_size(),
                            _stream(stream)), "w2a8_gemm")
+    return y
+
+
+def w2a8_gemm_h16(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor, w_scale_h: torch.Tensor,
+                  group: int, workspace: torch.Tensor, y: torch.Tensor | None = None,
+                  out_dtype: torch.dtype = torch.float32, stream=None):
+    """w2a8_gemm with binary16 weight scales (w_scale_h: float16 [N][K/group]) and an fp32 or bf16
+    result (the dtype of y, else out_dtype); see w2a8_gemm_h16 in include/w2a8.h."""
+    M, K = a.shape
+    N = packed.shape[0]
+    if w_scale_h.dtype != torch.float16:
+        raise TypeError("w_scale_h must be float16")
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype, device=a.device)
+    if y.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("y must be float32 or bfloat16")
+    _check(lib().w2a8_gemm_h16(_ptr(a), _ptr(a_scale), _ptr(packed), _ptr(w_scale_h), _ptr(y),
+                               1 if y.dtype == torch.bfloat16 else 0, M, N, K, group, _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _stream(stream)),
+           "w2a8_gemm_h16")
     return y
 
 

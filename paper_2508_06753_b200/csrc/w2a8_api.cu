@@ -8,14 +8,14 @@
 namespace w2a8 {
 
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
-                  const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
-                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st);
+                  const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
+                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16);
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
 
 bool prefill_supported(int M, int N, int K, int group);
-int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const float *w_scale,
-                   float *y, int32_t *partials, int M, int N, int K, int group, int *status,
-                   cudaStream_t st);
+int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
+                   void *y, int32_t *partials, int M, int N, int K, int group, int *status,
+                   cudaStream_t st, bool h16, bool y16);
 
 int env_int(const char *name, int dflt) {
     const char *v = getenv(name);
@@ -278,9 +278,11 @@ int w2a8_workspace_status(const void *workspace, void *stream) {
     return status;
 }
 
+// h16: w_scale holds binary16 values; y16 (with h16): y holds bf16 values.
 static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *packed,
-                       const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
-                       int group, void *workspace, size_t workspace_bytes, void *stream) {
+                       const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
+                       int group, void *workspace, size_t workspace_bytes, void *stream,
+                       bool h16 = false, bool y16 = false) {
     ShapeInfo si;
     if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
     if (!aligned16(a) || !aligned16(packed) || (y && !aligned16(y)) ||
@@ -293,9 +295,17 @@ static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *pa
     // many tokens: tensor-core path (tcgen05); few tokens, or shapes it does not tile: streaming path
     if (prefill_supported(M, N, K, group) && env_int("W2A8_PREFILL", 1) != 0)
         return launch_prefill(a, a_scale, packed, w_scale, y, partials, M, N, K, group,
-                              reinterpret_cast<int *>(workspace), (cudaStream_t)stream);
+                              reinterpret_cast<int *>(workspace), (cudaStream_t)stream, h16, y16);
     return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,
-                         (cudaStream_t)stream);
+                         (cudaStream_t)stream, h16, y16);
+}
+
+int w2a8_gemm_h16(const int8_t *a, const float *a_scale, const uint32_t *packed,
+                  const uint16_t *w_scale_h, void *y, int y_is_bf16, int M, int N, int K, int group,
+                  void *workspace, size_t workspace_bytes, void *stream) {
+    if (!a || !a_scale || !packed || !w_scale_h || !y) return W2A8_ERR_NULL;
+    return gemm_common(a, a_scale, packed, w_scale_h, y, nullptr, M, N, K, group, workspace,
+                       workspace_bytes, stream, true, y_is_bf16 != 0);
 }
 
 int w2a8_gemm(const int8_t *a, const float *a_scale, const uint32_t *packed, const float *w_scale,

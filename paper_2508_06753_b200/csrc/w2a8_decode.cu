@@ -35,6 +35,9 @@
 // One 128-bit unit per lane and channel holds word t of each of the four 64-k
 // slices of a block -- exactly what the four lanes of an MMA quad must supply
 // so that every MMA sums k of a single scale group.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "w2a8_common.cuh"
 
 namespace w2a8 {
@@ -64,7 +67,9 @@ struct DecodeParams {
     int chunks, blocks_per_chunk;
     int cluster;          // chunks > 1 and the chunks of a tile form one thread-block cluster
     int blocks_per_group; // 256-k blocks per scale group (groups of 256 and more)
-    int s_vec;            // the scales of a cell and channel can be copied as one 16- or 8-byte unit
+    int s_vec;            // the scales of a cell and channel can be copied as one unit (16/8 B fp32, 8/4 B binary16)
+    int h16;              // w_scale holds IEEE binary16 values (16-bit instances)
+    int y16;              // 16-bit instances only: y holds bf16 instead of fp32
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------
@@ -137,7 +142,8 @@ __device__ __forceinline__ uint4 ld_act16(const int8_t *p) {
 // w0s/w1s: this lane's four words (one per slice) of channels n0+gq and n0+gq+8;
 // sc0/sc1: the cell's scales of the same channels (shared memory, 16 bytes each);
 // brow[mt]: this lane's 16 activation bytes of slice 0 of the cell, token row of slab mt.
-template <int MT, int SPP, bool ONE, bool PARTIALS, bool FULL>
+// H16: the scales in shared memory are IEEE binary16 (2 bytes each) instead of fp32.
+template <int MT, int SPP, bool ONE, bool PARTIALS, bool FULL, bool H16>
 __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32_t (&w0s)[4],
                                              const uint32_t (&w1s)[4], const unsigned char *sc0,
                                              const unsigned char *sc1,
@@ -152,7 +158,24 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
 #pragma unroll
         for (int i = 0; i < 4; ++i) D[mt][i] = kMagicInt;
     float s0s[4 / SPP], s1s[4 / SPP];
-    if constexpr (!PARTIALS) {
+    if constexpr (!PARTIALS && H16) {
+        if constexpr (SPP == 4) {
+            s0s[0] = __half2float(*reinterpret_cast<const __half *>(sc0));
+            s1s[0] = __half2float(*reinterpret_cast<const __half *>(sc1));
+        } else if constexpr (SPP == 2) {
+            const float2 v0 = __half22float2(*reinterpret_cast<const __half2 *>(sc0));
+            const float2 v1 = __half22float2(*reinterpret_cast<const __half2 *>(sc1));
+            s0s[0] = v0.x; s0s[1] = v0.y; s1s[0] = v1.x; s1s[1] = v1.y;
+        } else {
+            const uint2 r0 = *reinterpret_cast<const uint2 *>(sc0), r1 = *reinterpret_cast<const uint2 *>(sc1);
+            const float2 v0 = __half22float2(*reinterpret_cast<const __half2 *>(&r0.x));
+            const float2 v1 = __half22float2(*reinterpret_cast<const __half2 *>(&r0.y));
+            const float2 v2 = __half22float2(*reinterpret_cast<const __half2 *>(&r1.x));
+            const float2 v3 = __half22float2(*reinterpret_cast<const __half2 *>(&r1.y));
+            s0s[0] = v0.x; s0s[1] = v0.y; s0s[2] = v1.x; s0s[3] = v1.y;
+            s1s[0] = v2.x; s1s[1] = v2.y; s1s[2] = v3.x; s1s[3] = v3.y;
+        }
+    } else if constexpr (!PARTIALS) {
         if constexpr (SPP == 4) {
             s0s[0] = *reinterpret_cast<const float *>(sc0);
             s1s[0] = *reinterpret_cast<const float *>(sc1);
@@ -228,7 +251,7 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
 // fully unrolled cell loop (slot and operand offsets are immediates), no
 // divisions and no 64-bit multiplies per cell.  Warps do not meet before the
 // final sum over the K-lanes.
-template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS>
+template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS, bool H16 = false>
 __global__ void __launch_bounds__(kDecodeThreads, W2A8_MINB(MT))
 w2a8_decode_kernel(const DecodeParams p) {
     constexpr int KS = kDecodeWarps / TG;
@@ -278,16 +301,34 @@ w2a8_decode_kernel(const DecodeParams p) {
     const uint32_t *wrow1 = wrow0 + (size_t)8 * p.words_per_row;
     // first scale of block kb0 in row n0 + (lane & 15)
     const float *srow = nullptr;
+    const unsigned short *srow_h = nullptr;          // the same place when the scales are binary16
     if constexpr (!PARTIALS) {
-        srow = p.w_scale + (size_t)(n0 + (lane & 15)) * p.G;
-        if constexpr (SPP != 4) srow += SPB * kb0;
+        const size_t first = (size_t)(n0 + (lane & 15)) * p.G + (SPP != 4 ? SPB * kb0 : 0);
+        if constexpr (H16) srow_h = reinterpret_cast<const unsigned short *>(p.w_scale) + first;
+        else               srow = p.w_scale + first;
     }
+    // binary16 scales that cannot be copied as one aligned unit (odd row pitch, or one scale per
+    // cell): loaded and stored by the lane itself -- slower, and rare
+    auto copy_scales_h = [&](int c, int first, int count) {
+        unsigned short *dst = reinterpret_cast<unsigned short *>(sslots + c * kScaleBytes + (lane & 15) * 16);
+        for (int i = 0; i < count; ++i) dst[i] = __ldg(srow_h + first + i);
+    };
     auto post_cell = [&](int c) {   // c is a constant after unrolling
         cp_async16(wslots_u32 + c * kSlotBytes, wrow0 + c * 16);
         cp_async16(wslots_u32 + c * kSlotBytes + 32 * 16, wrow1 + c * 16);
         if constexpr (!PARTIALS) {
             if (lane < 16) {
-                if constexpr (SPP == 4) {
+                if constexpr (H16) {
+                    if constexpr (SPP == 4) {
+                        const int kb = kb0 + c;
+                        copy_scales_h(c, p.blocks_per_group >= p.blocks ? 0 : kb / p.blocks_per_group, 1);
+                    } else if (p.s_vec) {
+                        if constexpr (SPP == 1) cp_async8(sslot_u32 + c * kScaleBytes, srow_h + c * SPB);
+                        else                    cp_async4(sslot_u32 + c * kScaleBytes, srow_h + c * SPB);
+                    } else {
+                        copy_scales_h(c, c * SPB, SPB);
+                    }
+                } else if constexpr (SPP == 4) {
                     const int kb = kb0 + c;
                     const int gi = p.blocks_per_group >= p.blocks ? 0 : kb / p.blocks_per_group;
                     cp_async4(sslot_u32 + c * kScaleBytes, srow + gi);
@@ -328,7 +369,14 @@ w2a8_decode_kernel(const DecodeParams p) {
             *reinterpret_cast<uint4 *>(wslots + tail_cell * kSlotBytes + r * (32 * 16)) = v;
         }
         if constexpr (!PARTIALS) {
-            if (lane < 16) {
+            if (lane < 16 && H16) {
+                if constexpr (SPP == 4) {
+                    const int kb = kb0 + tail_cell;
+                    copy_scales_h(tail_cell, p.blocks_per_group >= p.blocks ? 0 : kb / p.blocks_per_group, 1);
+                } else {
+                    copy_scales_h(tail_cell, tail_cell * SPB, (R + SPP - 1) / SPP);
+                }
+            } else if (lane < 16) {
                 float *dst = reinterpret_cast<float *>(sslots + tail_cell * kScaleBytes + lane * 16);
                 if constexpr (SPP == 4) {
                     const int kb = kb0 + tail_cell;
@@ -372,7 +420,7 @@ w2a8_decode_kernel(const DecodeParams p) {
             const int8_t *bc[MT];
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + c * kBlockK;
-            compute_cell<MT, SPP, ONE, PARTIALS, true>(p, w0s, w1s, sc0 + c * kScaleBytes, sc1 + c * kScaleBytes,
+            compute_cell<MT, SPP, ONE, PARTIALS, true, H16>(p, w0s, w1s, sc0 + c * kScaleBytes, sc1 + c * kScaleBytes,
                                                        bc, kb0 + c, n0, m0, gq, t, acc);
         }
     }
@@ -385,7 +433,7 @@ w2a8_decode_kernel(const DecodeParams p) {
         const int8_t *bc[MT];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + (size_t)tail_cell * kBlockK;
-        compute_cell<MT, SPP, ONE, PARTIALS, false>(p, w0s, w1s, sc0 + tail_cell * kScaleBytes,
+        compute_cell<MT, SPP, ONE, PARTIALS, false, H16>(p, w0s, w1s, sc0 + tail_cell * kScaleBytes,
                                                     sc1 + tail_cell * kScaleBytes, bc, kb0 + tail_cell,
                                                     n0, m0, gq, t, acc);
     }
@@ -436,11 +484,22 @@ w2a8_decode_kernel(const DecodeParams p) {
             return v;
         };
 
+        // final value of y[mm][nn]: fp32, or (16-bit instances, on request) rounded to bf16
+        auto store_y = [&](int mm, int nn, float v) {
+            v *= p.a_scale[mm] * (1.0f / kCodeGain);
+            if constexpr (H16) {
+                if (p.y16) {
+                    reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)mm * p.N + nn] = __float2bfloat16_rn(v);
+                    return;
+                }
+            }
+            p.y[(size_t)mm * p.N + nn] = v;
+        };
+
         if (p.chunks == 1) {
             for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
                 int mm, nn;
-                if (locate(e, mm, nn))
-                    p.y[(size_t)mm * p.N + nn] = cta_sum(e) * (p.a_scale[mm] * (1.0f / kCodeGain));
+                if (locate(e, mm, nn)) store_y(mm, nn, cta_sum(e));
             }
             W2A8_TRACE_POINT(6);
         } else if (p.cluster) {
@@ -462,7 +521,7 @@ w2a8_decode_kernel(const DecodeParams p) {
                 if (locate(e, mm, nn)) {
                     float v = 0.f;
                     for (int ch = 0; ch < p.chunks; ++ch) v += recv[ch * kElems + e];
-                    p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
+                    store_y(mm, nn, v);
                 }
             }
             W2A8_TRACE_POINT(7);
@@ -486,7 +545,7 @@ w2a8_decode_kernel(const DecodeParams p) {
                 if (locate(e, mm, nn)) {
                     float v = 0.f;
                     for (int ch = 0; ch < p.chunks; ++ch) v += __ldcg(p.ws + ch * MN + (size_t)mm * p.N + nn);
-                    p.y[(size_t)mm * p.N + nn] = v * (p.a_scale[mm] * (1.0f / kCodeGain));
+                    store_y(mm, nn, v);
                 }
             }
             if (threadIdx.x == 0) *counter = 0u;   // leave the workspace reusable
@@ -516,14 +575,15 @@ struct DecodePlan {
 // Launch plan for slabs of 8 * mt tokens.  One tile per CTA, its four warps take equal
 // runs of consecutive blocks of K (shortest serial work per warp).  K-chunks are added when a warp would
 // otherwise have more cells than landing slots, or when the grid would leave most SMs idle.
-static DecodePlan decode_plan_mt(int M, int N, int K, const ShapeInfo &si, int mt) {
+static DecodePlan decode_plan_mt(int M, int N, int K, const ShapeInfo &si, int mt, bool h16 = false) {
     DecodePlan pl;
     pl.mt = mt;
     pl.slabs = (M + 8 * pl.mt - 1) / (8 * pl.mt);
     const int ntiles = N / 16;
-    const int forced_tg = env_int("W2A8_TG", 0);
+    // the 16-bit instances exist for the default tile grouping and slot count only
+    const int forced_tg = h16 ? 0 : env_int("W2A8_TG", 0);
     pl.tg = (forced_tg == 1 || forced_tg == 2) ? forced_tg : 1;
-    { const int r = env_int("W2A8_RING", 0); pl.ring = (r == 4 || r == 8) ? r : kRound; }
+    { const int r = h16 ? 0 : env_int("W2A8_RING", 0); pl.ring = (r == 4 || r == 8) ? r : kRound; }
     const int ks = kDecodeWarps / pl.tg;
     const int forced = env_int("W2A8_CHUNKS", 0);
     int chunks = 1;
@@ -564,15 +624,15 @@ static DecodePlan decode_plan_mt(int M, int N, int K, const ShapeInfo &si, int m
 // once (8 CTAs per SM) -- measured faster on the small matrices of a layer (k/v, q/o), whose
 // grids are far from filling the GPU with wider slabs; otherwise the widest slab that covers M,
 // up to 32 tokens.  W2A8_MT forces a width.
-static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si) {
+static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si, bool h16 = false) {
     const int forced = env_int("W2A8_MT", 0);
-    if (forced >= 1 && forced <= 4) return decode_plan_mt(M, N, K, si, forced);
+    if (forced >= 1 && forced <= 4) return decode_plan_mt(M, N, K, si, forced, h16);
     const int widest = M > 32 ? 4 : (M + 7) / 8;
-    if (widest == 1) return decode_plan_mt(M, N, K, si, 1);
+    if (widest == 1) return decode_plan_mt(M, N, K, si, 1, h16);
     constexpr long long kResidentCtas = 148 * 8;
-    const DecodePlan narrow = decode_plan_mt(M, N, K, si, 1);
+    const DecodePlan narrow = decode_plan_mt(M, N, K, si, 1, h16);
     if ((long long)narrow.groups * narrow.chunks * narrow.slabs <= kResidentCtas) return narrow;
-    return decode_plan_mt(M, N, K, si, widest);
+    return decode_plan_mt(M, N, K, si, widest, h16);
 }
 
 constexpr size_t kStatusBytes = 256;   // workspace header: status word
@@ -615,6 +675,21 @@ static cudaError_t launch_decode_inst(const DecodeParams &p, int ring, dim3 grid
     return launch_decode_ring<MT, SPP, TG, kRound, ONE, PARTIALS>(p, grid, smem, st);
 }
 
+// 16-bit instances (binary16 scales, fp32 or bf16 result): default tile grouping and slot count.
+template <int MT, int SPP, bool ONE>
+static cudaError_t launch_decode_h16(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, true>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    return launch_kernel_cluster(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, true>, grid,
+                                 dim3(kDecodeThreads), smem, st, pdl_enabled(),
+                                 p.cluster ? (unsigned)p.chunks : 1u, p);
+}
+
 template <int MT, int SPP, int TG>
 static cudaError_t launch_decode_tg(const DecodeParams &p, int ring, bool want_partials, dim3 grid, size_t smem,
                                     cudaStream_t st) {
@@ -627,6 +702,10 @@ template <int MT, int SPP>
 static cudaError_t launch_decode_mt(const DecodeParams &p, const DecodePlan &pl, bool want_partials,
                                     cudaStream_t st) {
     dim3 grid(pl.groups, pl.chunks, pl.slabs);
+    if (p.h16) {
+        if (MT == 1 && p.M == 1) return launch_decode_h16<1, SPP, true>(p, grid, pl.smem, st);
+        return launch_decode_h16<MT, SPP, false>(p, grid, pl.smem, st);
+    }
     if (pl.tg == 1) return launch_decode_tg<MT, SPP, 1>(p, pl.ring, want_partials, grid, pl.smem, st);
     return launch_decode_tg<MT, SPP, 2>(p, pl.ring, want_partials, grid, pl.smem, st);
 }
@@ -642,14 +721,16 @@ static cudaError_t launch_decode_spp(const DecodeParams &p, const DecodePlan &pl
     }
 }
 
-// Enqueue the decode kernel.  `partials` != nullptr selects the parity export.
+// Enqueue the decode kernel.  `partials` != nullptr selects the parity export.  h16: w_scale
+// points at binary16 values; y16 (with h16 only): y points at bf16 values.
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
-                  const float *w_scale, float *y, int32_t *partials, int M, int N, int K,
-                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st) {
-    const DecodePlan pl = decode_plan(M, N, K, si);
+                  const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
+                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16) {
+    if (h16 && partials) return W2A8_ERR_SHAPE;
+    const DecodePlan pl = decode_plan(M, N, K, si, h16);
     DecodeParams p;
-    p.a = a; p.a_scale = a_scale; p.packed = packed; p.w_scale = w_scale;
-    p.y = y; p.partials = partials;
+    p.a = a; p.a_scale = a_scale; p.packed = packed; p.w_scale = reinterpret_cast<const float *>(w_scale);
+    p.y = reinterpret_cast<float *>(y); p.partials = partials; p.h16 = h16 ? 1 : 0; p.y16 = (h16 && y16) ? 1 : 0;
     p.M = M; p.N = N; p.K = K; p.G = si.G; p.group = group;
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
     p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;

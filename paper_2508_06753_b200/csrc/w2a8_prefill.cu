@@ -26,6 +26,8 @@
 // drain warps store y.  Every wait on an mbarrier is bounded; a wait that gives up
 // sets the status word of the workspace and the CTA winds down.
 #include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "w2a8_common.cuh"
 
@@ -55,6 +57,7 @@ struct PrefillParams {
     int M, N, K, G, group;
     int words_per_row;
     int slices_per_group;    // group / 64
+    int y16;                 // 16-bit instance only: y holds bf16 instead of fp32
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------
@@ -186,7 +189,8 @@ extern "C" int w2a8_debug_set_prefill_trace(void *buffer) {
 #define PF_TRACE(role, idx, point) do { } while (0)
 #endif
 
-template <bool PARTIALS>
+// H16: w_scale points at IEEE binary16 values; the result is fp32 or, with p.y16, bf16.
+template <bool PARTIALS, bool H16>
 __global__ void __launch_bounds__(kPfThreads, 1)
 w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillParams p) {
     extern __shared__ unsigned char pf_smem_raw[];
@@ -373,9 +377,14 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             // Scales are fetched eight groups ahead (a drain takes a few hundred cycles, a
             // global load several hundred): a ring of eight, refilled once per eight groups.
             const float *sc_row = PARTIALS ? nullptr : p.w_scale + (size_t)n * p.G;
+            const __half *sc_row_h = reinterpret_cast<const __half *>(p.w_scale) + (size_t)n * p.G;
+            auto ld_scale = [&](int gi) -> float {
+                if constexpr (H16) return __half2float(__ldg(sc_row_h + gi));
+                else               return __ldg(sc_row + gi);
+            };
             float sc_nxt[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) sc_nxt[u] = (!PARTIALS && u < ngroups) ? __ldg(sc_row + u) : 0.f;
+            for (int u = 0; u < 8; ++u) sc_nxt[u] = (!PARTIALS && u < ngroups) ? ld_scale(u) : 0.f;
             // Software pipeline over 32-column halves: while one half is converted and
             // accumulated, the next half (possibly of the next group) is on its way from TMEM.
             int v0[32], v1[32];                         // first / second half of the current group
@@ -386,7 +395,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     sc_cur[u] = sc_nxt[u];
-                    sc_nxt[u] = (!PARTIALS && g0 + 8 + u < ngroups) ? __ldg(sc_row + g0 + 8 + u) : 0.f;
+                    sc_nxt[u] = (!PARTIALS && g0 + 8 + u < ngroups) ? ld_scale(g0 + 8 + u) : 0.f;
                 }
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
@@ -445,7 +454,11 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
 #pragma unroll
                 for (int j = 0; j < kPfDrainCols; ++j) {
                     const int m = m0 + col0 + j;
-                    if (m < p.M) p.y[(size_t)m * p.N + n] = acc[j] * (__ldg(p.a_scale + m) * (1.0f / kCodeGain));
+                    if (m < p.M) {
+                        const float v = acc[j] * (__ldg(p.a_scale + m) * (1.0f / kCodeGain));
+                        if (H16 && p.y16) reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)m * p.N + n] = __float2bfloat16_rn(v);
+                        else              p.y[(size_t)m * p.N + n] = v;
+                    }
                 }
             }
         }
@@ -488,9 +501,10 @@ bool prefill_supported(int M, int N, int K, int group) {
 }
 
 // Enqueue the prefill kernel.  `partials` != nullptr selects the parity export.
-int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const float *w_scale,
-                   float *y, int32_t *partials, int M, int N, int K, int group, int *status,
-                   cudaStream_t st) {
+int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
+                   void *y, int32_t *partials, int M, int N, int K, int group, int *status,
+                   cudaStream_t st, bool h16, bool y16) {
+    if (h16 && partials) return W2A8_ERR_SHAPE;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return W2A8_ERR_CUDA;
     CUtensorMap map;
@@ -503,7 +517,8 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return W2A8_ERR_CUDA;
     PrefillParams p;
-    p.packed = packed; p.w_scale = w_scale; p.a_scale = a_scale; p.y = y; p.partials = partials;
+    p.packed = packed; p.w_scale = reinterpret_cast<const float *>(w_scale); p.a_scale = a_scale;
+    p.y = reinterpret_cast<float *>(y); p.partials = partials; p.y16 = (h16 && y16) ? 1 : 0;
     p.status = status;
     p.M = M; p.N = N; p.K = K; p.G = K / group; p.group = group;
     p.words_per_row = K / 16;
@@ -518,23 +533,20 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
     }
     const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
     dim3 grid((unsigned)(tiles < sm_count ? tiles : sm_count));   // persistent CTAs, one per SM
-    static bool configured[2] = {false, false};
-    cudaError_t e;
-    if (partials) {
-        if (!configured[1]) {
-            e = cudaFuncSetAttribute(w2a8_prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return W2A8_ERR_CUDA;
-            configured[1] = true;
+    static bool configured[3] = {false, false, false};
+    auto launch = [&](auto kernel, int slot) -> bool {
+        if (!configured[slot]) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+                return false;
+            configured[slot] = true;
         }
-        w2a8_prefill_kernel<true><<<grid, kPfThreads, smem, st>>>(map, p);
-    } else {
-        if (!configured[0]) {
-            e = cudaFuncSetAttribute(w2a8_prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return W2A8_ERR_CUDA;
-            configured[0] = true;
-        }
-        w2a8_prefill_kernel<false><<<grid, kPfThreads, smem, st>>>(map, p);
-    }
+        kernel<<<grid, kPfThreads, smem, st>>>(map, p);
+        return true;
+    };
+    const bool launched = partials ? launch(w2a8_prefill_kernel<true, false>, 1)
+                        : h16      ? launch(w2a8_prefill_kernel<false, true>, 2)
+                                   : launch(w2a8_prefill_kernel<false, false>, 0);
+    if (!launched) return W2A8_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
 

@@ -1,0 +1,140 @@
+"""GPU parity of the 16-bit recipe (binary16 weight scales, fp32 or bf16 result) against the CPU
+reference: fp32 results within 1e-4 * max|row|; bf16 results bit-equal to the round-to-nearest-even
+of the fp32 result the same kernel produces, and within one bf16 step of the reference's bf16 where
+the two fp32 values straddle a rounding boundary."""
+import numpy as np
+import pytest
+
+from paper_2508_06753_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2508_06753_b200 import binding, build
+    build.build()
+    binding.lib()
+    return torch, binding
+
+
+def _dev(torch, arr):
+    return torch.from_numpy(np.ascontiguousarray(arr)).cuda()
+
+
+def _bf16_dev(torch, bits):
+    return _dev(torch, bits.view(np.int16)).view(torch.bfloat16)
+
+
+def _bf16_bits_to_f64(bits):
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def _check(torch, b, oracle, M, N, K, group, seed, ternary=False, frac=0.0, sel=None):
+    g = K if group == 0 else group
+    codes = synth.weight_codes(seed, N, K, ternary)
+    s_h = synth.weight_scales_h(seed, N, K // g)
+    bits = synth.activations_bf16(seed, M, K, frac)
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_bf16_dev(torch, bits))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    s_h_dev = _dev(torch, s_h.view(np.int16)).view(torch.float16)
+    y32 = b.w2a8_gemm_h16(a, s_a, packed, s_h_dev, g, ws)
+    y16 = b.w2a8_gemm_h16(a, s_a, packed, s_h_dev, g, ws, out_dtype=torch.bfloat16)
+    # the fp32-scale entry on the widened scales: the same arithmetic, so the same bits
+    y_wide = b.w2a8_gemm(a, s_a, packed, s_h_dev.float(), g, ws)
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    assert y16.dtype == torch.bfloat16 and y32.dtype == torch.float32
+    assert torch.equal(y32, y_wide), "binary16 scales must give the bits of the widened fp32 scales"
+    assert torch.equal(y16, y32.to(torch.bfloat16)), "bf16 result must be the RNE rounding of the fp32 result"
+
+    a_ref, s_ref = oracle.quantize(bits)
+    assert np.array_equal(a.cpu().numpy(), a_ref)
+    if sel is None:
+        sel = np.arange(N)
+    r32, r16 = oracle.gemm_h(a_ref, s_ref, codes[sel], s_h[sel], g)
+    got32 = y32.cpu().numpy()[:, sel]
+    rowmax = np.abs(r32).max(axis=1)
+    err = np.abs(got32.astype(np.float64) - r32.astype(np.float64)).max(axis=1)
+    assert (err <= TOL * rowmax).all(), float((err / np.maximum(TOL * rowmax, 1e-30)).max())
+    got16 = y16.view(torch.int16).cpu().numpy().view(np.uint16)[:, sel]
+    d = np.abs(_bf16_bits_to_f64(got16) - _bf16_bits_to_f64(r16))
+    step = np.abs(_bf16_bits_to_f64(r16)) * 2.0 ** -7          # >= one bf16 step at that magnitude
+    assert (d <= step + TOL * rowmax[:, None]).all()
+    assert (got16 == r16).mean() >= 0.98                       # straddled boundaries are rare
+    return y32
+
+
+CASES = [
+    # M, N, K, group (0 = K), ternary, outlier fraction
+    (1, 16, 64, 64, False, 0.0),            # smallest legal problem
+    (1, 2048, 2048, 128, False, 0.0),       # the recipe's group
+    (3, 48, 448, 64, False, 0.0),           # ragged K, odd number of groups per row (no vector copies)
+    (1, 1600, 1600, 64, False, 0.0),        # ragged K, 25 groups per row
+    (2, 64, 2176, 128, False, 0.0),         # 17 groups per row, trailing block of two slices
+    (5, 32, 1600, 0, True, 0.0),            # one scale per channel, ragged K
+    (4, 1040, 4096, 64, False, 0.0),
+    (8, 256, 4096, 128, True, 0.01),
+    (9, 256, 2048, 128, False, 0.0),        # two 8-token slabs
+    (16, 512, 4096, 128, False, 0.0),
+    (17, 128, 1024, 256, False, 0.0),       # one scale per block
+    (32, 256, 8192, 128, False, 0.01),
+    (1, 256, 8192, 128, True, 0.0),         # split-K inside a cluster
+    (1, 16, 28672, 128, False, 0.01),       # longest K of any configuration
+    (33, 64, 512, 64, False, 0.0),
+    (64, 128, 256, 0, False, 0.0),          # tensor-core kernel, smallest tile grid
+    (128, 256, 512, 128, False, 0.0),       # tensor-core kernel
+    (200, 384, 768, 64, False, 0.01),       # tensor-core kernel, ragged token tile
+    (70, 48, 768, 128, False, 0.0),         # many tokens, shape the tensor-core kernel does not tile
+]
+
+
+@pytest.mark.parametrize("M,N,K,group,ternary,frac", CASES)
+def test_h16_against_reference(gpu, oracle, M, N, K, group, ternary, frac):
+    torch, b = gpu
+    _check(torch, b, oracle, M, N, K, group, seed=M * 37 + N + K, ternary=ternary, frac=frac)
+
+
+@pytest.mark.parametrize("chunks", [2, 5, 59])
+@pytest.mark.parametrize("M,group", [(1, 128), (12, 64), (20, 0)])
+def test_h16_forced_chunking(gpu, oracle, chunks, M, group, monkeypatch):
+    """Split-K through clusters (few chunks) and through the workspace (many)."""
+    torch, b = gpu
+    monkeypatch.setenv("W2A8_CHUNKS", str(chunks))
+    _check(torch, b, oracle, M, 80, 14336 + 256 * 3, group, seed=chunks + M)
+
+
+@pytest.mark.parametrize("M", [1, 16, 2048])
+def test_h16_full_size_gate_sampled(gpu, oracle, M):
+    """The largest linear of the 8B layer with the recipe's group of 128, in the launch
+    configuration the benchmark's 16-bit probe times; reference on sampled channels."""
+    torch, b = gpu
+    K, N = 4096, 14336
+    rng = np.random.default_rng(23)
+    sel = np.unique(np.concatenate([np.arange(16), np.arange(N - 16, N), rng.choice(N, size=32, replace=False)]))
+    y = _check(torch, b, oracle, M, N, K, 128, seed=91 + M, ternary=True, sel=sel)
+    assert torch.isfinite(y).all()
+
+
+def test_h16_argument_errors(gpu):
+    torch, b = gpu
+    M, N, K, g = 2, 32, 256, 64
+    a = torch.zeros((M, K), dtype=torch.int8, device="cuda")
+    s_a = torch.ones((M,), dtype=torch.float32, device="cuda")
+    packed = torch.zeros((N, K // 16), dtype=torch.int32, device="cuda")
+    s_h = torch.ones((N, K // g + 8), dtype=torch.float16, device="cuda")
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    with pytest.raises(TypeError):
+        b.w2a8_gemm_h16(a, s_a, packed, s_h.float(), g, ws)
+    with pytest.raises(b.W2A8Error):                                   # scales not 16-byte aligned
+        b.w2a8_gemm_h16(a, s_a, packed, s_h.view(-1)[1:1 + N * (K // g)].view(N, K // g), g, ws)
+    with pytest.raises(b.W2A8Error):                                   # group does not divide K
+        b.w2a8_gemm_h16(a, s_a, packed, s_h, 96, ws)
+    with pytest.raises(b.W2A8Error):                                   # workspace too small
+        b.w2a8_gemm_h16(a, s_a, packed, s_h, g, ws[:8])
+    torch.cuda.synchronize()
