@@ -377,14 +377,49 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             // Scales are fetched eight groups ahead (a drain takes a few hundred cycles, a
             // global load several hundred): a ring of eight, refilled once per eight groups.
             const float *sc_row = PARTIALS ? nullptr : p.w_scale + (size_t)n * p.G;
-            const __half *sc_row_h = reinterpret_cast<const __half *>(p.w_scale) + (size_t)n * p.G;
-            auto ld_scale = [&](int gi) -> float {
-                if constexpr (H16) return __half2float(__ldg(sc_row_h + gi));
-                else               return __ldg(sc_row + gi);
-            };
-            float sc_nxt[8];
+            const unsigned short *sc_row_h = reinterpret_cast<const unsigned short *>(p.w_scale) + (size_t)n * p.G;
+            // The ring holds what the loads return, untouched: any instruction that reads a
+            // loaded register makes the warp wait for that load.  fp32: eight values.  binary16:
+            // eight values widened when they are taken out -- fetched as one 16-byte load when the
+            // row pitch allows (G % 8 == 0: registers 0..3 hold two scales each), else as eight
+            // 16-bit loads into 32-bit registers.
+            const bool vec8 = H16 && (p.G % 8 == 0);
+            uint32_t sc_nxt[8];
+            auto refill = [&](int g0) {
+                if constexpr (PARTIALS) {
+                    return;
+                } else if constexpr (H16) {
+                    if (vec8) {
+                        if (g0 < ngroups) {
+                            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(sc_row_h + g0));
+                            sc_nxt[0] = v.x; sc_nxt[1] = v.y; sc_nxt[2] = v.z; sc_nxt[3] = v.w;
+                        }
+                    } else {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) sc_nxt[u] = (!PARTIALS && u < ngroups) ? ld_scale(u) : 0.f;
+                        for (int u = 0; u < 8; ++u)
+                            if (g0 + u < ngroups)
+                                asm volatile("ld.global.nc.u16 %0, [%1];" : "=r"(sc_nxt[u]) : "l"(sc_row_h + g0 + u));
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (g0 + u < ngroups) sc_nxt[u] = __float_as_uint(__ldg(sc_row + g0 + u));
+                }
+            };
+            auto take = [&](int u) -> float {          // u is a constant after unrolling
+                if constexpr (H16) {
+                    // one conversion that names the half of the register it reads
+                    const __half2 pair = *reinterpret_cast<const __half2 *>(&sc_nxt[u >> 1]);
+                    const __half2 lone = *reinterpret_cast<const __half2 *>(&sc_nxt[u]);
+                    if (vec8) return (u & 1) ? __high2float(pair) : __low2float(pair);
+                    return __low2float(lone);
+                } else {
+                    return __uint_as_float(sc_nxt[u]);
+                }
+            };
+#pragma unroll
+            for (int u = 0; u < 8; ++u) sc_nxt[u] = 0u;
+            refill(0);
             // Software pipeline over 32-column halves: while one half is converted and
             // accumulated, the next half (possibly of the next group) is on its way from TMEM.
             int v0[32], v1[32];                         // first / second half of the current group
@@ -394,9 +429,9 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 float sc_cur[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    sc_cur[u] = sc_nxt[u];
-                    sc_nxt[u] = (!PARTIALS && g0 + 8 + u < ngroups) ? ld_scale(g0 + 8 + u) : 0.f;
+                    sc_cur[u] = take(u);
                 }
+                refill(g0 + 8);
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const int gi = g0 + u;
