@@ -384,6 +384,77 @@ def concat_probe(rep, reps=200):
                     "GB/s uses the byte count of the 7-GEMM layer", "per_m": out}
 
 
+def recipe16_probe(rep, peaks, group=128, reps=200):
+    """Extra row (not the headline): the same layer stored the way the paper's end-to-end ternary
+    section describes -- groups of 128 along K, binary16 weight scales -- with bf16 results, through
+    w2a8_gemm_h16: 7 GEMMs + 4 a8_quantize per pass.  GB/s uses this recipe's own (smaller) byte
+    count: 2 + 16/128 bit per weight, 2 bytes per result."""
+    torch, b, cfg = rep.torch, rep.b, rep.cfg
+    dev = rep.ws.device
+
+    def bytes_of(M, N, K):
+        return K * N // 4 + (K // group) * N * 2 + M * K + 4 * M + 2 * M * N
+
+    copies = []
+    for c in range(len(rep.copies)):
+        mats = []
+        for idx, (name, K, N) in enumerate(rep.shapes):
+            if K % group:
+                return None
+            s_h = synth.weight_scales_h(synth.shape_seed(cfg, idx) + 100 * c, N, K // group)
+            mats.append((rep.copies[c][idx][0], torch.from_numpy(s_h.view(np.int16)).to(dev).view(torch.float16)))
+        copies.append(mats)
+    out = {}
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        for M in cfg["Ms"]:
+            bufs = rep.per_m[M]
+            ys = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _, _, N in rep.shapes]
+            ws = b.new_workspace(max(b.w2a8_workspace_bytes(M, N, K, group) for _, K, N in rep.shapes), device=dev)
+
+            def one_pass(c):
+                done = set()
+                for idx, (name, K, N) in enumerate(rep.shapes):
+                    inp = rep.input_of[name]
+                    if inp not in done:
+                        b.a8_quantize(bufs["x"][inp], bufs["a"][inp], bufs["s"][inp])
+                        done.add(inp)
+                    packed, s_h = copies[c][idx]
+                    b.w2a8_gemm_h16(bufs["a"][inp], bufs["s"][inp], packed, s_h, group, ws, ys[idx])
+            for c in range(len(copies)):
+                one_pass(c)
+            torch.cuda.synchronize()
+            try:
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=stream):
+                    for c in range(len(copies)):
+                        one_pass(c)
+                run = gr.replay
+            except Exception:
+                def run():
+                    for c in range(len(copies)):
+                        one_pass(c)
+            for _ in range(3):
+                run()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = max(reps // len(copies), 3)
+            e0.record()
+            for _ in range(n):
+                run()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / (n * len(copies))
+            nbytes = sum(bytes_of(M, N, K) for _, K, N in rep.shapes)
+            out[str(M)] = {"us_per_layer": ms * 1e3, "bytes_per_layer": nbytes,
+                           "gbs": nbytes / (ms * 1e-3) / 1e9,
+                           "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    torch.cuda.current_stream().wait_stream(stream)
+    return {"what": f"group {group}, binary16 weight scales, bf16 results (w2a8_gemm_h16): 7 GEMMs + 4 "
+                    "a8_quantize per layer pass; GB/s on this recipe's own byte count", "per_m": out}
+
+
 def e2e_measure(rep, steps, warmup):
     """Same workload through w2a8_linear_host: pinned host activations in, host
     outputs back, copies inside the timed region."""
@@ -571,6 +642,7 @@ def run_ours(args):
         for M in cfg["Ms"]:
             probes.append(kernel_probe(rep, M, big))
     concat = concat_probe(rep) if rank == 0 else None
+    recipe16 = recipe16_probe(rep, peaks) if rank == 0 else None
     prefill = None
     if rank == 0 and not args.no_prefill:
         prefill = prefill_probe(device, peaks)
@@ -613,6 +685,7 @@ def run_ours(args):
         "gpu_launches": args.steps * len(cfg["Ms"]) * rep.kernels_per_pass,
         "roofline": roofline, "roofline_by_m": roofline_by_m, "cpu_baseline": cpu, "per_m": per_m,
         "kernel_probes": probes, "concatenated_qkv_gateup": concat,
+        "recipe_g128_binary16_scales_bf16_out": recipe16,
         "prefill": prefill,
     }
     print(json.dumps(out))
