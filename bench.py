@@ -320,6 +320,61 @@ def kernel_probe(rep, M, shape_idx, reps=30):
                 distinct_weight_bytes=distinct, launches=reps * len(mats))
 
 
+def small_shape_probe(device, peaks, l2_bytes, reps=20):
+    """Extra rows (not the headline): the small square-ish matrices the paper also times (Sec. III:
+    1600x1600, 2560x2560, 3840x2560, 3200x3200), where launch latency dominates.  One GEMV (M = 1,
+    group 64) per launch, back to back in a CUDA graph over enough distinct weight copies to exceed
+    twice the L2."""
+    import torch
+    from paper_2508_06753_b200 import binding as b
+    rows = []
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    for K, N in ((1600, 1600), (2560, 2560), (2560, 3840), (3200, 3200)):
+        g, M = 64, 1
+        codes, s_w = synth.make_linear(K + N, K, N, g)
+        packed = b.w2_pack(torch.from_numpy(codes).to(device))
+        sw = torch.from_numpy(s_w).to(device)
+        per = packed.numel() * 4 + sw.numel() * 4
+        ncopy = int(np.ceil(2.2 * l2_bytes / per))
+        mats = [(packed.clone(), sw.clone()) for _ in range(ncopy)]
+        x = torch.from_numpy(synth.activations_bf16(K, M, K).view(np.int16)).to(device).view(torch.bfloat16)
+        a, s_a = b.a8_quantize(x)
+        y = torch.empty((M, N), dtype=torch.float32, device=device)
+        ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g), device=device)
+
+        def body():
+            for pk, sc in mats:
+                b.w2a8_gemm(a, s_a, pk, sc, g, ws, y)
+        with torch.cuda.stream(stream):
+            body()
+            torch.cuda.synchronize()
+            try:
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=stream):
+                    body()
+                run = gr.replay
+            except Exception:
+                run = body
+            for _ in range(3):
+                run()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                run()
+            e1.record()
+            torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (reps * ncopy)
+        nbytes = gemm_bytes(M, N, K, g)
+        rows.append({"shape": f"{K}x{N}", "M": M, "group": g, "us_per_launch": us, "bytes_per_launch": nbytes,
+                     "gbs": nbytes / us / 1e3, "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
+                     "weight_copies": ncopy})
+        del mats
+    torch.cuda.current_stream().wait_stream(stream)
+    return rows
+
+
 def concat_probe(rep, reps=200):
     """Extra row (not the headline): the same layer with q|k|v and gate|up concatenated along N,
     i.e. 4 GEMMs + 4 a8_quantize per pass instead of 7 + 4.  Packed rows are independent, so the
@@ -643,6 +698,7 @@ def run_ours(args):
             probes.append(kernel_probe(rep, M, big))
     concat = concat_probe(rep) if rank == 0 else None
     recipe16 = recipe16_probe(rep, peaks) if rank == 0 else None
+    small = small_shape_probe(device, peaks, l2) if rank == 0 else None
     prefill = None
     if rank == 0 and not args.no_prefill:
         prefill = prefill_probe(device, peaks)
@@ -686,6 +742,7 @@ def run_ours(args):
         "roofline": roofline, "roofline_by_m": roofline_by_m, "cpu_baseline": cpu, "per_m": per_m,
         "kernel_probes": probes, "concatenated_qkv_gateup": concat,
         "recipe_g128_binary16_scales_bf16_out": recipe16,
+        "paper_small_shapes_m1": small,
         "prefill": prefill,
     }
     print(json.dumps(out))

@@ -148,6 +148,9 @@ CASES = [
     (33, 64, 512, 64, False, 0.0),         # more than one 32-token chunk
     (70, 48, 768, 128, False, 0.0),
     (1, 16, 28672, 128, False, 0.01),      # longest K of any configuration
+    (1, 2560, 2560, 64, False, 0.0),       # the paper's other small shapes (Sec. III)
+    (1, 3840, 2560, 64, False, 0.0),
+    (4, 3200, 3200, 64, True, 0.0),
 ]
 
 
