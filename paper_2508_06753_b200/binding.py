@@ -76,8 +76,10 @@ def _check(status: int, where: str):
 
 
 def _stream(stream=None) -> int:
-    s = stream if stream is not None else torch.cuda.current_stream()
-    return int(s.cuda_stream)
+    if stream is not None:
+        return int(stream.cuda_stream)
+    # raw handle of the current stream of the current device, without building a Stream object
+    return int(torch._C._cuda_getCurrentRawStream(torch.cuda.current_device()))
 
 
 def _ptr(t) -> int:

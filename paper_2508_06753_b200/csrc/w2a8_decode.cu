@@ -624,7 +624,7 @@ static DecodePlan decode_plan_mt(int M, int N, int K, const ShapeInfo &si, int m
 // once (8 CTAs per SM) -- measured faster on the small matrices of a layer (k/v, q/o), whose
 // grids are far from filling the GPU with wider slabs; otherwise the widest slab that covers M,
 // up to 32 tokens.  W2A8_MT forces a width.
-static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si, bool h16 = false) {
+static DecodePlan decode_plan_uncached(int M, int N, int K, const ShapeInfo &si, bool h16) {
     const int forced = env_int("W2A8_MT", 0);
     if (forced >= 1 && forced <= 4) return decode_plan_mt(M, N, K, si, forced, h16);
     const int widest = M > 32 ? 4 : (M + 7) / 8;
@@ -633,6 +633,30 @@ static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si, bool h16
     const DecodePlan narrow = decode_plan_mt(M, N, K, si, 1, h16);
     if ((long long)narrow.groups * narrow.chunks * narrow.slabs <= kResidentCtas) return narrow;
     return decode_plan_mt(M, N, K, si, widest, h16);
+}
+
+// The plan depends on the shape and on the W2A8_* switches of the environment.  Every entry
+// point asks for it two to four times per call (workspace check, launch), and each evaluation
+// reads a dozen environment variables, so the last plan is kept per thread together with a
+// fingerprint of the environment block: the addresses of its strings (the C library makes a
+// new string whenever a variable is set to a new value, so any change moves the fingerprint).
+extern "C" char **environ;
+static uint64_t env_fingerprint() {
+    uint64_t h = 1469598103934665603ull;
+    for (char **e = environ; e && *e; ++e) h = (h ^ (uint64_t)(uintptr_t)*e) * 1099511628211ull;
+    return h;
+}
+
+static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si, bool h16 = false) {
+    struct Key { int M, N, K, G, h16; uint64_t env; };
+    thread_local Key key = {0, 0, 0, 0, 0, 0};
+    thread_local DecodePlan cached;
+    const uint64_t env = env_fingerprint();
+    if (key.M == M && key.N == N && key.K == K && key.G == si.G && key.h16 == (int)h16 && key.env == env)
+        return cached;
+    cached = decode_plan_uncached(M, N, K, si, h16);
+    key = {M, N, K, si.G, (int)h16, env};
+    return cached;
 }
 
 constexpr size_t kStatusBytes = 256;   // workspace header: status word
