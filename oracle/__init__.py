@@ -150,3 +150,18 @@ def gemm_h(a: np.ndarray, a_scale: np.ndarray, codes: np.ndarray, w_scale_h: np.
     _load().ref_gemm_h(_p(a), _p(a_scale), _p(codes), _p(w_scale_h), ctypes.c_int(M),
                        ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(g), _p(y32), _p(y16))
     return y32, y16
+
+
+def gemm_a16(x_bf16_bits: np.ndarray, codes: np.ndarray, w_scale: np.ndarray, g: int) -> np.ndarray:
+    """16-bit activations, no quantiser: fp32 y[M][N] = sum_k x[m][k] (q[n][k] - 2) s_w[n][k/g]
+    (double accumulation, rounded once).  x: bf16 bit patterns uint16 [M][K]."""
+    x = np.ascontiguousarray(x_bf16_bits, dtype=np.uint16)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    w_scale = np.ascontiguousarray(w_scale, dtype=np.float32)
+    M, K = x.shape
+    N = codes.shape[0]
+    assert codes.shape[1] == K and K % g == 0 and w_scale.shape == (N, K // g)
+    y = np.empty((M, N), dtype=np.float32)
+    _load().ref_gemm_a16(_p(x), _p(codes), _p(w_scale), ctypes.c_int(M), ctypes.c_int(N),
+                         ctypes.c_int(K), ctypes.c_int(g), _p(y))
+    return y

@@ -36,6 +36,11 @@
  *       the same sums as ref_gemm with each scale first widened exactly to
  *       fp32, and an optional bf16 result (round to nearest even of the
  *       fp32 result).
+ *   ref_gemm_a16 : the alternative kernel of Sec. II ("Alternative
+ *       implementation"): the 2-bit weights are used as 16-bit values against
+ *       16-bit activations, with no activation quantisation and no
+ *       dequantisation step: y = sum_k x[k] * (value[k] * scale[group of k]),
+ *       here with x in bf16 and the sum written group by group.
  *
  * Parity pins: every routine here is pinned by tests that do not reuse this
  * code (hand-written golden words, exhaustive exact-rational evaluation of
@@ -259,5 +264,31 @@ void ref_gemm_h(const int8_t *a, const float *a_scale, const uint8_t *codes,
             float r = (float)((double)a_scale[m] * acc);
             y32[(size_t)m * N + n] = r;
             if (y16) y16[(size_t)m * N + n] = ref_float_to_bf16(r);
+        }
+}
+
+/* ------------------------------------------- 16-bit activations, no quantiser */
+/*
+ * y[m][n] = fp32( sum_gi w_scale[n][gi] * sum_{k in gi} x[m][k] * (q[n][k] - 2) ),
+ * x given as bf16 bit patterns, everything carried in double in index order
+ * (every product x * (q - 2) is exact in double, and so is its product with
+ * nothing else until the scale).
+ * x: [M][K] bf16 bits; codes: [N][K]; w_scale: [N][K/g] fp32; y: [M][N] fp32.
+ */
+void ref_gemm_a16(const uint16_t *x, const uint8_t *codes, const float *w_scale,
+                  int M, int N, int K, int g, float *y) {
+    int G = K / g;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int m = 0; m < M; ++m) {
+            double acc = 0.0;
+            for (int gi = 0; gi < G; ++gi) {
+                double p = 0.0;
+                for (int k = gi * g; k < (gi + 1) * g; ++k)
+                    p += (double)bf16_to_float(x[(size_t)m * K + k]) *
+                         (double)((int)(codes[(size_t)n * K + k] & 3) - 2);
+                acc += (double)w_scale[(size_t)n * G + gi] * p;
+            }
+            y[(size_t)m * N + n] = (float)acc;
         }
 }
