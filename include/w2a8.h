@@ -156,6 +156,34 @@ int w2a8_gemm_h16(const int8_t* a, const float* a_scale, const uint32_t* packed,
                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The alternative kernel of Sec. II ("Alternative implementation"): the 2-bit
+ * weights are turned into 16-bit values and multiplied with 16-bit
+ * activations, so the activations are not quantised and no dequantisation
+ * follows:
+ *
+ *   y[m][n] = sum_gi w_scale[n][gi] * sum_{k in group gi} x[m][k] * (q[n][k] - 2)
+ *
+ *   x_bf16   device, [M][K] bf16, row-major, 16-byte aligned
+ *   packed, w_scale, y (fp32 [M][N]), shapes, group, workspace (sized by
+ *   w2a8_workspace_bytes), stream, error codes, asynchronous completion:
+ *   as for w2a8_gemm.  No a8_quantize call is needed before it.
+ *
+ * Arithmetic: the codes become the bf16 values q - 2 (exact), every product
+ * with a bf16 activation is exact in fp32, and the products of one scale group
+ * are summed in fp32 by the tensor core (`mma.sync` bf16, fp32 accumulate; the
+ * order inside the instruction is the hardware's); each group sum is then
+ * multiplied by its fp32 scale and added in fp32.  Where the paper folds the
+ * scale into the 16-bit weight (exact only for ternary codes and a 16-bit
+ * scale), this build applies it to the group sum, which is exact for all four
+ * code values and keeps fp32 scales.  The result differs from the exact sum by
+ * fp32 summation error only (of the order sqrt(K) * 2^-24 relative to the
+ * magnitude of the terms).  The streaming kernel serves every M (there is no
+ * tensor-memory variant of this entry); it is meant for few tokens.
+ */
+int w2a16_gemm(const void* x_bf16, const uint32_t* packed, const float* w_scale, float* y,
+               int M, int N, int K, int group, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * w2a8_gemm_partials -- parity/debug export of the exact int32 per-group sums
  * P[m][n][gi] computed by the same inner-product code as w2a8_gemm.
  *   partials [M][N][K/group] int32, fully overwritten.

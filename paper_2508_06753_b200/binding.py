@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libw2a8.so")
 EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
-    "w2a8_gemm_h16", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
+    "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
 ]
 
 _lib = None
@@ -53,6 +53,7 @@ def lib() -> ctypes.CDLL:
         L.w2a8_workspace_status.argtypes = [vp, vp]
         L.w2a8_gemm.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_h16.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp, sz, vp]
+        L.w2a16_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_partials.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear_host_workspace_bytes.restype = sz
@@ -171,6 +172,20 @@ def w2a8_gemm_h16(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor, 
                                1 if y.dtype == torch.bfloat16 else 0, M, N, K, group, _ptr(workspace),
                                workspace.numel() * workspace.element_size(), _stream(stream)),
            "w2a8_gemm_h16")
+    return y
+
+
+def w2a16_gemm(x: torch.Tensor, packed: torch.Tensor, w_scale: torch.Tensor, group: int,
+               workspace: torch.Tensor, y: torch.Tensor | None = None, stream=None):
+    """bf16 x [M][K] (device, not quantised) -> y fp32 [M][N]; see w2a16_gemm in include/w2a8.h."""
+    M, K = x.shape
+    N = packed.shape[0]
+    if x.dtype != torch.bfloat16:
+        raise TypeError("x must be bfloat16")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    _check(lib().w2a16_gemm(_ptr(x), _ptr(packed), _ptr(w_scale), _ptr(y), M, N, K, group, _ptr(workspace),
+                            workspace.numel() * workspace.element_size(), _stream(stream)), "w2a16_gemm")
     return y
 
 

@@ -9,7 +9,8 @@ namespace w2a8 {
 
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
-                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16);
+                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16,
+                  bool a16);
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
 
 bool prefill_supported(int M, int N, int K, int group);
@@ -282,7 +283,7 @@ int w2a8_workspace_status(const void *workspace, void *stream) {
 static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *packed,
                        const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
                        int group, void *workspace, size_t workspace_bytes, void *stream,
-                       bool h16 = false, bool y16 = false) {
+                       bool h16 = false, bool y16 = false, bool a16 = false) {
     ShapeInfo si;
     if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
     if (!aligned16(a) || !aligned16(packed) || (y && !aligned16(y)) ||
@@ -293,11 +294,18 @@ static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *pa
     if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
     if (int st = check_device()) return st;
     // many tokens: tensor-core path (tcgen05); few tokens, or shapes it does not tile: streaming path
-    if (prefill_supported(M, N, K, group) && env_int("W2A8_PREFILL", 1) != 0)
+    if (!a16 && prefill_supported(M, N, K, group) && env_int("W2A8_PREFILL", 1) != 0)
         return launch_prefill(a, a_scale, packed, w_scale, y, partials, M, N, K, group,
                               reinterpret_cast<int *>(workspace), (cudaStream_t)stream, h16, y16);
     return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,
-                         (cudaStream_t)stream, h16, y16);
+                         (cudaStream_t)stream, h16, y16, a16);
+}
+
+int w2a16_gemm(const void *x_bf16, const uint32_t *packed, const float *w_scale, float *y, int M, int N,
+               int K, int group, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!x_bf16 || !packed || !w_scale || !y) return W2A8_ERR_NULL;
+    return gemm_common(reinterpret_cast<const int8_t *>(x_bf16), nullptr, packed, w_scale, y, nullptr, M, N, K,
+                       group, workspace, workspace_bytes, stream, false, false, true);
 }
 
 int w2a8_gemm_h16(const int8_t *a, const float *a_scale, const uint32_t *packed,

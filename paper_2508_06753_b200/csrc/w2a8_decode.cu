@@ -69,6 +69,7 @@ struct DecodeParams {
     int blocks_per_group; // 256-k blocks per scale group (groups of 256 and more)
     int s_vec;            // the scales of a cell and channel can be copied as one unit (16/8 B fp32, 8/4 B binary16)
     int h16;              // w_scale holds IEEE binary16 values (16-bit instances)
+    int a16;              // a holds bf16 activations, a_scale is unused (16-bit-activation instances)
     int y16;              // 16-bit instances only: y holds bf16 instead of fp32
 };
 
@@ -241,6 +242,84 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
     }
 }
 
+// The same cell for 16-bit activations and no activation quantiser (the alternative kernel of
+// Sec. II): the codes become the bf16 values q - 2 (exact), the activations are the caller's
+// bf16 values as they are, and the products are summed in fp32 by `mma.sync.m16n8k16`; the
+// group scale multiplies the fp32 sum of its group.
+// A lane's word of a slice holds code l (k = 16 t + l of the slice) at bits 8 (l mod 4) +
+// 2 (l div 4); MMA j of the slice takes l = 4 j .. 4 j + 3: after a shift by 2 j the four codes
+// sit in the four bytes.  0x4300 | q is the bf16 value 128 + q, so a byte permute with 0x43 and
+// one packed subtraction of 130 give the two bf16 weights of a register.
+// brow[mt]: this lane's 32 activation bytes (16 bf16) of slice 0, token row of slab mt.
+template <int MT, int SPP, bool ONE, bool FULL>
+__device__ __forceinline__ void compute_cell_a16(const DecodeParams &p, const uint32_t (&w0s)[4],
+                                                 const uint32_t (&w1s)[4], const unsigned char *sc0,
+                                                 const unsigned char *sc1,
+                                                 const int8_t *const (&brow)[MT], float (&acc)[MT][4]) {
+    const int R = FULL ? 4 : p.tail_slices;
+    float s0s[4 / SPP], s1s[4 / SPP];
+    if constexpr (SPP == 4) {
+        s0s[0] = *reinterpret_cast<const float *>(sc0);
+        s1s[0] = *reinterpret_cast<const float *>(sc1);
+    } else if constexpr (SPP == 2) {
+        const float2 v0 = *reinterpret_cast<const float2 *>(sc0);
+        const float2 v1 = *reinterpret_cast<const float2 *>(sc1);
+        s0s[0] = v0.x; s0s[1] = v0.y; s1s[0] = v1.x; s1s[1] = v1.y;
+    } else {
+        const float4 v0 = *reinterpret_cast<const float4 *>(sc0);
+        const float4 v1 = *reinterpret_cast<const float4 *>(sc1);
+        s0s[0] = v0.x; s0s[1] = v0.y; s0s[2] = v0.z; s0s[3] = v0.w;
+        s1s[0] = v1.x; s1s[1] = v1.y; s1s[2] = v1.z; s1s[3] = v1.w;
+    }
+    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+    const __nv_bfloat162 bias = __floats2bfloat162_rn(130.f, 130.f);
+    auto weights = [&](uint32_t c, uint32_t sel) -> uint32_t {
+        const uint32_t u = __byte_perm(c, 0x43434343u, sel);
+        const __nv_bfloat162 v = __hsub2(*reinterpret_cast<const __nv_bfloat162 *>(&u), bias);
+        return *reinterpret_cast<const uint32_t *>(&v);
+    };
+    float D[MT][4];   // fp32 sums of the current group; a group never outlives a cell
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        if (s < R) {
+            const bool first = (s % SPP) == 0;
+            const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
+            uint32_t X[MT][8];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const uint4 lo = ld_act16(brow[mt] + s * (2 * kSliceK));
+                const uint4 hi = ld_act16(brow[mt] + s * (2 * kSliceK) + 16);
+                X[mt][0] = lo.x; X[mt][1] = lo.y; X[mt][2] = lo.z; X[mt][3] = lo.w;
+                X[mt][4] = hi.x; X[mt][5] = hi.y; X[mt][6] = hi.z; X[mt][7] = hi.w;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t c0 = (w0s[s] >> (2 * j)) & 0x03030303u;
+                const uint32_t c1 = (w1s[s] >> (2 * j)) & 0x03030303u;
+                const uint32_t a0 = weights(c0, 0x4140u), a1 = weights(c1, 0x4140u);
+                const uint32_t a2 = weights(c0, 0x4342u), a3 = weights(c1, 0x4342u);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    if (first && j == 0) mma_bf16_16x8x16(D[mt], a0, a1, a2, a3, X[mt][2 * j], X[mt][2 * j + 1], zero);
+                    else                 mma_bf16_16x8x16(D[mt], a0, a1, a2, a3, X[mt][2 * j], X[mt][2 * j + 1], D[mt]);
+                }
+            }
+            if (last) {
+                const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    acc[mt][0] = fmaf(s0, D[mt][0], acc[mt][0]);
+                    acc[mt][2] = fmaf(s1, D[mt][2], acc[mt][2]);
+                    if constexpr (!ONE) {
+                        acc[mt][1] = fmaf(s0, D[mt][1], acc[mt][1]);
+                        acc[mt][3] = fmaf(s1, D[mt][3], acc[mt][3]);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // MT: 8-token slabs per CTA; SPP: 64-k slices per scale group (capped at 4);
 // TG: tiles the four warps of a CTA work on side by side (K-lanes per tile = 4 / TG);
 // RING: cells a warp can hold (the launch plan never gives it more); ONE: a single
@@ -251,7 +330,8 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
 // fully unrolled cell loop (slot and operand offsets are immediates), no
 // divisions and no 64-bit multiplies per cell.  Warps do not meet before the
 // final sum over the K-lanes.
-template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS, bool H16 = false>
+// A16: p.a holds the caller's bf16 activations (no quantiser, no token scale): compute_cell_a16.
+template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS, bool H16 = false, bool A16 = false>
 __global__ void __launch_bounds__(kDecodeThreads, W2A8_MINB(MT))
 w2a8_decode_kernel(const DecodeParams p) {
     constexpr int KS = kDecodeWarps / TG;
@@ -259,6 +339,7 @@ w2a8_decode_kernel(const DecodeParams p) {
     constexpr int kScaleBytes = 16 * 16;        // scales of one cell: 16 channels x 16 B
     constexpr int kWarpBytes = RING * (kSlotBytes + kScaleBytes);
     constexpr int SPB = 4 / SPP;                // scales per block and channel
+    constexpr int kActBytes = A16 ? 2 : 1;      // bytes per activation
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -404,7 +485,7 @@ w2a8_decode_kernel(const DecodeParams p) {
     const int8_t *brow[MT];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
-        brow[mt] = p.a + (size_t)(m0 + min(8 * mt + gq, mrows - 1)) * p.K + (size_t)kb0 * kBlockK + t * 16;
+        brow[mt] = p.a + ((size_t)(m0 + min(8 * mt + gq, mrows - 1)) * p.K + (size_t)kb0 * kBlockK + t * 16) * kActBytes;
     const size_t MN = (size_t)p.M * p.N;
     const unsigned char *sc0 = sslots + gq * 16, *sc1 = sc0 + 8 * 16;
 
@@ -419,9 +500,12 @@ w2a8_decode_kernel(const DecodeParams p) {
             const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
             const int8_t *bc[MT];
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + c * kBlockK;
-            compute_cell<MT, SPP, ONE, PARTIALS, true, H16>(p, w0s, w1s, sc0 + c * kScaleBytes, sc1 + c * kScaleBytes,
-                                                       bc, kb0 + c, n0, m0, gq, t, acc);
+            for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + c * (kBlockK * kActBytes);
+            if constexpr (A16)
+                compute_cell_a16<MT, SPP, ONE, true>(p, w0s, w1s, sc0 + c * kScaleBytes, sc1 + c * kScaleBytes, bc, acc);
+            else
+                compute_cell<MT, SPP, ONE, PARTIALS, true, H16>(p, w0s, w1s, sc0 + c * kScaleBytes,
+                                                                sc1 + c * kScaleBytes, bc, kb0 + c, n0, m0, gq, t, acc);
         }
     }
     if (tail_mine) {   // the trailing block is this warp's last cell; its words and scales were stored directly
@@ -432,10 +516,14 @@ w2a8_decode_kernel(const DecodeParams p) {
         const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
         const int8_t *bc[MT];
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + (size_t)tail_cell * kBlockK;
-        compute_cell<MT, SPP, ONE, PARTIALS, false, H16>(p, w0s, w1s, sc0 + tail_cell * kScaleBytes,
-                                                    sc1 + tail_cell * kScaleBytes, bc, kb0 + tail_cell,
-                                                    n0, m0, gq, t, acc);
+        for (int mt = 0; mt < MT; ++mt) bc[mt] = brow[mt] + (size_t)tail_cell * (kBlockK * kActBytes);
+        if constexpr (A16)
+            compute_cell_a16<MT, SPP, ONE, false>(p, w0s, w1s, sc0 + tail_cell * kScaleBytes,
+                                                  sc1 + tail_cell * kScaleBytes, bc, acc);
+        else
+            compute_cell<MT, SPP, ONE, PARTIALS, false, H16>(p, w0s, w1s, sc0 + tail_cell * kScaleBytes,
+                                                             sc1 + tail_cell * kScaleBytes, bc, kb0 + tail_cell,
+                                                             n0, m0, gq, t, acc);
     }
     W2A8_TRACE_POINT(5);
 
@@ -486,7 +574,7 @@ w2a8_decode_kernel(const DecodeParams p) {
 
         // final value of y[mm][nn]: fp32, or (16-bit instances, on request) rounded to bf16
         auto store_y = [&](int mm, int nn, float v) {
-            v *= p.a_scale[mm] * (1.0f / kCodeGain);
+            if constexpr (!A16) v *= p.a_scale[mm] * (1.0f / kCodeGain);   // bf16 weights carry no gain
             if constexpr (H16) {
                 if (p.y16) {
                     reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)mm * p.N + nn] = __float2bfloat16_rn(v);
@@ -714,6 +802,21 @@ static cudaError_t launch_decode_h16(const DecodeParams &p, dim3 grid, size_t sm
                                  p.cluster ? (unsigned)p.chunks : 1u, p);
 }
 
+// 16-bit-activation instances (bf16 x, fp32 scales, fp32 result): default grouping and slots.
+template <int MT, int SPP, bool ONE>
+static cudaError_t launch_decode_a16(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, true>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    return launch_kernel_cluster(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, true>, grid,
+                                 dim3(kDecodeThreads), smem, st, pdl_enabled(),
+                                 p.cluster ? (unsigned)p.chunks : 1u, p);
+}
+
 template <int MT, int SPP, int TG>
 static cudaError_t launch_decode_tg(const DecodeParams &p, int ring, bool want_partials, dim3 grid, size_t smem,
                                     cudaStream_t st) {
@@ -726,6 +829,10 @@ template <int MT, int SPP>
 static cudaError_t launch_decode_mt(const DecodeParams &p, const DecodePlan &pl, bool want_partials,
                                     cudaStream_t st) {
     dim3 grid(pl.groups, pl.chunks, pl.slabs);
+    if (p.a16) {
+        if (MT == 1 && p.M == 1) return launch_decode_a16<1, SPP, true>(p, grid, pl.smem, st);
+        return launch_decode_a16<MT, SPP, false>(p, grid, pl.smem, st);
+    }
     if (p.h16) {
         if (MT == 1 && p.M == 1) return launch_decode_h16<1, SPP, true>(p, grid, pl.smem, st);
         return launch_decode_h16<MT, SPP, false>(p, grid, pl.smem, st);
@@ -746,15 +853,19 @@ static cudaError_t launch_decode_spp(const DecodeParams &p, const DecodePlan &pl
 }
 
 // Enqueue the decode kernel.  `partials` != nullptr selects the parity export.  h16: w_scale
-// points at binary16 values; y16 (with h16 only): y points at bf16 values.
+// points at binary16 values; y16 (with h16 only): y points at bf16 values.  a16: a points at
+// bf16 activations and a_scale is not read.
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
-                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16) {
-    if (h16 && partials) return W2A8_ERR_SHAPE;
-    const DecodePlan pl = decode_plan(M, N, K, si, h16);
+                  int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16,
+                  bool a16) {
+    if ((h16 || a16) && partials) return W2A8_ERR_SHAPE;
+    if (h16 && a16) return W2A8_ERR_SHAPE;
+    const DecodePlan pl = decode_plan(M, N, K, si, h16 || a16);
     DecodeParams p;
     p.a = a; p.a_scale = a_scale; p.packed = packed; p.w_scale = reinterpret_cast<const float *>(w_scale);
     p.y = reinterpret_cast<float *>(y); p.partials = partials; p.h16 = h16 ? 1 : 0; p.y16 = (h16 && y16) ? 1 : 0;
+    p.a16 = a16 ? 1 : 0;
     p.M = M; p.N = N; p.K = K; p.G = si.G; p.group = group;
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
     p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;

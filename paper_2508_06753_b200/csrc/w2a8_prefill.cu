@@ -384,7 +384,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             // row pitch allows (G % 8 == 0: registers 0..3 hold two scales each), else as eight
             // 16-bit loads into 32-bit registers.
             const bool vec8 = H16 && (p.G % 8 == 0);
-            uint32_t sc_nxt[8];
+            uint32_t sc_nxt[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
             auto refill = [&](int g0) {
                 if constexpr (PARTIALS) {
                     return;
@@ -417,8 +417,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     return __uint_as_float(sc_nxt[u]);
                 }
             };
-#pragma unroll
-            for (int u = 0; u < 8; ++u) sc_nxt[u] = 0u;
             refill(0);
             // Software pipeline over 32-column halves: while one half is converted and
             // accumulated, the next half (possibly of the next group) is on its way from TMEM.
