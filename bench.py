@@ -510,6 +510,59 @@ def recipe16_probe(rep, peaks, group=128, reps=200):
                     "a8_quantize per layer pass; GB/s on this recipe's own byte count", "per_m": out}
 
 
+def a16_probe(rep, peaks, reps=200):
+    """Extra row (not the headline): the same layer through w2a16_gemm -- bf16 activations against
+    the 2-bit weights, no activation quantiser: 7 launches per pass instead of 11.  GB/s on this
+    entry's own byte count (bf16 activations: 2 bytes each, no token scales)."""
+    torch, b, cfg = rep.torch, rep.b, rep.cfg
+    dev = rep.ws.device
+
+    def bytes_of(M, N, K, g):
+        return K * N // 4 + (K // g) * N * 4 + 2 * M * K + 4 * M * N
+
+    out = {}
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        for M in cfg["Ms"]:
+            bufs = rep.per_m[M]
+
+            def one_pass(c):
+                for idx, (name, K, N) in enumerate(rep.shapes):
+                    packed, s_w, g = rep.copies[c][idx]
+                    b.w2a16_gemm(bufs["x"][rep.input_of[name]], packed, s_w, g, rep.ws, bufs["y"][idx])
+            for c in range(len(rep.copies)):
+                one_pass(c)
+            torch.cuda.synchronize()
+            try:
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=stream):
+                    for c in range(len(rep.copies)):
+                        one_pass(c)
+                run = gr.replay
+            except Exception:
+                def run():
+                    for c in range(len(rep.copies)):
+                        one_pass(c)
+            for _ in range(3):
+                run()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = max(reps // len(rep.copies), 3)
+            e0.record()
+            for _ in range(n):
+                run()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / (n * len(rep.copies))
+            nbytes = sum(bytes_of(M, N, K, synth.config_group(cfg, K)) for _, K, N in rep.shapes)
+            out[str(M)] = {"us_per_layer": ms * 1e3, "bytes_per_layer": nbytes, "gbs": nbytes / (ms * 1e-3) / 1e9,
+                           "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    torch.cuda.current_stream().wait_stream(stream)
+    return {"what": "w2a16_gemm (bf16 activations, no a8_quantize): 7 launches per layer pass; GB/s on this "
+                    "entry's own byte count", "per_m": out}
+
+
 def e2e_measure(rep, steps, warmup):
     """Same workload through w2a8_linear_host: pinned host activations in, host
     outputs back, copies inside the timed region."""
@@ -699,6 +752,7 @@ def run_ours(args):
     concat = concat_probe(rep) if rank == 0 else None
     recipe16 = recipe16_probe(rep, peaks) if rank == 0 else None
     small = small_shape_probe(device, peaks, l2) if rank == 0 else None
+    a16 = a16_probe(rep, peaks) if rank == 0 else None
     prefill = None
     if rank == 0 and not args.no_prefill:
         prefill = prefill_probe(device, peaks)
@@ -743,6 +797,7 @@ def run_ours(args):
         "kernel_probes": probes, "concatenated_qkv_gateup": concat,
         "recipe_g128_binary16_scales_bf16_out": recipe16,
         "paper_small_shapes_m1": small,
+        "w2a16_no_quantiser": a16,
         "prefill": prefill,
     }
     print(json.dumps(out))

@@ -247,9 +247,12 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
 // bf16 values as they are, and the products are summed in fp32 by `mma.sync.m16n8k16`; the
 // group scale multiplies the fp32 sum of its group.
 // A lane's word of a slice holds code l (k = 16 t + l of the slice) at bits 8 (l mod 4) +
-// 2 (l div 4); MMA j of the slice takes l = 4 j .. 4 j + 3: after a shift by 2 j the four codes
-// sit in the four bytes.  0x4300 | q is the bf16 value 128 + q, so a byte permute with 0x43 and
-// one packed subtraction of 130 give the two bf16 weights of a register.
+// 2 (l div 4); MMA j of the slice takes l = 4 j .. 4 j + 3, the two bits at offset 2 j of each
+// byte.  With the code left where it is, (0x43 - j) << 8 | (q << 2 j) is the bf16 value
+// 2^(7 - 2 j) + q for j = 0, 1, 2 (the code sits in the mantissa, one unit of it worth 1), so a
+// mask, a byte permute with the exponent byte and one packed subtraction of 2^(7 - 2 j) + 2 give
+// the two bf16 weights of a register; j = 3 would reach the exponent bit and is shifted down to
+// the j = 0 form.
 // brow[mt]: this lane's 32 activation bytes (16 bf16) of slice 0, token row of slab mt.
 template <int MT, int SPP, bool ONE, bool FULL>
 __device__ __forceinline__ void compute_cell_a16(const DecodeParams &p, const uint32_t (&w0s)[4],
@@ -272,10 +275,10 @@ __device__ __forceinline__ void compute_cell_a16(const DecodeParams &p, const ui
         s1s[0] = v1.x; s1s[1] = v1.y; s1s[2] = v1.z; s1s[3] = v1.w;
     }
     const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-    const __nv_bfloat162 bias = __floats2bfloat162_rn(130.f, 130.f);
-    auto weights = [&](uint32_t c, uint32_t sel) -> uint32_t {
-        const uint32_t u = __byte_perm(c, 0x43434343u, sel);
-        const __nv_bfloat162 v = __hsub2(*reinterpret_cast<const __nv_bfloat162 *>(&u), bias);
+    auto weights = [&](uint32_t c, uint32_t expo, float off, uint32_t sel) -> uint32_t {
+        const uint32_t u = __byte_perm(c, expo, sel);
+        const __nv_bfloat162 v = __hsub2(*reinterpret_cast<const __nv_bfloat162 *>(&u),
+                                         __floats2bfloat162_rn(off, off));
         return *reinterpret_cast<const uint32_t *>(&v);
     };
     float D[MT][4];   // fp32 sums of the current group; a group never outlives a cell
@@ -294,10 +297,13 @@ __device__ __forceinline__ void compute_cell_a16(const DecodeParams &p, const ui
             }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint32_t c0 = (w0s[s] >> (2 * j)) & 0x03030303u;
-                const uint32_t c1 = (w1s[s] >> (2 * j)) & 0x03030303u;
-                const uint32_t a0 = weights(c0, 0x4140u), a1 = weights(c1, 0x4140u);
-                const uint32_t a2 = weights(c0, 0x4342u), a3 = weights(c1, 0x4342u);
+                // j is a constant after unrolling
+                const uint32_t c0 = j < 3 ? (w0s[s] & (0x03030303u << (2 * j))) : ((w0s[s] >> 6) & 0x03030303u);
+                const uint32_t c1 = j < 3 ? (w1s[s] & (0x03030303u << (2 * j))) : ((w1s[s] >> 6) & 0x03030303u);
+                const uint32_t expo = j == 1 ? 0x42424242u : j == 2 ? 0x41414141u : 0x43434343u;
+                const float off = j == 1 ? 34.f : j == 2 ? 10.f : 130.f;
+                const uint32_t a0 = weights(c0, expo, off, 0x4140u), a1 = weights(c1, expo, off, 0x4140u);
+                const uint32_t a2 = weights(c0, expo, off, 0x4342u), a3 = weights(c1, expo, off, 0x4342u);
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     if (first && j == 0) mma_bf16_16x8x16(D[mt], a0, a1, a2, a3, X[mt][2 * j], X[mt][2 * j + 1], zero);
