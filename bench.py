@@ -932,17 +932,28 @@ def run_kernel_profile(args):
     a, s_a = b.a8_quantize(x)
     ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g), device=dev)
     y = torch.empty((M, N), dtype=torch.float32, device=dev)
+    if args.profile_entry == "a16":
+        def gemm(pk, sw):
+            b.w2a16_gemm(x, pk, sw, g, ws, y)
+    elif args.profile_entry == "h16":
+        mats = [(pk, sw.half()) for pk, sw in mats]
+
+        def gemm(pk, sw):
+            b.w2a8_gemm_h16(a, s_a, pk, sw, g, ws, y)
+    else:
+        def gemm(pk, sw):
+            b.w2a8_gemm(a, s_a, pk, sw, g, ws, y)
     for i in range(args.profile_reps):                      # warm-up
-        b.w2a8_gemm(a, s_a, mats[i % copies][0], mats[i % copies][1], g, ws, y)
+        gemm(*mats[i % copies])
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.profile_reps):
-        b.w2a8_gemm(a, s_a, mats[i % copies][0], mats[i % copies][1], g, ws, y)
+        gemm(*mats[i % copies])
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / args.profile_reps
-    print(json.dumps({"profile_shape": f"{K}x{N}", "M": M, "group": g, "copies": copies,
+    print(json.dumps({"profile_shape": f"{K}x{N}", "entry": args.profile_entry, "M": M, "group": g, "copies": copies,
                       "launches": 2 * args.profile_reps, "us_per_launch_direct": us,
                       "bytes_per_launch": gemm_bytes(M, N, K, g),
                       "gbs": gemm_bytes(M, N, K, g) / us / 1e3}))
@@ -978,6 +989,8 @@ def main():
     ap.add_argument("--profile-m", type=int, default=1)
     ap.add_argument("--profile-group", type=int, default=64)
     ap.add_argument("--profile-reps", type=int, default=10)
+    ap.add_argument("--profile-entry", default="a8", choices=["a8", "h16", "a16"],
+                    help="entry point the profile run launches: w2a8_gemm, w2a8_gemm_h16 or w2a16_gemm")
     args = ap.parse_args()
     if args.profile_shape:
         run_kernel_profile(args)
