@@ -126,8 +126,10 @@ int w2a8_workspace_status(const void *workspace, void *stream);
  *   y       [M][N] fp32, row-major, fully overwritten
  *   workspace / workspace_bytes: see w2a8_workspace_bytes.
  * M >= 64 with N % 128 == 0 and K % 256 == 0 takes the tensor-core kernel
- * (tcgen05, 128 x 128 output tiles); everything else takes the memory-bound
- * streaming kernel (weights read once per slab of up to 32 tokens).
+ * (tcgen05, 128 x 128 output tiles) when there are enough output tiles for it
+ * to be the faster one (M * N above about 0.95 million per round of 148
+ * tiles); everything else takes the memory-bound streaming kernel (weights
+ * read once per slab of up to 32 tokens).  w2a8_kernel_for reports the choice.
  */
 int w2a8_gemm(const int8_t *a, const float *a_scale, const uint32_t *packed,
               const float *w_scale, float *y, int M, int N, int K, int group,
@@ -182,6 +184,15 @@ int w2a8_gemm_h16(const int8_t* a, const float* a_scale, const uint32_t* packed,
  */
 int w2a16_gemm(const void* x_bf16, const uint32_t* packed, const float* w_scale, float* y,
                int M, int N, int K, int group, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Which kernel w2a8_gemm / w2a8_gemm_h16 / w2a8_linear use for a shape:
+ * 0 = streaming kernel, 1 = tensor-core kernel, W2A8_ERR_SHAPE for a shape
+ * that is not accepted.  Host only, launches nothing.  (The paper picks its
+ * kernel variant per shape with an auto-tuner, Sec. II; here the rule is fixed
+ * and measured.)
+ */
+int w2a8_kernel_for(int M, int N, int K, int group);
 
 /*
  * w2a8_gemm_partials -- parity/debug export of the exact int32 per-group sums

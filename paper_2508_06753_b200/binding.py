@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libw2a8.so")
 EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
-    "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
+    "w2a8_kernel_for", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
 ]
 
 _lib = None
@@ -53,6 +53,7 @@ def lib() -> ctypes.CDLL:
         L.w2a8_workspace_status.argtypes = [vp, vp]
         L.w2a8_gemm.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_h16.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp, sz, vp]
+        L.w2a8_kernel_for.argtypes = [i, i, i, i]
         L.w2a16_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_partials.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
@@ -153,6 +154,13 @@ def w2a8_gemm(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor, w_sc
                            group, _ptr(workspace), workspace.numel() * workspace.element_size(),
                            _stream(stream)), "w2a8_gemm")
     return y
+
+
+def w2a8_kernel_for(M: int, N: int, K: int, group: int) -> str:
+    """'streaming' or 'tensor_core': the kernel w2a8_gemm uses for this shape."""
+    r = int(lib().w2a8_kernel_for(M, N, K, group))
+    _check(r if r < 0 else 0, "w2a8_kernel_for")
+    return "tensor_core" if r == 1 else "streaming"
 
 
 def w2a8_gemm_h16(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor, w_scale_h: torch.Tensor,

@@ -14,6 +14,7 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
 
 bool prefill_supported(int M, int N, int K, int group);
+bool prefill_preferred(int M, int N, int K, int group);
 int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
                    void *y, int32_t *partials, int M, int N, int K, int group, int *status,
                    cudaStream_t st, bool h16, bool y16);
@@ -279,6 +280,22 @@ int w2a8_workspace_status(const void *workspace, void *stream) {
     return status;
 }
 
+// W2A8_PREFILL: 0 = never the tensor-core kernel, 2 = whenever it supports the shape, else
+// (default) when it supports the shape and is expected to be the faster one.
+static bool takes_tensor_core_kernel(int M, int N, int K, int group) {
+    if (!prefill_supported(M, N, K, group)) return false;
+    const int mode = env_int("W2A8_PREFILL", 1);
+    if (mode == 0) return false;
+    if (mode == 2) return true;
+    return prefill_preferred(M, N, K, group);
+}
+
+int w2a8_kernel_for(int M, int N, int K, int group) {
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
+    return takes_tensor_core_kernel(M, N, K, group) ? 1 : 0;
+}
+
 // h16: w_scale holds binary16 values; y16 (with h16): y holds bf16 values.
 static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *packed,
                        const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
@@ -293,8 +310,9 @@ static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *pa
     const size_t need = decode_workspace_bytes(M, N, K, si);
     if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
     if (int st = check_device()) return st;
-    // many tokens: tensor-core path (tcgen05); few tokens, or shapes it does not tile: streaming path
-    if (!a16 && prefill_supported(M, N, K, group) && env_int("W2A8_PREFILL", 1) != 0)
+    // many tokens: tensor-core path (tcgen05); few tokens, shapes it does not tile, or too few
+    // output tiles to fill the GPU: streaming path
+    if (!a16 && takes_tensor_core_kernel(M, N, K, group))
         return launch_prefill(a, a_scale, packed, w_scale, y, partials, M, N, K, group,
                               reinterpret_cast<int *>(workspace), (cudaStream_t)stream, h16, y16);
     return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,

@@ -533,6 +533,19 @@ bool prefill_supported(int M, int N, int K, int group) {
     return true;
 }
 
+// Whether the tensor-core kernel is expected to beat the streaming kernel on a shape it supports.
+// Its grid is one CTA per 128 x 128 output tile (at most one per SM), each walking all of K, so a
+// problem with few tiles leaves most SMs idle: on B200 a round of tiles takes about 7 ns per unit
+// of K, the streaming kernel about 8e-15 s per token x weight, which crosses at M * N of about
+// 0.95 million per round (measured: 14336x4096 at M = 128: 94 us against 66 us streaming; at
+// M = 256: 97 against 127; 4096x4096 at M = 64: 31 against 11).
+bool prefill_preferred(int M, int N, int K, int group) {
+    (void)K; (void)group;
+    const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
+    const long long rounds = (tiles + 147) / 148;
+    return (long long)M * N > rounds * 950000ll;
+}
+
 // Enqueue the prefill kernel.  `partials` != nullptr selects the parity export.
 int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
                    void *y, int32_t *partials, int M, int N, int K, int group, int *status,

@@ -95,8 +95,9 @@ CASES = [
 
 
 @pytest.mark.parametrize("M,N,K,group,ternary,frac", CASES)
-def test_h16_against_reference(gpu, oracle, M, N, K, group, ternary, frac):
+def test_h16_against_reference(gpu, oracle, M, N, K, group, ternary, frac, monkeypatch):
     torch, b = gpu
+    monkeypatch.setenv("W2A8_PREFILL", "2")     # small many-token shapes: exercise the tensor-core kernel
     _check(torch, b, oracle, M, N, K, group, seed=M * 37 + N + K, ternary=ternary, frac=frac)
 
 

@@ -20,6 +20,13 @@ def gpu():
     return torch, binding
 
 
+@pytest.fixture(autouse=True)
+def force_tensor_core_kernel(monkeypatch):
+    """Small shapes would be given to the streaming kernel by the dispatch rule; these tests are
+    about the tensor-core kernel, so it is taken whenever it supports the shape."""
+    monkeypatch.setenv("W2A8_PREFILL", "2")
+
+
 def _dev(torch, arr):
     return torch.from_numpy(np.ascontiguousarray(arr)).cuda()
 
@@ -44,6 +51,7 @@ CASES = [
 def test_prefill_against_reference(gpu, oracle, M, N, K, group):
     torch, b = gpu
     g = K if group == 0 else group
+    assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
     codes, s_w = synth.make_linear(7 * M + N + K, K, N, g)
     bits = synth.activations_bf16(M + K, M, K)
     packed = b.w2_pack(_dev(torch, codes))
@@ -72,8 +80,10 @@ def test_prefill_matches_streaming_path(gpu, monkeypatch):
     packed = b.w2_pack(_dev(torch, codes))
     a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
     ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
     y_tc = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws).cpu().numpy()
     monkeypatch.setenv("W2A8_PREFILL", "0")
+    assert b.w2a8_kernel_for(M, N, K, g) == "streaming"
     y_st = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws).cpu().numpy()
     assert np.abs(y_tc - y_st).max() <= TOL * np.abs(y_st).max()
 
@@ -101,3 +111,32 @@ def test_prefill_full_size_sampled_rows(gpu, oracle, K, N):
     got = y.cpu().numpy()[rows].astype(np.float64)
     err = np.abs(got - y_ref).max(axis=1)
     assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), float((err / np.abs(y_ref).max(axis=1)).max())
+
+
+def test_dispatch_rule(gpu, oracle, monkeypatch):
+    """Default dispatch: few output tiles go to the streaming kernel even with many tokens; both
+    choices give the reference result on a shape next to the boundary."""
+    torch, b = gpu
+    monkeypatch.delenv("W2A8_PREFILL", raising=False)
+    assert b.w2a8_kernel_for(2048, 14336, 4096, 64) == "tensor_core"
+    assert b.w2a8_kernel_for(512, 4096, 14336, 64) == "tensor_core"
+    assert b.w2a8_kernel_for(128, 4096, 14336, 64) == "streaming"       # 32 tiles on 148 SMs
+    assert b.w2a8_kernel_for(64, 4096, 4096, 64) == "streaming"
+    assert b.w2a8_kernel_for(256, 4096, 4096, 64) == "tensor_core"
+    assert b.w2a8_kernel_for(63, 14336, 4096, 64) == "streaming"        # below the token threshold
+    assert b.w2a8_kernel_for(512, 1040, 4096, 64) == "streaming"        # N not a multiple of 128
+    M, N, K, g = 224, 4096, 512, 64                                     # M * N just below the boundary
+    assert b.w2a8_kernel_for(M, N, K, g) == "streaming"
+    codes, s_w = synth.make_linear(11, K, N, g)
+    bits = synth.activations_bf16(11, M, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    a_ref, s_ref = oracle.quantize(bits)
+    y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+    for mode in ("1", "2"):
+        monkeypatch.setenv("W2A8_PREFILL", mode)
+        y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws).cpu().numpy()
+        assert b.w2a8_workspace_status(ws) == 0
+        err = np.abs(y.astype(np.float64) - y_ref).max(axis=1)
+        assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), mode
