@@ -195,6 +195,17 @@ int w2a16_gemm(const void* x_bf16, const uint32_t* packed, const float* w_scale,
 int w2a8_kernel_for(int M, int N, int K, int group);
 
 /*
+ * How many of the N output channels the tensor-core kernel computes for this
+ * shape: 0 when the streaming kernel takes the whole problem, N when the
+ * tensor-core kernel does, and a multiple of 128 in between when the last
+ * channel tiles are given to the streaming kernel in a second launch (the
+ * tensor-core kernel works in rounds of one 128 x 128 tile per SM, and a last
+ * round with a handful of tiles costs as much as a full one).  Host only.
+ * W2A8_ERR_SHAPE for a shape that is not accepted.
+ */
+int w2a8_tensor_core_channels(int M, int N, int K, int group);
+
+/*
  * w2a8_gemm_partials -- parity/debug export of the exact int32 per-group sums
  * P[m][n][gi] computed by the same inner-product code as w2a8_gemm.
  *   partials [M][N][K/group] int32, fully overwritten.

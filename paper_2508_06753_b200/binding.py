@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libw2a8.so")
 EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
-    "w2a8_kernel_for", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
+    "w2a8_kernel_for", "w2a8_tensor_core_channels", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
 ]
 
 _lib = None
@@ -54,6 +54,7 @@ def lib() -> ctypes.CDLL:
         L.w2a8_gemm.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_h16.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp, sz, vp]
         L.w2a8_kernel_for.argtypes = [i, i, i, i]
+        L.w2a8_tensor_core_channels.argtypes = [i, i, i, i]
         L.w2a16_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_partials.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
@@ -161,6 +162,14 @@ def w2a8_kernel_for(M: int, N: int, K: int, group: int) -> str:
     r = int(lib().w2a8_kernel_for(M, N, K, group))
     _check(r if r < 0 else 0, "w2a8_kernel_for")
     return "tensor_core" if r == 1 else "streaming"
+
+
+def w2a8_tensor_core_channels(M: int, N: int, K: int, group: int) -> int:
+    """Channels of the problem computed by the tensor-core kernel (0 .. N); the rest, if any, is
+    computed by the streaming kernel."""
+    r = int(lib().w2a8_tensor_core_channels(M, N, K, group))
+    _check(r if r < 0 else 0, "w2a8_tensor_core_channels")
+    return r
 
 
 def w2a8_gemm_h16(a: torch.Tensor, a_scale: torch.Tensor, packed: torch.Tensor, w_scale_h: torch.Tensor,

@@ -10,14 +10,15 @@ namespace w2a8 {
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16,
-                  bool a16);
+                  bool a16, int ldy);
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
 
 bool prefill_supported(int M, int N, int K, int group);
 bool prefill_preferred(int M, int N, int K, int group);
 int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
                    void *y, int32_t *partials, int M, int N, int K, int group, int *status,
-                   cudaStream_t st, bool h16, bool y16);
+                   cudaStream_t st, bool h16, bool y16, int ldy);
+int prefill_channel_split(int M, int N, int K, int group);
 
 int env_int(const char *name, int dflt) {
     const char *v = getenv(name);
@@ -257,10 +258,23 @@ int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, voi
     return e == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
 
+static bool takes_tensor_core_kernel(int M, int N, int K, int group);
+static int tensor_core_channels(int M, int N, int K, int group);
+
 size_t w2a8_workspace_bytes(int M, int N, int K, int group) {
     ShapeInfo si;
     if (!shape_ok(M, N, K, group, &si)) return 0;
-    return decode_workspace_bytes(M, N, K, si);
+    size_t need = decode_workspace_bytes(M, N, K, si);
+    if (takes_tensor_core_kernel(M, N, K, group)) {
+        // the last channel tiles may be given to the streaming kernel, with a plan of its own
+        const int n_tc = tensor_core_channels(M, N, K, group);
+        ShapeInfo rest;
+        if (n_tc < N && shape_ok(M, N - n_tc, K, group, &rest)) {
+            const size_t r = decode_workspace_bytes(M, N - n_tc, K, rest);
+            if (r > need) need = r;
+        }
+    }
+    return need;
 }
 
 int w2a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream) {
@@ -290,10 +304,23 @@ static bool takes_tensor_core_kernel(int M, int N, int K, int group) {
     return prefill_preferred(M, N, K, group);
 }
 
+// Channels the tensor-core kernel takes (the rest, if any, goes to the streaming kernel in a
+// second launch): all of them with W2A8_PREFILL=2 or W2A8_PF_SPLIT=0.
+static int tensor_core_channels(int M, int N, int K, int group) {
+    if (env_int("W2A8_PREFILL", 1) == 2 || env_int("W2A8_PF_SPLIT", 1) == 0) return N;
+    return prefill_channel_split(M, N, K, group);
+}
+
 int w2a8_kernel_for(int M, int N, int K, int group) {
     ShapeInfo si;
     if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
     return takes_tensor_core_kernel(M, N, K, group) ? 1 : 0;
+}
+
+int w2a8_tensor_core_channels(int M, int N, int K, int group) {
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
+    return takes_tensor_core_kernel(M, N, K, group) ? tensor_core_channels(M, N, K, group) : 0;
 }
 
 // h16: w_scale holds binary16 values; y16 (with h16): y holds bf16 values.
@@ -307,16 +334,29 @@ static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *pa
         (w_scale && !aligned16(w_scale)) || (partials && !aligned16(partials)) ||
         (a_scale && (reinterpret_cast<uintptr_t>(a_scale) & 3u)))
         return W2A8_ERR_ALIGN;
-    const size_t need = decode_workspace_bytes(M, N, K, si);
+    const size_t need = w2a8_workspace_bytes(M, N, K, group);
     if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
     if (int st = check_device()) return st;
     // many tokens: tensor-core path (tcgen05); few tokens, shapes it does not tile, or too few
     // output tiles to fill the GPU: streaming path
-    if (!a16 && takes_tensor_core_kernel(M, N, K, group))
-        return launch_prefill(a, a_scale, packed, w_scale, y, partials, M, N, K, group,
-                              reinterpret_cast<int *>(workspace), (cudaStream_t)stream, h16, y16);
+    if (!a16 && takes_tensor_core_kernel(M, N, K, group)) {
+        // The tensor-core kernel takes the first n_tc channels; when a last round of a few tiles
+        // would cost a whole round, the remaining channel tiles go to the streaming kernel in a
+        // second launch (rows of the packed matrix and of the scales are independent; both kernels
+        // write their own columns of y).  The parity export is never split.
+        const int n_tc = partials ? N : tensor_core_channels(M, N, K, group);
+        int st = launch_prefill(a, a_scale, packed, w_scale, y, partials, M, n_tc, K, group,
+                                reinterpret_cast<int *>(workspace), (cudaStream_t)stream, h16, y16, N);
+        ShapeInfo rest;
+        if (st != W2A8_OK || n_tc >= N || !shape_ok(M, N - n_tc, K, group, &rest)) return st;
+        const size_t scale_bytes = h16 ? 2 : 4, y_bytes = (h16 && y16) ? 2 : 4;
+        return launch_decode(a, a_scale, packed + (size_t)n_tc * si.words_per_row,
+                             reinterpret_cast<const char *>(w_scale) + (size_t)n_tc * si.G * scale_bytes,
+                             reinterpret_cast<char *>(y) + (size_t)n_tc * y_bytes, nullptr, M, N - n_tc, K,
+                             group, rest, workspace, (cudaStream_t)stream, h16, y16, false, N);
+    }
     return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,
-                         (cudaStream_t)stream, h16, y16, a16);
+                         (cudaStream_t)stream, h16, y16, a16, N);
 }
 
 int w2a16_gemm(const void *x_bf16, const uint32_t *packed, const float *w_scale, float *y, int M, int N,
@@ -360,7 +400,7 @@ int w2a8_linear(const void *x_bf16, int8_t *a, float *a_scale, const uint32_t *p
     if (!aligned16(x_bf16) || !aligned16(a) || !aligned16(packed) || !aligned16(y) || !aligned16(w_scale) ||
         (reinterpret_cast<uintptr_t>(a_scale) & 3u))
         return W2A8_ERR_ALIGN;
-    const size_t need = decode_workspace_bytes(M, N, K, si);
+    const size_t need = w2a8_workspace_bytes(M, N, K, group);
     if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
     if (int st = check_device()) return st;
     // Two launches chained by programmatic dependent launch.  A single-launch form (M extra CTAs

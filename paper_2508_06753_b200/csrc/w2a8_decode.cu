@@ -70,6 +70,7 @@ struct DecodeParams {
     int s_vec;            // the scales of a cell and channel can be copied as one unit (16/8 B fp32, 8/4 B binary16)
     int h16;              // w_scale holds IEEE binary16 values (16-bit instances)
     int a16;              // a holds bf16 activations, a_scale is unused (16-bit-activation instances)
+    int ldy;              // elements between consecutive token rows of y (>= N)
     int y16;              // 16-bit instances only: y holds bf16 instead of fp32
 };
 
@@ -583,11 +584,11 @@ w2a8_decode_kernel(const DecodeParams p) {
             if constexpr (!A16) v *= p.a_scale[mm] * (1.0f / kCodeGain);   // bf16 weights carry no gain
             if constexpr (H16) {
                 if (p.y16) {
-                    reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)mm * p.N + nn] = __float2bfloat16_rn(v);
+                    reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)mm * p.ldy + nn] = __float2bfloat16_rn(v);
                     return;
                 }
             }
-            p.y[(size_t)mm * p.N + nn] = v;
+            p.y[(size_t)mm * p.ldy + nn] = v;
         };
 
         if (p.chunks == 1) {
@@ -870,14 +871,14 @@ static cudaError_t launch_decode_spp(const DecodeParams &p, const DecodePlan &pl
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16,
-                  bool a16) {
+                  bool a16, int ldy) {
     if ((h16 || a16) && partials) return W2A8_ERR_SHAPE;
     if (h16 && a16) return W2A8_ERR_SHAPE;
     const DecodePlan pl = decode_plan(M, N, K, si, h16 || a16);
     DecodeParams p;
     p.a = a; p.a_scale = a_scale; p.packed = packed; p.w_scale = reinterpret_cast<const float *>(w_scale);
     p.y = reinterpret_cast<float *>(y); p.partials = partials; p.h16 = h16 ? 1 : 0; p.y16 = (h16 && y16) ? 1 : 0;
-    p.a16 = a16 ? 1 : 0;
+    p.a16 = a16 ? 1 : 0; p.ldy = ldy;
     p.M = M; p.N = N; p.K = K; p.G = si.G; p.group = group;
     p.blocks = si.blocks; p.tail_slices = si.tail_slices; p.words_per_row = si.words_per_row;
     p.chunks = pl.chunks; p.blocks_per_chunk = pl.blocks_per_chunk;

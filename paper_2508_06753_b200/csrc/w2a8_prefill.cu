@@ -58,6 +58,7 @@ struct PrefillParams {
     int words_per_row;
     int slices_per_group;    // group / 64
     int y16;                 // 16-bit instance only: y holds bf16 instead of fp32
+    int ldy;                 // elements between consecutive token rows of y (>= N)
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------
@@ -489,8 +490,8 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     const int m = m0 + col0 + j;
                     if (m < p.M) {
                         const float v = acc[j] * (__ldg(p.a_scale + m) * (1.0f / kCodeGain));
-                        if (H16 && p.y16) reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)m * p.N + n] = __float2bfloat16_rn(v);
-                        else              p.y[(size_t)m * p.N + n] = v;
+                        if (H16 && p.y16) reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)m * p.ldy + n] = __float2bfloat16_rn(v);
+                        else              p.y[(size_t)m * p.ldy + n] = v;
                     }
                 }
             }
@@ -546,10 +547,30 @@ bool prefill_preferred(int M, int N, int K, int group) {
     return (long long)M * N > rounds * 950000ll;
 }
 
+// How many of the N channels the tensor-core kernel should take when the rest may go to the
+// streaming kernel.  Tiles are handed out in rounds of 148; a last round with a handful of tiles
+// costs as much as a full one (4096x14336 at M = 512: 448 tiles = 3 rounds + 4 tiles).  Tiles are
+// ordered channel tile first, so giving the last few channel tiles (at most eight) to the
+// streaming kernel can remove that round.  Same cost model as prefill_preferred, plus 2 us for
+// the extra launch.  Returns a multiple of 128 in (0, N].
+int prefill_channel_split(int M, int N, int K, int group) {
+    (void)group;
+    const int ct = N / kPfBM, tiles_m = (M + kPfBN - 1) / kPfBN;
+    double best = 1e30;
+    int best_ct = ct;
+    for (int c = ct; c >= 1 && c >= ct - 8; --c) {
+        const long long rounds = ((long long)c * tiles_m + 147) / 148;
+        double t = (double)rounds * K * 7.0e-9;
+        if (c < ct) t += 2.0e-6 + 8.0e-15 * (double)M * (double)(ct - c) * kPfBM * (double)K;
+        if (t < best * 0.97) { best = t; best_ct = c; }      // a split has to pay by 3 % or more
+    }
+    return best_ct * kPfBM;
+}
+
 // Enqueue the prefill kernel.  `partials` != nullptr selects the parity export.
 int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
                    void *y, int32_t *partials, int M, int N, int K, int group, int *status,
-                   cudaStream_t st, bool h16, bool y16) {
+                   cudaStream_t st, bool h16, bool y16, int ldy) {
     if (h16 && partials) return W2A8_ERR_SHAPE;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return W2A8_ERR_CUDA;
@@ -565,6 +586,7 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
     PrefillParams p;
     p.packed = packed; p.w_scale = reinterpret_cast<const float *>(w_scale); p.a_scale = a_scale;
     p.y = reinterpret_cast<float *>(y); p.partials = partials; p.y16 = (h16 && y16) ? 1 : 0;
+    p.ldy = ldy;
     p.status = status;
     p.M = M; p.N = N; p.K = K; p.G = K / group; p.group = group;
     p.words_per_row = K / 16;

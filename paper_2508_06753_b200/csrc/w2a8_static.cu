@@ -10,7 +10,7 @@ namespace w2a8 {
 int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16,
-                  bool a16);
+                  bool a16, int ldy);
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
 size_t decode_workspace_header_bytes(int M, int N, int K, const ShapeInfo &si);
 }  // namespace w2a8
@@ -64,5 +64,5 @@ extern "C" int w2a8_gemm_static(const int8_t *a, const float *a_scale, const uin
         cudaSuccess)
         return W2A8_ERR_CUDA;
     return launch_decode(a, a_scale, packed, w_scale, y, nullptr, M, N, K, group, si, scratch,
-                         (cudaStream_t)stream, false, false, false);
+                         (cudaStream_t)stream, false, false, false, N);
 }

@@ -140,3 +140,49 @@ def test_dispatch_rule(gpu, oracle, monkeypatch):
         assert b.w2a8_workspace_status(ws) == 0
         err = np.abs(y.astype(np.float64) - y_ref).max(axis=1)
         assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), mode
+
+
+@pytest.mark.parametrize("h16", [False, True])
+def test_channel_split_between_the_two_kernels(gpu, oracle, monkeypatch, h16):
+    """150 channel tiles on 148 SMs: the tensor-core kernel takes 148 of them, the streaming kernel
+    the last 256 channels, both writing their own columns of y."""
+    torch, b = gpu
+    monkeypatch.delenv("W2A8_PREFILL", raising=False)
+    M, N, K, g = 128, 19200, 1024, 64
+    assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
+    assert b.w2a8_tensor_core_channels(M, N, K, g) == 148 * 128
+    assert b.w2a8_tensor_core_channels(2048, 14336, 4096, 64) == 111 * 128      # 1776 tiles = 12 rounds
+    assert b.w2a8_tensor_core_channels(512, 14336, 4096, 64) == 111 * 128       # 444 tiles = 3 rounds
+    assert b.w2a8_tensor_core_channels(512, 4096, 14336, 64) == 4096            # one round: nothing to gain
+    assert b.w2a8_tensor_core_channels(16, 4096, 4096, 64) == 0
+    codes = synth.weight_codes(3, N, K)
+    bits = synth.activations_bf16(3, M, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    a_ref, s_ref = oracle.quantize(bits)
+    if h16:
+        s_h = synth.weight_scales_h(3, N, K // g)
+        y = b.w2a8_gemm_h16(a, s_a, packed, _dev(torch, s_h.view(np.int16)).view(torch.float16), g, ws,
+                            out_dtype=torch.bfloat16)
+        y_ref, _ = oracle.gemm_h(a_ref, s_ref, codes, s_h, g)
+        tol = 2.0 ** -8 + TOL
+        y = y.float()
+    else:
+        s_w = synth.weight_scales(3, N, K // g)
+        y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
+        y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+        tol = TOL
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max(axis=1)
+    assert (err <= tol * np.abs(y_ref).max(axis=1)).all()
+    # the same problem with the split switched off gives the same bits in the tensor-core part
+    # and values within tolerance in the rest
+    monkeypatch.setenv("W2A8_PF_SPLIT", "0")
+    assert b.w2a8_tensor_core_channels(M, N, K, g) == N
+    if not h16:
+        y_all = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(y_all[:, :148 * 128], y[:, :148 * 128])
+        assert (y_all[:, 148 * 128:] - y[:, 148 * 128:]).abs().max() <= TOL * y.abs().max()
