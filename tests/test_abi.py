@@ -101,3 +101,43 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(FileNotFoundError):
         binding.lib()
+
+
+def test_dispatch_queries_need_no_gpu(lib, monkeypatch):
+    """Which kernel serves a shape, and how the channels are split between the two kernels, is
+    host logic: pinned here on the shapes of the benchmark configurations."""
+    from paper_2508_06753_b200 import binding as b
+    for name in ("W2A8_PREFILL", "W2A8_PF_SPLIT"):
+        monkeypatch.delenv(name, raising=False)
+    # few tokens: streaming kernel
+    for M in (1, 4, 16, 32, 63):
+        assert b.w2a8_kernel_for(M, 14336, 4096, 64) == "streaming"
+        assert b.w2a8_tensor_core_channels(M, 14336, 4096, 64) == 0
+    # prefill configuration: tensor-core kernel; a ragged last round of tiles is trimmed
+    assert b.w2a8_kernel_for(512, 14336, 4096, 64) == "tensor_core"
+    assert b.w2a8_tensor_core_channels(512, 14336, 4096, 64) == 111 * 128       # 444 tiles = 3 x 148
+    assert b.w2a8_tensor_core_channels(2048, 14336, 4096, 64) == 111 * 128      # 1776 tiles = 12 x 148
+    assert b.w2a8_tensor_core_channels(8192, 14336, 4096, 64) == 14336          # the rest would cost more than a round
+    assert b.w2a8_tensor_core_channels(2048, 4096, 14336, 64) == 4096
+    # too few output tiles for 148 SMs: streaming kernel even with many tokens
+    assert b.w2a8_kernel_for(128, 4096, 14336, 64) == "streaming"
+    assert b.w2a8_kernel_for(64, 4096, 4096, 64) == "streaming"
+    # shapes the tensor-core kernel does not tile
+    assert b.w2a8_kernel_for(512, 1040, 4096, 64) == "streaming"
+    assert b.w2a8_kernel_for(512, 4096, 4160, 64) == "streaming"
+    # switches
+    monkeypatch.setenv("W2A8_PREFILL", "0")
+    assert b.w2a8_kernel_for(2048, 14336, 4096, 64) == "streaming"
+    monkeypatch.setenv("W2A8_PREFILL", "2")
+    assert b.w2a8_kernel_for(64, 128, 256, 64) == "tensor_core"
+    assert b.w2a8_tensor_core_channels(512, 14336, 4096, 64) == 14336
+    monkeypatch.setenv("W2A8_PREFILL", "1")
+    monkeypatch.setenv("W2A8_PF_SPLIT", "0")
+    assert b.w2a8_tensor_core_channels(512, 14336, 4096, 64) == 14336
+    # the workspace covers the plan of the streamed remainder as well
+    monkeypatch.delenv("W2A8_PF_SPLIT")
+    with_split = b.w2a8_workspace_bytes(512, 14336, 4096, 64)
+    monkeypatch.setenv("W2A8_PF_SPLIT", "0")
+    assert with_split >= b.w2a8_workspace_bytes(512, 14336, 4096, 64) > 0
+    with pytest.raises(b.W2A8Error):
+        b.w2a8_kernel_for(4, 100, 4096, 64)
