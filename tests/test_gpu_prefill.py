@@ -88,13 +88,18 @@ def test_prefill_matches_streaming_path(gpu, monkeypatch):
     assert np.abs(y_tc - y_st).max() <= TOL * np.abs(y_st).max()
 
 
+@pytest.mark.parametrize("dispatch", ["as_benchmarked", "tensor_core_only"])
 @pytest.mark.parametrize("K,N", [(4096, 14336), (14336, 4096)])
-def test_prefill_full_size_sampled_rows(gpu, oracle, K, N):
+def test_prefill_full_size_sampled_rows(gpu, oracle, K, N, dispatch, monkeypatch):
     """Prefill configuration at full size (M = 2048, group 64): every channel of a sample of
     token rows -- first and last row of the first, a middle and the last token tile, plus a few
-    seeded ones -- against the reference."""
+    seeded ones -- against the reference.  "as_benchmarked" is the default dispatch, in which the
+    last 128 channels of 4096x14336 are computed by the streaming kernel."""
     torch, b = gpu
     M, g = 2048, 64
+    if dispatch == "as_benchmarked":
+        monkeypatch.delenv("W2A8_PREFILL", raising=False)
+        assert b.w2a8_tensor_core_channels(M, N, K, g) == (111 * 128 if N == 14336 else N)
     codes, s_w = synth.make_linear(4000 + K, K, N, g)
     bits = synth.activations_bf16(4000 + N, M, K)
     packed = b.w2_pack(_dev(torch, codes))
