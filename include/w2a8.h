@@ -92,7 +92,8 @@ int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, voi
 
 /*
  * Workspace size in bytes that w2a8_gemm / w2a8_gemm_partials need for this
- * problem (status word, split-K arrival counters and partial outputs).  Returns 0 for
+ * problem (status word, split-K arrival counters and partial outputs; the
+ * larger of what the kernels that may serve the shape need).  Returns 0 for
  * shapes that violate the shape rules.  The workspace must be zero-filled once
  * (w2a8_workspace_init) before its first use; the kernels leave it reusable.
  * One workspace serves any sequence of calls on one stream as long as it is at
@@ -130,6 +131,10 @@ int w2a8_workspace_status(const void *workspace, void *stream);
  * to be the faster one (M * N above about 0.95 million per round of 148
  * tiles); everything else takes the memory-bound streaming kernel (weights
  * read once per slab of up to 32 tokens).  w2a8_kernel_for reports the choice.
+ * A problem given to the tensor-core kernel may leave its last (at most
+ * eight) 128-channel tiles to the streaming kernel, as a second launch on the
+ * same stream (w2a8_tensor_core_channels); the result does not depend on it
+ * beyond fp32 summation order.
  */
 int w2a8_gemm(const int8_t *a, const float *a_scale, const uint32_t *packed,
               const float *w_scale, float *y, int M, int N, int K, int group,
