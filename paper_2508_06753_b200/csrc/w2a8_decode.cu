@@ -47,9 +47,16 @@ constexpr int kDecodeThreads = kDecodeWarps * 32;
 // Resident CTAs per SM the compiler must allow.  One slab: 8 (64 registers), which also lets
 // every 4-CTA cluster of a split-K launch be resident at once (clusters are placed inside one
 // GPC; with 7 per SM the last few clusters of a 1024-CTA grid waited for a second round).
+// RELAX instances (one or two slabs, fp32 scales, default grouping) are compiled for 7 CTAs per
+// SM instead: 72 registers, no pressure on the compiler for one slab and one wave instead of one
+// and a half for a two-slab grid of up to 1036 CTAs.  The launch code picks them for grids that
+// fit 7 per SM and do not need the eighth slot (measured: 4096x14336 at M = 4 5.39 -> 5.15 us, at
+// M = 16 9.64 -> 8.92 us; 4096x1024 2.33 -> 2.22 us; but 14336x4096 with its 1024-CTA cluster
+// grid 6.0 -> 8.3 us, which therefore stays on the 8-per-SM instance).
 #ifndef W2A8_MINB
 #define W2A8_MINB(MT) ((MT) == 1 ? 8 : 3)
 #endif
+constexpr int kRelaxedCtasPerSm = 7;
 constexpr int kRound = 4;                      // landing slots (cells) per warp
 
 struct DecodeParams {
@@ -338,8 +345,9 @@ __device__ __forceinline__ void compute_cell_a16(const DecodeParams &p, const ui
 // divisions and no 64-bit multiplies per cell.  Warps do not meet before the
 // final sum over the K-lanes.
 // A16: p.a holds the caller's bf16 activations (no quantiser, no token scale): compute_cell_a16.
-template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS, bool H16 = false, bool A16 = false>
-__global__ void __launch_bounds__(kDecodeThreads, W2A8_MINB(MT))
+template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS, bool H16 = false, bool A16 = false,
+          bool RELAX = false>
+__global__ void __launch_bounds__(kDecodeThreads, RELAX ? kRelaxedCtasPerSm : W2A8_MINB(MT))
 w2a8_decode_kernel(const DecodeParams p) {
     constexpr int KS = kDecodeWarps / TG;
     constexpr int kSlotBytes = 2 * 32 * 16;     // weights of one cell: two channels x 32 lanes x 16 B
@@ -794,8 +802,37 @@ static cudaError_t launch_decode_ring(const DecodeParams &p, dim3 grid, size_t s
                                  p.cluster ? (unsigned)p.chunks : 1u, p);
 }
 
+// RELAX instance of the default configuration (see kRelaxedCtasPerSm).
+template <int MT, int SPP, bool ONE>
+static cudaError_t launch_decode_relaxed(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, false, true>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    return launch_kernel_cluster(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, false, true>, grid,
+                                 dim3(kDecodeThreads), smem, st, pdl_enabled(),
+                                 p.cluster ? (unsigned)p.chunks : 1u, p);
+}
+
+// Whether the grid is better served by the 7-per-SM instance: it has to fit 7 per SM at once
+// (cluster grids: with room to spare, clusters are placed inside one GPC), and a two-slab grid
+// must be too large for the 4 per SM its roomier default instance gets.
+static bool prefer_relaxed(int mt, const DecodeParams &p, dim3 grid) {
+    if (env_int("W2A8_RELAX", 1) == 0 || mt > 2) return false;
+    const long long ctas = (long long)grid.x * grid.y * grid.z;
+    if (p.cluster) return mt == 1 && ctas <= 148ll * kRelaxedCtasPerSm / 2;
+    if (ctas > 148ll * kRelaxedCtasPerSm) return false;
+    return mt == 1 || ctas > 148ll * 4;
+}
+
 template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
 static cudaError_t launch_decode_inst(const DecodeParams &p, int ring, dim3 grid, size_t smem, cudaStream_t st) {
+    if constexpr (MT <= 2 && TG == 1 && !PARTIALS) {
+        if (ring == kRound && prefer_relaxed(MT, p, grid)) return launch_decode_relaxed<MT, SPP, ONE>(p, grid, smem, st);
+    }
     if (ring == 8) return launch_decode_ring<MT, SPP, TG, 8, ONE, PARTIALS>(p, grid, smem, st);
     return launch_decode_ring<MT, SPP, TG, kRound, ONE, PARTIALS>(p, grid, smem, st);
 }
