@@ -846,7 +846,9 @@ def prefill_probe(device, peaks, Ms=(512, 2048, 8192), reps=5):
                 out[label] = e0.elapsed_time(e1) / reps
             ops = 2.0 * M * N * K
             tops = ops / (out["gemm"] * 1e-3) / 1e12
-            rows.append({"shape": f"{K}x{N}", "M": M, "group": g, "ms_gemm": out["gemm"],
+            rows.append({"shape": f"{K}x{N}", "M": M, "group": g,
+                         "channels_on_tensor_cores": b.w2a8_tensor_core_channels(M, N, K, g),
+                         "ms_gemm": out["gemm"],
                          "ms_quantize_gemm": out["quantize+gemm"], "tops": tops,
                          "tops_with_quantize": ops / (out["quantize+gemm"] * 1e-3) / 1e12,
                          "frac_of_measured_int8_burst": tops / int8_peak_burst,
