@@ -34,8 +34,8 @@ CFG_INDEX = 1
 METRIC = "W2A8 GEMM HBM GB/s at M=1-16 (Llama-3-8B decoder-layer linears, M in {1,4,16}, group 64)"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode kernel on the
-# 4096x14336, M=1, group-64 GEMM (ncu capture summarised in profiles/decode_gate_m1_ncu.md);
-# the algorithmic bytes of that launch are 18,411,524.
+# 4096x14336, M=1, group-64 GEMM (ncu capture of one launch); the algorithmic bytes of that
+# launch are 18,411,524.
 NCU_TRAFFIC_BYTES_GATE_M1 = 18_378_752
 
 

@@ -21,9 +21,9 @@
  *       i.e. already in the order an int8 dot-product instruction wants.
  *       The concrete bit layout ("W2P") is this build's own and is written
  *       out below; the paper's AVX2 layout is not reproduced.
- *   ref_quantize : Sec. II-D, "multiply the entries with the inverse of the
- *       scales, then convert to int8", scale from the abs-max of the
- *       quantisation granule (here: one token = all K entries).
+ *   ref_quantize : Sec. II-D: scale from the abs-max of the quantisation
+ *       granule (here: one token = all K entries); every entry times the
+ *       inverse of that scale, rounded to nearest even, as int8.
  *   ref_partials : Sec. II-C microkernel result: int32 = sum of
  *       int8 activation x (2-bit weight as int8), exact.
  *   ref_gemm : Sec. II-D dequantisation: int32 -> float, times the product

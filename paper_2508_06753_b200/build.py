@@ -46,15 +46,23 @@ def build(force: bool = False, verbose: bool = False) -> str:
             if not force and not _stale():
                 return LIB
             tmp = LIB + f".tmp{os.getpid()}"
-            cmd = [_nvcc(), "-std=c++17", "-O3", "-lineinfo",
-                   "-gencode", "arch=compute_100a,code=sm_100a",
-                   "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
-                   "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-                   "-o", tmp] + sources()
+            common = [_nvcc(), "-std=c++17", "-O3", "-lineinfo",
+                      "-gencode", "arch=compute_100a,code=sm_100a",
+                      "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
             if verbose:
-                cmd.insert(1, "-Xptxas")
-                cmd.insert(2, "-v")
-            subprocess.run(cmd, check=True)
+                common[1:1] = ["-Xptxas", "-v"]
+            # one object per source file, compiled side by side, then one link
+            objdir = os.path.join(PKG, "build")
+            os.makedirs(objdir, exist_ok=True)
+            objs = [os.path.join(objdir, os.path.basename(src)[:-3] + f".{os.getpid()}.o") for src in sources()]
+            procs = [subprocess.Popen(common + ["-c", src, "-o", obj]) for src, obj in zip(sources(), objs)]
+            failed = [src for src, pr in zip(sources(), procs) if pr.wait() != 0]
+            if failed:
+                raise subprocess.CalledProcessError(1, "nvcc -c " + " ".join(failed))
+            subprocess.run(common[:1] + ["-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static",
+                                         "-o", tmp] + objs, check=True)
+            for obj in objs:
+                os.remove(obj)
             os.replace(tmp, LIB)        # atomic: nobody ever loads a half-written library
         finally:
             fcntl.flock(lock, fcntl.LOCK_UN)

@@ -12,6 +12,7 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   int group, const ShapeInfo &si, void *workspace, cudaStream_t st, bool h16, bool y16,
                   bool a16, int ldy);
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
+size_t decode_workspace_header_bytes(int M, int N, int K, const ShapeInfo &si);
 
 bool prefill_supported(int M, int N, int K, int group);
 bool prefill_preferred(int M, int N, int K, int group);
@@ -30,17 +31,45 @@ bool pdl_enabled() {
     return on;
 }
 
-int check_device() {
+int current_device() {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) return W2A8_ERR_CUDA;
-    static int cached_dev = -1, cached_status = 0;
-    if (dev == cached_dev) return cached_status;
-    int major = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
-        return W2A8_ERR_CUDA;
-    cached_status = (major == 10) ? W2A8_OK : W2A8_ERR_ARCH;
-    cached_dev = dev;
-    return cached_status;
+    return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
+namespace {
+struct DeviceInfo {
+    std::atomic<int> known{0};   // 0 = not looked up yet
+    int status = 0, sms = 0;
+};
+DeviceInfo g_devices[kMaxDevices];
+
+// Architecture check and SM count of the current device, looked up once per device.
+const DeviceInfo *device_info() {
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices) return nullptr;
+    DeviceInfo &d = g_devices[dev];
+    if (!d.known.load(std::memory_order_acquire)) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return nullptr;
+        // racing threads write the same values
+        d.status = (major == 10) ? W2A8_OK : W2A8_ERR_ARCH;
+        d.sms = sms > 0 ? sms : 1;
+        d.known.store(1, std::memory_order_release);
+    }
+    return &d;
+}
+}  // namespace
+
+int check_device() {
+    const DeviceInfo *d = device_info();
+    return d ? d->status : W2A8_ERR_CUDA;
+}
+
+int sm_count() {
+    const DeviceInfo *d = device_info();
+    return d ? d->sms : 148;
 }
 
 // ---- w2_pack ---------------------------------------------------------------------
@@ -323,22 +352,33 @@ int w2a8_tensor_core_channels(int M, int N, int K, int group) {
     return takes_tensor_core_kernel(M, N, K, group) ? tensor_core_channels(M, N, K, group) : 0;
 }
 
-// h16: w_scale holds binary16 values; y16 (with h16): y holds bf16 values.
-static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *packed,
-                       const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
-                       int group, void *workspace, size_t workspace_bytes, void *stream,
-                       bool h16 = false, bool y16 = false, bool a16 = false) {
+}  // extern "C"
+
+namespace w2a8 {
+// Bytes at the start of a workspace that have to be zero when a GEMM call starts (status word and
+// split-K arrival counters of whichever kernels serve the shape).  The kernels leave them zero.
+size_t gemm_header_bytes(int M, int N, int K, int group) {
     ShapeInfo si;
-    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
-    if (!aligned16(a) || !aligned16(packed) || (y && !aligned16(y)) ||
-        (w_scale && !aligned16(w_scale)) || (partials && !aligned16(partials)) ||
-        (a_scale && (reinterpret_cast<uintptr_t>(a_scale) & 3u)))
-        return W2A8_ERR_ALIGN;
-    const size_t need = w2a8_workspace_bytes(M, N, K, group);
-    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
-    if (int st = check_device()) return st;
-    // many tokens: tensor-core path (tcgen05); few tokens, shapes it does not tile, or too few
-    // output tiles to fill the GPU: streaming path
+    if (!shape_ok(M, N, K, group, &si)) return 0;
+    size_t need = decode_workspace_header_bytes(M, N, K, si);
+    if (takes_tensor_core_kernel(M, N, K, group)) {
+        const int n_tc = tensor_core_channels(M, N, K, group);
+        ShapeInfo rest;
+        if (n_tc < N && shape_ok(M, N - n_tc, K, group, &rest)) {
+            const size_t r = decode_workspace_header_bytes(M, N - n_tc, K, rest);
+            if (r > need) need = r;
+        }
+    }
+    return need;
+}
+
+// Pick the kernel(s) for a checked problem and enqueue them.  Many tokens: tensor-core path
+// (tcgen05); few tokens, shapes it does not tile, or too few output tiles to fill the GPU:
+// streaming path.  h16: w_scale holds binary16 values; y16 (with h16): y holds bf16 values;
+// a16: a holds bf16 activations.
+int gemm_dispatch(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
+                  void *y, int32_t *partials, int M, int N, int K, int group, const ShapeInfo &si,
+                  void *workspace, void *stream, bool h16, bool y16, bool a16) {
     if (!a16 && takes_tensor_core_kernel(M, N, K, group)) {
         // The tensor-core kernel takes the first n_tc channels; when a last round of a few tiles
         // would cost a whole round, the remaining channel tiles go to the streaming kernel in a
@@ -357,6 +397,26 @@ static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *pa
     }
     return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,
                          (cudaStream_t)stream, h16, y16, a16, N);
+}
+}  // namespace w2a8
+
+extern "C" {
+
+static int gemm_common(const int8_t *a, const float *a_scale, const uint32_t *packed,
+                       const void *w_scale, void *y, int32_t *partials, int M, int N, int K,
+                       int group, void *workspace, size_t workspace_bytes, void *stream,
+                       bool h16 = false, bool y16 = false, bool a16 = false) {
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
+    if (!aligned16(a) || !aligned16(packed) || (y && !aligned16(y)) ||
+        (w_scale && !aligned16(w_scale)) || (partials && !aligned16(partials)) ||
+        (a_scale && (reinterpret_cast<uintptr_t>(a_scale) & 3u)))
+        return W2A8_ERR_ALIGN;
+    const size_t need = w2a8_workspace_bytes(M, N, K, group);
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
+    if (int st = check_device()) return st;
+    return gemm_dispatch(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace, stream,
+                         h16, y16, a16);
 }
 
 int w2a16_gemm(const void *x_bf16, const uint32_t *packed, const float *w_scale, float *y, int M, int N,

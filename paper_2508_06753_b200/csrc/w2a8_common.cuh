@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "w2a8.h"
 
 namespace w2a8 {
@@ -54,6 +56,14 @@ __device__ __forceinline__ void promote2(float &acc0, float &acc1, int d0, int d
 // acquire), this CTA's rank, and a read of another CTA's shared memory.
 __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The two halves of a cluster barrier, for a phase whose only purpose is "every CTA of the
+// cluster has started": arrive early, wait late.
+__device__ __forceinline__ void cluster_arrive_relaxed() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
 }
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -169,5 +179,29 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
 
 bool pdl_enabled();
 int check_device();  // W2A8_OK or W2A8_ERR_ARCH / W2A8_ERR_CUDA
+
+// ---- per-device state -------------------------------------------------------
+// One process may drive several GPUs, and function attributes, the SM count and
+// the architecture check belong to a device, not to the process: everything that
+// is looked up once is kept per device ordinal.
+constexpr int kMaxDevices = 64;
+int current_device();   // ordinal of the current device, or -1
+int sm_count();         // multiprocessors of the current device (148 on B200), >= 1
+
+// Raise the dynamic shared-memory limit of `kernel` once per device.  `done` is a
+// table owned by the caller (one per kernel instantiation); two threads racing on
+// the same entry both make the (idempotent) call.
+struct PerDeviceFlags {
+    std::atomic<bool> done[kMaxDevices];
+};
+template <typename... KArgs>
+inline cudaError_t allow_dynamic_smem(void (*kernel)(KArgs...), PerDeviceFlags &flags, int bytes) {
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (flags.done[dev].load(std::memory_order_acquire)) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) flags.done[dev].store(true, std::memory_order_release);
+    return e;
+}
 
 }  // namespace w2a8

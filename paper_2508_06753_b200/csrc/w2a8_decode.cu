@@ -38,7 +38,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
-#include "w2a8_common.cuh"
+#include "w2a8_cell.cuh"
 
 namespace w2a8 {
 
@@ -80,175 +80,6 @@ struct DecodeParams {
     int ldy;              // elements between consecutive token rows of y (>= N)
     int y16;              // 16-bit instances only: y holds bf16 instead of fp32
 };
-
-// ---- PTX wrappers ------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-// per-thread asynchronous copies into shared memory
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-// n is a constant after unrolling
-__device__ __forceinline__ void cp_async_wait_pending(int n) {
-    switch (n) {
-        case 0: cp_async_wait_group<0>(); break;
-        case 1: cp_async_wait_group<1>(); break;
-        case 2: cp_async_wait_group<2>(); break;
-        case 3: cp_async_wait_group<3>(); break;
-        case 4: cp_async_wait_group<4>(); break;
-        case 5: cp_async_wait_group<5>(); break;
-        case 6: cp_async_wait_group<6>(); break;
-        default: cp_async_wait_group<7>(); break;
-    }
-}
-
-// Optional timeline trace (build with -DW2A8_TRACE): every warp records the
-// global timer at a few points of the kernel into a caller-provided buffer.
-#ifdef W2A8_TRACE
-__device__ unsigned long long *g_trace = nullptr;
-__device__ const float *g_trace_y0 = nullptr;     // launches are told apart by their output pointer:
-__device__ unsigned long long g_trace_ystride = 1;   // launch id = (y - y0) / ystride
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long v;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(v));
-    return v;
-}
-#define W2A8_TRACE_POINT(i)                                                                      \
-    do {                                                                                         \
-        if (g_trace && (threadIdx.x & 31) == 0) {                                                \
-            const size_t launch = (size_t)(p.y - g_trace_y0) / g_trace_ystride;                  \
-            const size_t ctas = (size_t)gridDim.x * gridDim.y * gridDim.z;                       \
-            g_trace[((launch * ctas + ((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + \
-                      blockIdx.x) * kDecodeWarps + (threadIdx.x >> 5)) * 8 + (i)] = global_ns(); \
-        }                                                                                        \
-    } while (0)
-#else
-#define W2A8_TRACE_POINT(i) do { } while (0)
-#endif
-
-__device__ __forceinline__ uint4 ld_act16(const int8_t *p) {
-    // plain (L1-allocating) load: the activations are written by the previous kernel of the
-    // stream and are only read after the wait for it, so the read-only path is not used
-    uint4 v;
-    asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
-// One cell: 4 slices x (unpack, 2 MMAs per token slab, promotion at group ends).
-// w0s/w1s: this lane's four words (one per slice) of channels n0+gq and n0+gq+8;
-// sc0/sc1: the cell's scales of the same channels (shared memory, 16 bytes each);
-// brow[mt]: this lane's 16 activation bytes of slice 0 of the cell, token row of slab mt.
-// H16: the scales in shared memory are IEEE binary16 (2 bytes each) instead of fp32.
-template <int MT, int SPP, bool ONE, bool PARTIALS, bool FULL, bool H16>
-__device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32_t (&w0s)[4],
-                                             const uint32_t (&w1s)[4], const unsigned char *sc0,
-                                             const unsigned char *sc1,
-                                             const int8_t *const (&brow)[MT], int kb, int n0, int m0,
-                                             int gq, int t, float (&acc)[MT][4]) {
-    // FULL: the block has all four slices (always, except possibly the last block of K)
-    const int R = FULL ? 4 : p.tail_slices;
-    const int magic[4] = {kMagicInt, kMagicInt, kMagicInt, kMagicInt};
-    int D[MT][4];   // int32 accumulators of the current group; a group never outlives a cell
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) D[mt][i] = kMagicInt;
-    float s0s[4 / SPP], s1s[4 / SPP];
-    if constexpr (!PARTIALS && H16) {
-        if constexpr (SPP == 4) {
-            s0s[0] = __half2float(*reinterpret_cast<const __half *>(sc0));
-            s1s[0] = __half2float(*reinterpret_cast<const __half *>(sc1));
-        } else if constexpr (SPP == 2) {
-            const float2 v0 = __half22float2(*reinterpret_cast<const __half2 *>(sc0));
-            const float2 v1 = __half22float2(*reinterpret_cast<const __half2 *>(sc1));
-            s0s[0] = v0.x; s0s[1] = v0.y; s1s[0] = v1.x; s1s[1] = v1.y;
-        } else {
-            const uint2 r0 = *reinterpret_cast<const uint2 *>(sc0), r1 = *reinterpret_cast<const uint2 *>(sc1);
-            const float2 v0 = __half22float2(*reinterpret_cast<const __half2 *>(&r0.x));
-            const float2 v1 = __half22float2(*reinterpret_cast<const __half2 *>(&r0.y));
-            const float2 v2 = __half22float2(*reinterpret_cast<const __half2 *>(&r1.x));
-            const float2 v3 = __half22float2(*reinterpret_cast<const __half2 *>(&r1.y));
-            s0s[0] = v0.x; s0s[1] = v0.y; s0s[2] = v1.x; s0s[3] = v1.y;
-            s1s[0] = v2.x; s1s[1] = v2.y; s1s[2] = v3.x; s1s[3] = v3.y;
-        }
-    } else if constexpr (!PARTIALS) {
-        if constexpr (SPP == 4) {
-            s0s[0] = *reinterpret_cast<const float *>(sc0);
-            s1s[0] = *reinterpret_cast<const float *>(sc1);
-        } else if constexpr (SPP == 2) {
-            const float2 v0 = *reinterpret_cast<const float2 *>(sc0);
-            const float2 v1 = *reinterpret_cast<const float2 *>(sc1);
-            s0s[0] = v0.x; s0s[1] = v0.y; s1s[0] = v1.x; s1s[1] = v1.y;
-        } else {
-            const float4 v0 = *reinterpret_cast<const float4 *>(sc0);
-            const float4 v1 = *reinterpret_cast<const float4 *>(sc1);
-            s0s[0] = v0.x; s0s[1] = v0.y; s0s[2] = v0.z; s0s[3] = v0.w;
-            s1s[0] = v1.x; s1s[1] = v1.y; s1s[2] = v1.z; s1s[3] = v1.w;
-        }
-    }
-#pragma unroll
-    for (int s = 0; s < 4; ++s) {
-        if (s < R) {
-            const uint32_t w0 = w0s[s], w1 = w1s[s];
-            const uint32_t a0 = lane_codes(w0, 0), a1 = lane_codes(w1, 0);
-            const uint32_t a2 = lane_codes(w0, 1), a3 = lane_codes(w1, 1);
-            const uint32_t a4 = lane_codes(w0, 2), a5 = lane_codes(w1, 2);
-            const uint32_t a6 = lane_codes(w0, 3), a7 = lane_codes(w1, 3);
-            const bool first = (s % SPP) == 0;
-            const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                const uint4 b = ld_act16(brow[mt] + s * kSliceK);
-                if (first) mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, magic);
-                else       mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, D[mt]);
-                mma_s8_16x8x32(D[mt], a4, a5, a6, a7, b.z, b.w, D[mt]);
-                if (last) {
-                    if constexpr (PARTIALS) {
-                        const int gi = (SPP == 1) ? 4 * kb + s
-                                     : (SPP == 2) ? 2 * kb + (s >> 1)
-                                                  : (int)(((long long)kb * kBlockK) / p.group);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int mm = m0 + 8 * mt + 2 * t + (i & 1);
-                            const int nn = n0 + gq + 8 * (i >> 1);
-                            if (mm < p.M)
-                                atomicAdd(p.partials + ((size_t)mm * p.N + nn) * p.G + gi,
-                                          (D[mt][i] - kMagicInt) >> 6);
-                        }
-                    } else {
-                        const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
-                        if constexpr (ONE) {
-                            acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
-                            acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
-                        } else if constexpr (MT == 1) {
-                            // packed fp32 pairs: measured faster for one slab, slower for more
-                            promote2(acc[mt][0], acc[mt][1], D[mt][0], D[mt][1], s0);
-                            promote2(acc[mt][2], acc[mt][3], D[mt][2], D[mt][3], s1);
-                        } else {
-                            acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
-                            acc[mt][1] = fmaf(s0, __int_as_float(D[mt][1]) - kMagicFloat, acc[mt][1]);
-                            acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
-                            acc[mt][3] = fmaf(s1, __int_as_float(D[mt][3]) - kMagicFloat, acc[mt][3]);
-                        }
-                    }
-                }
-            }
-        }
-    }
-}
 
 // The same cell for 16-bit activations and no activation quantiser (the alternative kernel of
 // Sec. II): the codes become the bf16 values q - 2 (exact), the activations are the caller's
@@ -368,7 +199,10 @@ w2a8_decode_kernel(const DecodeParams p) {
     const int nb = kb_end - kb_begin;
     const int m0 = blockIdx.z * (8 * MT);
     const int mrows = min(8 * MT, p.M - m0);
-    W2A8_TRACE_POINT(0);
+    // Split-K in a cluster ends with stores into the shared memory of the cluster's first CTA,
+    // which may only be touched once that CTA is known to be running: every CTA arrives here and
+    // waits just before its first remote store (the wait costs nothing by then).
+    if (p.cluster) cluster_arrive_relaxed();
 
     // This warp's cells: the chunk is cut into KS runs of consecutive blocks, one per K-lane; cell c
     // is block kb0 + c of tile tile0 + tl (at most RING of them).  Consecutive blocks matter for the
@@ -484,9 +318,7 @@ w2a8_decode_kernel(const DecodeParams p) {
             }
         }
     }
-    W2A8_TRACE_POINT(1);
     pdl_wait();
-    W2A8_TRACE_POINT(2);
 
     float acc[MT][4];
 #pragma unroll
@@ -540,7 +372,6 @@ w2a8_decode_kernel(const DecodeParams p) {
                                                              sc1 + tail_cell * kScaleBytes, bc, kb0 + tail_cell,
                                                              n0, m0, gq, t, acc);
     }
-    W2A8_TRACE_POINT(5);
 
     if constexpr (!PARTIALS) {
         // ---- sum the K-lanes of each tile in a fixed order -----------------------
@@ -604,7 +435,6 @@ w2a8_decode_kernel(const DecodeParams p) {
                 int mm, nn;
                 if (locate(e, mm, nn)) store_y(mm, nn, cta_sum(e));
             }
-            W2A8_TRACE_POINT(6);
         } else if (p.cluster) {
             // ---- split-K inside a thread-block cluster: the chunks of a tile are the CTAs of one
             //      cluster.  Every CTA writes its sums into the receive buffer of rank 0 (remote
@@ -612,12 +442,12 @@ w2a8_decode_kernel(const DecodeParams p) {
             const uint32_t recv_u32 = smem_u32(smem + kDecodeWarps * kWarpBytes);
             const float *recv = reinterpret_cast<const float *>(smem + kDecodeWarps * kWarpBytes);
             const uint32_t rank = cluster_ctarank();
+            cluster_wait();            // all CTAs of the cluster have started (arrive at kernel entry)
             for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
                 int mm, nn;
                 if (locate(e, mm, nn)) st_cluster_f32(recv_u32 + (rank * kElems + e) * 4, 0, cta_sum(e));
             }
             cluster_sync();
-            W2A8_TRACE_POINT(6);
             if (rank != 0) return;
             for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
                 int mm, nn;
@@ -627,7 +457,6 @@ w2a8_decode_kernel(const DecodeParams p) {
                     store_y(mm, nn, v);
                 }
             }
-            W2A8_TRACE_POINT(7);
         } else {
             // ---- split-K through the workspace: the last CTA to arrive sums the partial outputs
             //      chunk by chunk ------------------------------------------------------------------
@@ -635,7 +464,6 @@ w2a8_decode_kernel(const DecodeParams p) {
                 int mm, nn;
                 if (locate(e, mm, nn)) __stcg(p.ws + chunk * MN + (size_t)mm * p.N + nn, cta_sum(e));
             }
-            W2A8_TRACE_POINT(6);
             __threadfence();
             __syncthreads();
             unsigned *counter = p.counters + (size_t)blockIdx.z * ntiles + tile0;
@@ -652,20 +480,9 @@ w2a8_decode_kernel(const DecodeParams p) {
                 }
             }
             if (threadIdx.x == 0) *counter = 0u;   // leave the workspace reusable
-            W2A8_TRACE_POINT(7);
         }
     }
 }
-
-#ifdef W2A8_TRACE
-extern "C" int w2a8_debug_set_trace(void *buffer, const float *y0, unsigned long long ystride) {
-    unsigned long long *b = reinterpret_cast<unsigned long long *>(buffer);
-    if (cudaMemcpyToSymbol(g_trace, &b, sizeof(b)) != cudaSuccess) return W2A8_ERR_CUDA;
-    if (cudaMemcpyToSymbol(g_trace_y0, &y0, sizeof(y0)) != cudaSuccess) return W2A8_ERR_CUDA;
-    if (ystride == 0) ystride = 1;
-    return cudaMemcpyToSymbol(g_trace_ystride, &ystride, sizeof(ystride)) == cudaSuccess ? 0 : W2A8_ERR_CUDA;
-}
-#endif
 
 // ---- host side -----------------------------------------------------------------
 int env_int(const char *name, int dflt);
@@ -704,7 +521,7 @@ static DecodePlan decode_plan_mt(int M, int N, int K, const ShapeInfo &si, int m
         // warp) as long as all CTAs are still resident at once (8 per SM for one slab, 4 for
         // wider slabs); beyond that the extra round of CTAs costs more than the split gains.
         const int min_warps = env_int("W2A8_MIN_WARPS", 2000);
-        const long long resident = 148ll * (mt == 1 ? 8 : 4);
+        const long long resident = (long long)sm_count() * (mt == 1 ? 8 : 4);
         auto ctas = [&](int c) { return (long long)pl.groups * pl.slabs * c; };
         while ((ctas(chunks) * kDecodeWarps < min_warps || ctas(chunks * 2) <= resident) &&
                (si.blocks / (chunks * 2)) >= ks)
@@ -738,7 +555,7 @@ static DecodePlan decode_plan_uncached(int M, int N, int K, const ShapeInfo &si,
     else if (M <= 32) widest = 2;
     else { const int slabs = (M + 31) / 32; widest = ((M + slabs - 1) / slabs + 7) / 8; }
     if (widest == 1) return decode_plan_mt(M, N, K, si, 1, h16);
-    constexpr long long kResidentCtas = 148 * 8;
+    const long long kResidentCtas = (long long)sm_count() * 8;
     const DecodePlan narrow = decode_plan_mt(M, N, K, si, 1, h16);
     if ((long long)narrow.groups * narrow.chunks * narrow.slabs <= kResidentCtas) return narrow;
     return decode_plan_mt(M, N, K, si, widest, h16);
@@ -757,14 +574,16 @@ static uint64_t env_fingerprint() {
 }
 
 static DecodePlan decode_plan(int M, int N, int K, const ShapeInfo &si, bool h16 = false) {
-    struct Key { int M, N, K, G, h16; uint64_t env; };
-    thread_local Key key = {0, 0, 0, 0, 0, 0};
+    struct Key { int M, N, K, G, h16, dev; uint64_t env; };
+    thread_local Key key = {0, 0, 0, 0, 0, -2, 0};
     thread_local DecodePlan cached;
     const uint64_t env = env_fingerprint();
-    if (key.M == M && key.N == N && key.K == K && key.G == si.G && key.h16 == (int)h16 && key.env == env)
+    const int dev = current_device();    // the plan depends on the SM count of the device
+    if (key.M == M && key.N == N && key.K == K && key.G == si.G && key.h16 == (int)h16 && key.dev == dev &&
+        key.env == env)
         return cached;
     cached = decode_plan_uncached(M, N, K, si, h16);
-    key = {M, N, K, si.G, (int)h16, env};
+    key = {M, N, K, si.G, (int)h16, dev, env};
     return cached;
 }
 
@@ -790,13 +609,8 @@ size_t decode_workspace_header_bytes(int M, int N, int K, const ShapeInfo &si) {
 
 template <int MT, int SPP, int TG, int RING, bool ONE, bool PARTIALS>
 static cudaError_t launch_decode_ring(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
-    static bool configured = false;   // one attribute call per instantiation and process
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, TG, RING, ONE, PARTIALS>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDeviceFlags configured;   // per kernel instantiation
+    if (cudaError_t e = allow_dynamic_smem(w2a8_decode_kernel<MT, SPP, TG, RING, ONE, PARTIALS>, configured, 200 * 1024)) return e;
     return launch_kernel_cluster(w2a8_decode_kernel<MT, SPP, TG, RING, ONE, PARTIALS>, grid,
                                  dim3(kDecodeThreads), smem, st, pdl_enabled(),
                                  p.cluster ? (unsigned)p.chunks : 1u, p);
@@ -805,13 +619,8 @@ static cudaError_t launch_decode_ring(const DecodeParams &p, dim3 grid, size_t s
 // RELAX instance of the default configuration (see kRelaxedCtasPerSm).
 template <int MT, int SPP, bool ONE>
 static cudaError_t launch_decode_relaxed(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, false, true>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDeviceFlags configured;   // per kernel instantiation
+    if (cudaError_t e = allow_dynamic_smem(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, false, true>, configured, 200 * 1024)) return e;
     return launch_kernel_cluster(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, false, true>, grid,
                                  dim3(kDecodeThreads), smem, st, pdl_enabled(),
                                  p.cluster ? (unsigned)p.chunks : 1u, p);
@@ -823,9 +632,10 @@ static cudaError_t launch_decode_relaxed(const DecodeParams &p, dim3 grid, size_
 static bool prefer_relaxed(int mt, const DecodeParams &p, dim3 grid) {
     if (env_int("W2A8_RELAX", 1) == 0 || mt > 2) return false;
     const long long ctas = (long long)grid.x * grid.y * grid.z;
-    if (p.cluster) return mt == 1 && ctas <= 148ll * kRelaxedCtasPerSm / 2;
-    if (ctas > 148ll * kRelaxedCtasPerSm) return false;
-    return mt == 1 || ctas > 148ll * 4;
+    const long long sms = sm_count();
+    if (p.cluster) return mt == 1 && ctas <= sms * kRelaxedCtasPerSm / 2;
+    if (ctas > sms * kRelaxedCtasPerSm) return false;
+    return mt == 1 || ctas > sms * 4;
 }
 
 template <int MT, int SPP, int TG, bool ONE, bool PARTIALS>
@@ -840,13 +650,8 @@ static cudaError_t launch_decode_inst(const DecodeParams &p, int ring, dim3 grid
 // 16-bit instances (binary16 scales, fp32 or bf16 result): default tile grouping and slot count.
 template <int MT, int SPP, bool ONE>
 static cudaError_t launch_decode_h16(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, true>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDeviceFlags configured;   // per kernel instantiation
+    if (cudaError_t e = allow_dynamic_smem(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, true>, configured, 200 * 1024)) return e;
     return launch_kernel_cluster(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, true>, grid,
                                  dim3(kDecodeThreads), smem, st, pdl_enabled(),
                                  p.cluster ? (unsigned)p.chunks : 1u, p);
@@ -855,13 +660,8 @@ static cudaError_t launch_decode_h16(const DecodeParams &p, dim3 grid, size_t sm
 // 16-bit-activation instances (bf16 x, fp32 scales, fp32 result): default grouping and slots.
 template <int MT, int SPP, bool ONE>
 static cudaError_t launch_decode_a16(const DecodeParams &p, dim3 grid, size_t smem, cudaStream_t st) {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, true>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDeviceFlags configured;   // per kernel instantiation
+    if (cudaError_t e = allow_dynamic_smem(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, true>, configured, 200 * 1024)) return e;
     return launch_kernel_cluster(w2a8_decode_kernel<MT, SPP, 1, kRound, ONE, false, false, true>, grid,
                                  dim3(kDecodeThreads), smem, st, pdl_enabled(),
                                  p.cluster ? (unsigned)p.chunks : 1u, p);

@@ -169,27 +169,6 @@ __host__ __device__ constexpr uint32_t pf_instr_desc(int m, int n) {
          | ((uint32_t)(m >> 4) << 24);    // M / 16
 }
 
-// Optional timeline trace (build with -DW2A8_TRACE): CTA (0,0) records the global
-// timer per role and iteration: slot = role * 4096 + index * 4 + point.
-#ifdef W2A8_TRACE
-__device__ unsigned long long *g_pf_trace = nullptr;   // 5 roles x 4096 slots
-__device__ __forceinline__ void pf_trace(int role, int idx, int point) {
-    if (g_pf_trace && blockIdx.x == 0 && idx < 1024) {
-        unsigned long long v;
-        if (role >= 3) v = (unsigned long long)clock64();      // SM cycles for the drain and MMA-group roles
-        else asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(v));
-        g_pf_trace[role * 4096 + idx * 4 + point] = v;
-    }
-}
-extern "C" int w2a8_debug_set_prefill_trace(void *buffer) {
-    unsigned long long *b = reinterpret_cast<unsigned long long *>(buffer);
-    return cudaMemcpyToSymbol(g_pf_trace, &b, sizeof(b)) == cudaSuccess ? 0 : W2A8_ERR_CUDA;
-}
-#define PF_TRACE(role, idx, point) pf_trace(role, idx, point)
-#else
-#define PF_TRACE(role, idx, point) do { } while (0)
-#endif
-
 // H16: w_scale points at IEEE binary16 values; the result is fp32 or, with p.y16, bf16.
 template <bool PARTIALS, bool H16>
 __global__ void __launch_bounds__(kPfThreads, 1)
@@ -253,15 +232,13 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             int s = 0;
             uint32_t full_parity = 0;
             int unit0 = 0;                  // units of the tiles before this one
-            int trace_it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
                 int pos = 0;                // 64-k slices already issued in the current group
                 int group_idx = 0;          // scale groups of this tile completed so far
-                for (int it = 0; it < nstages && ok; ++it, ++trace_it) {
+                for (int it = 0; it < nstages && ok; ++it) {
                     ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
                     if (!ok) break;
-                    if (mma_id == 1) PF_TRACE(1, trace_it, 0);
                     pf_tc_fence_after();
                     const uint64_t stage_off = (uint64_t)((uint32_t)(s * kPfStageBytes) >> 4);
 #pragma unroll
@@ -293,7 +270,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         }
                     }
                     pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
-                    if (mma_id == 1) PF_TRACE(1, trace_it, 1);
                     if (++s == kPfStages) { s = 0; full_parity ^= 1u; }
                 }
             }
@@ -314,11 +290,11 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         };
         uint4 w_nxt[kUnits];
         if ((int)blockIdx.x < ntiles) request(w_nxt, blockIdx.x, 0);
-        int s = 0, round = 0, trace_it = 0;
+        int s = 0, round = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
             const int m0 = (tile % tiles_m) * kPfBN;
-            for (int it = 0; it < nstages; ++it, ++trace_it) {
+            for (int it = 0; it < nstages; ++it) {
                 uint4 w[kUnits];
 #pragma unroll
                 for (int i = 0; i < kUnits; ++i) w[i] = w_nxt[i];
@@ -336,7 +312,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
                     pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
                     pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
-                    PF_TRACE(2, trace_it, 0);
                 }
                 unsigned char *a_stage = smem_gen + s * kPfStageBytes;
 #pragma unroll
@@ -356,7 +331,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
                 __syncwarp();
                 if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full[s]));
-                if (warp == 2 && lane == 0) PF_TRACE(2, trace_it, 1);
                 if (++s == kPfStages) { s = 0; ++round; }
             }
         }
@@ -368,7 +342,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         const uint32_t tlane = tmem_base + ((uint32_t)(q4 * 32) << 16) + col0;
         bool ok = true;
         int unit0 = 0;                              // units of the tiles before this one
-        int trace_g = 0;
         for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
             const int n = (tile / tiles_m) * kPfBM + ch;
             const int m0 = (tile % tiles_m) * kPfBN;
@@ -439,7 +412,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     const int buf = 2 * (unit & 1) + (gi & 1);
                     const float sc = sc_cur[u];
                     pf_tmem_ld_wait();                     // first half of group gi is in v0
-                    if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, trace_g + gi, 0);
                     pf_tmem_ld32(tlane + buf * kPfBN + 32, v1);
                     if (PARTIALS) {
 #pragma unroll
@@ -458,7 +430,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         __syncwarp();
                         if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[unit & 1]));
                     }
-                    if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, trace_g + gi, 1);
                     if (gi + 1 < ngroups) {                // request the first half of the next group
                         const int nunit = unit0 + ((gi + 1) >> 1);
                         if (((gi + 1) & 1) == 0) {         // it opens a new unit: wait for its MMAs
@@ -479,11 +450,9 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         for (int j = 0; j < 32; j += 2)
                             pf_fma2(acc[32 + j], acc[32 + j + 1], (float)v1[j], (float)v1[j + 1], sc);
                     }
-                    if (warp == 2 + kPfUnpackWarps && lane == 0) PF_TRACE(3, trace_g + gi, 2);
                 }
             }
             pf_tmem_ld_wait();
-            trace_g += ngroups;
             if (!PARTIALS && ok) {
 #pragma unroll
                 for (int j = 0; j < kPfDrainCols; ++j) {
@@ -543,12 +512,13 @@ bool prefill_supported(int M, int N, int K, int group) {
 bool prefill_preferred(int M, int N, int K, int group) {
     (void)K; (void)group;
     const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
-    const long long rounds = (tiles + 147) / 148;
+    const long long sms = sm_count();
+    const long long rounds = (tiles + sms - 1) / sms;
     return (long long)M * N > rounds * 950000ll;
 }
 
 // How many of the N channels the tensor-core kernel should take when the rest may go to the
-// streaming kernel.  Tiles are handed out in rounds of 148; a last round with a handful of tiles
+// streaming kernel.  Tiles are handed out in rounds of one tile per SM (148 on B200); a last round with a handful of tiles
 // costs as much as a full one (4096x14336 at M = 512: 448 tiles = 3 rounds + 4 tiles).  Tiles are
 // ordered channel tile first, so giving the last few channel tiles (at most eight) to the
 // streaming kernel can remove that round.  Same cost model as prefill_preferred, plus 2 us for
@@ -556,10 +526,11 @@ bool prefill_preferred(int M, int N, int K, int group) {
 int prefill_channel_split(int M, int N, int K, int group) {
     (void)group;
     const int ct = N / kPfBM, tiles_m = (M + kPfBN - 1) / kPfBN;
+    const long long sms = sm_count();
     double best = 1e30;
     int best_ct = ct;
     for (int c = ct; c >= 1 && c >= ct - 8; --c) {
-        const long long rounds = ((long long)c * tiles_m + 147) / 148;
+        const long long rounds = ((long long)c * tiles_m + sms - 1) / sms;
         double t = (double)rounds * K * 7.0e-9;
         if (c < ct) t += 2.0e-6 + 8.0e-15 * (double)M * (double)(ct - c) * kPfBM * (double)K;
         if (t < best * 0.97) { best = t; best_ct = c; }      // a split has to pay by 3 % or more
@@ -592,22 +563,12 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
     p.words_per_row = K / 16;
     p.slices_per_group = group / 64;
     const size_t smem = (size_t)kPfStages * kPfStageBytes + 1024;
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
-            sm_count = 148;
-    }
     const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
-    dim3 grid((unsigned)(tiles < sm_count ? tiles : sm_count));   // persistent CTAs, one per SM
-    static bool configured[3] = {false, false, false};
+    const int sms = sm_count();
+    dim3 grid((unsigned)(tiles < sms ? tiles : sms));   // persistent CTAs, one per SM
+    static PerDeviceFlags configured[3];
     auto launch = [&](auto kernel, int slot) -> bool {
-        if (!configured[slot]) {
-            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-                return false;
-            configured[slot] = true;
-        }
+        if (allow_dynamic_smem(kernel, configured[slot], (int)smem) != cudaSuccess) return false;
         kernel<<<grid, kPfThreads, smem, st>>>(map, p);
         return true;
     };

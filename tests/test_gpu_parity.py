@@ -7,6 +7,7 @@ import os
 import numpy as np
 import pytest
 
+from conftest import Guarded
 from paper_2508_06753_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -114,16 +115,26 @@ def _problem(seed, M, N, K, group, ternary=False, frac=0.0):
 
 
 def _run_gpu(torch, b, codes, s_w, bits, g, want_partials=True):
+    """The hot path through the C ABI.  Outputs, int32 sums and the workspace sit between canary
+    words, checked after the calls: nothing may be written outside them."""
     M, K = bits.shape
     N = codes.shape[0]
     packed = b.w2_pack(_dev(torch, codes))
     a, s_a = b.a8_quantize(_bf16_dev(torch, bits))
-    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
-    y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
-    y2 = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
-    P = b.w2a8_gemm_partials(a, packed, g, ws) if want_partials else None
+    ws_bytes = (b.w2a8_workspace_bytes(M, N, K, g) + 15) // 16 * 16
+    gws = Guarded(torch, (max(ws_bytes, 256),), torch.uint8)
+    b.w2a8_workspace_init(gws.view)
+    gy = Guarded(torch, (M, N), torch.float32, float("nan"))
+    gy2 = Guarded(torch, (M, N), torch.float32, float("nan"))
+    y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, gws.view, gy.view)
+    y2 = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, gws.view, gy2.view)
+    gp = Guarded(torch, (M, N, K // g), torch.int32) if want_partials else None
+    P = b.w2a8_gemm_partials(a, packed, g, gws.view, gp.view) if want_partials else None
     torch.cuda.synchronize()
-    assert b.w2a8_workspace_status(ws) == 0
+    assert b.w2a8_workspace_status(gws.view) == 0
+    gy.check("y"), gy2.check("y"), gws.check("workspace")
+    if gp is not None:
+        gp.check("partials")
     assert torch.equal(y, y2), "repeated calls must be bitwise equal"
     return (a.cpu().numpy(), s_a.cpu().numpy(), y.cpu().numpy(),
             None if P is None else P.cpu().numpy())
@@ -230,6 +241,44 @@ def test_zero_token_row_and_zero_weights(gpu, oracle):
     assert ok, worst
 
 
+def test_second_device_after_first(gpu, oracle):
+    """One process, two GPUs: function attributes, the SM count and the architecture check are
+    kept per device, so the same shapes run on device 1 after device 0 (no peer access, no
+    collectives).  Skipped where only one device is visible."""
+    torch, b = gpu
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs two visible devices")
+    for M, N, K, g in [(1, 2048, 2048, 64), (16, 256, 4096, 64), (1, 256, 8192, 64), (256, 4096, 1024, 64)]:
+        codes, s_w, bits, g = _problem(M + N, M, N, K, g)
+        a_ref, s_ref = oracle.quantize(bits)
+        y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+        for dev in (0, 1):
+            with torch.cuda.device(dev):
+                d = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(f"cuda:{dev}")
+                packed = b.w2_pack(d(codes))
+                a, s_a = b.a8_quantize(d(bits.view(np.int16)).view(torch.bfloat16))
+                ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g), device=f"cuda:{dev}")
+                y = b.w2a8_gemm(a, s_a, packed, d(s_w), g, ws)
+                torch.cuda.synchronize()
+                assert b.w2a8_workspace_status(ws) == 0
+                ok, worst = _row_err_ok(y.cpu().numpy(), y_ref)
+                assert ok, (dev, worst)
+
+
+def test_status_word_read_back(gpu):
+    """The device status word at the start of a workspace is what w2a8_workspace_status returns:
+    the code a kernel leaves when one of its bounded waits gives up (-7) is written here from the
+    host -- no kernel is made to time out -- and read back; a fresh workspace reads 0."""
+    torch, b = gpu
+    ws = b.new_workspace(4096)
+    assert b.w2a8_workspace_status(ws) == 0
+    ws[:4].copy_(torch.tensor([-7], dtype=torch.int32).view(torch.uint8))
+    assert b.w2a8_workspace_status(ws) == -7
+    assert "wait" in b.status_string(-7)
+    b.w2a8_workspace_init(ws)
+    assert b.w2a8_workspace_status(ws) == 0
+
+
 @pytest.mark.parametrize("M,pinned", [(4, True), (4, False), (1, True), (40, True)])
 def test_linear_host_end_to_end(gpu, oracle, M, pinned):
     """Host buffers in, host buffers out: page-locked buffers with few tokens are read and
@@ -280,7 +329,7 @@ def test_pdl_off_matches(gpu, oracle):
 
 # ---------------------------------------------- full-size shapes, sampled channels
 FULL = [
-    (1, "8b"), (16, "8b"), (8, "8b-ternary"), (32, "70b"),
+    (1, "8b"), (4, "8b"), (16, "8b"), (1, "8b-ternary"), (8, "8b-ternary"), (1, "70b"), (8, "70b"), (32, "70b"),
 ]
 
 

@@ -88,34 +88,61 @@ def test_prefill_matches_streaming_path(gpu, monkeypatch):
     assert np.abs(y_tc - y_st).max() <= TOL * np.abs(y_st).max()
 
 
-@pytest.mark.parametrize("dispatch", ["as_benchmarked", "tensor_core_only"])
-@pytest.mark.parametrize("K,N", [(4096, 14336), (14336, 4096)])
-def test_prefill_full_size_sampled_rows(gpu, oracle, K, N, dispatch, monkeypatch):
-    """Prefill configuration at full size (M = 2048, group 64): every channel of a sample of
-    token rows -- first and last row of the first, a middle and the last token tile, plus a few
-    seeded ones -- against the reference.  "as_benchmarked" is the default dispatch, in which the
-    last 128 channels of 4096x14336 are computed by the streaming kernel."""
+def _sample_rows(M, seed, count=128):
+    """First and last row of the first, a middle and the last 128-token tile, plus seeded rows."""
+    mid = (M // 128 // 2) * 128
+    fixed = [0, 127, mid, mid + 127, M - 128, M - 1]
+    extra = [int(r) for r in np.random.default_rng(seed).choice(M, size=count, replace=False)]
+    return sorted(set(fixed + extra))
+
+
+FULL_SIZE = [(M, K, N, d) for M in (512, 2048, 8192) for K, N in ((4096, 14336), (14336, 4096))
+             for d in (("as_benchmarked", "tensor_core_only") if M == 2048 else ("as_benchmarked",))]
+
+
+@pytest.mark.parametrize("M,K,N,dispatch", FULL_SIZE)
+def test_prefill_full_size_sampled_rows(gpu, oracle, M, K, N, dispatch, monkeypatch):
+    """Prefill configuration at full size (group 64) for every token count the benchmark times:
+    every channel of at least 128 sampled token rows -- first and last row of the first, a middle
+    and the last token tile, plus seeded ones -- against the reference, and the exact int32 sums
+    of the first and the last 128-channel tile for the same rows.  "as_benchmarked" is the default
+    dispatch, in which the last 128 channels of 4096x14336 are computed by the streaming kernel."""
     torch, b = gpu
-    M, g = 2048, 64
+    g = 64
     if dispatch == "as_benchmarked":
         monkeypatch.delenv("W2A8_PREFILL", raising=False)
-        assert b.w2a8_tensor_core_channels(M, N, K, g) == (111 * 128 if N == 14336 else N)
+        assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
+        if M <= 2048:
+            assert b.w2a8_tensor_core_channels(M, N, K, g) == (111 * 128 if N == 14336 else N)
     codes, s_w = synth.make_linear(4000 + K, K, N, g)
-    bits = synth.activations_bf16(4000 + N, M, K)
+    bits = synth.activations_bf16(4000 + N + M, M, K)
     packed = b.w2_pack(_dev(torch, codes))
     a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
     ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
     y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
     torch.cuda.synchronize()
     assert b.w2a8_workspace_status(ws) == 0
-    rows = sorted(set([0, 127, 1024, 1151, M - 128, M - 1] +
-                      [int(r) for r in np.random.default_rng(K).integers(0, M, size=6)]))
+    rows = _sample_rows(M, K + M)
+    assert len(rows) >= 128
     a_ref, s_ref = oracle.quantize(bits[rows])
-    assert np.array_equal(a.cpu().numpy()[rows], a_ref)
+    idx = torch.tensor(rows, device="cuda")
+    assert np.array_equal(a[idx].cpu().numpy(), a_ref)
     y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
-    got = y.cpu().numpy()[rows].astype(np.float64)
+    got = y[idx].cpu().numpy().astype(np.float64)
     err = np.abs(got - y_ref).max(axis=1)
     assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), float((err / np.abs(y_ref).max(axis=1)).max())
+    assert bool(torch.isfinite(y).all())
+    # exact int32 sums: all tokens against the first and the last channel tile (channels are
+    # independent, so their packed rows form a problem of their own), compared on the sampled rows
+    monkeypatch.setenv("W2A8_PREFILL", "2")
+    sel = np.concatenate([np.arange(128), np.arange(N - 128, N)])
+    sub = packed[torch.from_numpy(sel).cuda()].contiguous()
+    ws2 = b.new_workspace(b.w2a8_workspace_bytes(M, 256, K, g))
+    assert b.w2a8_kernel_for(M, 256, K, g) == "tensor_core"
+    P = b.w2a8_gemm_partials(a, sub, g, ws2)
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws2) == 0
+    assert np.array_equal(P[idx].cpu().numpy(), oracle.partials(a_ref, codes[sel], g))
 
 
 def test_dispatch_rule(gpu, oracle, monkeypatch):
