@@ -129,8 +129,10 @@ int w2a8_workspace_status(const void *workspace, void *stream);
  * M >= 64 with N % 128 == 0 and K % 256 == 0 takes the tensor-core kernel
  * (tcgen05, 128 x 128 output tiles) when there are enough output tiles for it
  * to be the faster one (M * N above about 0.95 million per round of 148
- * tiles); everything else takes the memory-bound streaming kernel (weights
- * read once per slab of up to 32 tokens).  w2a8_kernel_for reports the choice.
+ * tiles); everything else takes a memory-bound streaming kernel (weights
+ * read once per slab of up to 32 tokens): the one-shot kernel, or, for problems
+ * of at most 128 tiles of 16 channels with K % 256 == 0 and at most 32 tokens,
+ * the persistent one.  w2a8_kernel_for reports tensor-core or streaming.
  * A problem given to the tensor-core kernel may leave its last (at most
  * eight) 128-channel tiles to the streaming kernel, as a second launch on the
  * same stream (w2a8_tensor_core_channels); the result does not depend on it
@@ -220,21 +222,75 @@ int w2a8_gemm_partials(const int8_t *a, const uint32_t *packed, int32_t *partial
                        void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * w2a8_linear -- a8_quantize and w2a8_gemm in one call: y = W2A8(x) for bf16
- * activations in device memory (the fused "bf16 in, scaled output" operator of
- * Sec. II-D, where computing the abs-max scales inside the GEMM pays off for
- * GEMV-sized problems and not for large GEMMs).
+ * w2a8_gemm_grouped -- w2a8_gemm for `count` (1 .. 4) weight matrices that
+ * share their activations (q|k|v of an attention block, gate|up of an MLP):
+ * y[i] = W2A8(a; packed[i], w_scale[i]) for every i.  All matrices have the
+ * same K and group; N[i] may differ.  The matrices stay where they are in
+ * memory (no concatenated copy).  This is the K-splitting / launch-amortising
+ * side of Sec. II-D: small GEMV shapes are bound by launch and fork-join cost,
+ * so several of them are walked by one persistent launch (one CTA per SM, tiles
+ * of all matrices dealt to the CTAs) when that is expected to be faster than
+ * one launch per matrix, and otherwise run as `count` w2a8_gemm launches.
+ *   a, a_scale                     as for w2a8_gemm (DEVICE)
+ *   packed, w_scale, y, N          HOST arrays of `count` entries; the entries of
+ *                                  the first three are DEVICE pointers as for w2a8_gemm
+ *   workspace                      w2a8_grouped_workspace_bytes(count, N, M, K, group)
+ * Each y[i] holds, bit for bit, what w2a8_gemm computes for matrix i with the
+ * same kernel choice; with either kernel it is within the tolerance of
+ * w2a8_gemm's contract and repeated calls give equal bits.
+ */
+int w2a8_gemm_grouped(const int8_t *a, const float *a_scale, int count, const uint32_t *const *packed,
+                      const float *const *w_scale, float *const *y, const int *N, int M, int K, int group,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/* Workspace bytes for the grouped entry points (0 for arguments they reject). */
+size_t w2a8_grouped_workspace_bytes(int count, const int *N, int M, int K, int group);
+
+/*
+ * w2a8_linear_grouped -- bf16 activations in, scaled outputs of `count`
+ * matrices out: the fused operator of Sec. II-D ("abs-max scales inside the
+ * GEMM or in a kernel of their own", exposed there as a tuning knob and found
+ * ahead for GEMV-sized problems only).  `fuse` is that knob:
+ *   W2A8_FUSE_OFF   a8_quantize as a launch of its own, then w2a8_gemm_grouped
+ *   W2A8_FUSE_ON    one launch: every CTA of the persistent kernel computes the
+ *                   token scales and the int8 rows itself (same operations as
+ *                   a8_quantize, same bits) into its shared memory.  Possible for
+ *                   at most 8 tokens, K % 256 == 0 and rows that fit shared
+ *                   memory; where it is not possible this behaves like _OFF.
+ *   W2A8_FUSE_AUTO  _ON when the rows a CTA has to scan are small (M * K up to
+ *                   32768 values; W2A8_FUSE_MAX_ELEMS in the environment), else _OFF
+ *   x_bf16     [M][K] bf16 bit patterns, DEVICE
+ *   a, a_scale DEVICE buffers that receive what a8_quantize would write; they may
+ *              be NULL when the call fuses (then nothing is written), and must
+ *              not be NULL otherwise (W2A8_ERR_NULL)
+ *   the rest as for w2a8_gemm_grouped.
+ * w2a8_grouped_plan reports what a call will do: bit 0 = one launch of the
+ * persistent kernel for the whole group, bit 1 = that launch also quantises.
+ * a and a_scale are bitwise those of a8_quantize; every y is bitwise that of
+ * w2a8_gemm_grouped when that call takes the persistent kernel too, and differs
+ * from it by fp32 summation order only otherwise.
+ */
+#define W2A8_FUSE_AUTO (-1)
+#define W2A8_FUSE_OFF 0
+#define W2A8_FUSE_ON 1
+int w2a8_linear_grouped(const void *x_bf16, int8_t *a, float *a_scale, int count, const uint32_t *const *packed,
+                        const float *const *w_scale, float *const *y, const int *N, int M, int K, int group,
+                        int fuse, void *workspace, size_t workspace_bytes, void *stream);
+int w2a8_grouped_plan(int count, const int *N, int M, int K, int group, int fuse);
+
+/*
+ * w2a8_linear -- w2a8_linear_grouped for one matrix with W2A8_FUSE_AUTO:
+ * y = W2A8(x) for bf16 activations in device memory.
  *   x_bf16  [M][K] bf16 bit patterns, DEVICE
  *   a, a_scale   caller-provided DEVICE buffers ([M][K] int8, [M] fp32) that
  *           receive exactly what a8_quantize would write; they stay valid, so
- *           later w2a8_gemm calls on other weight matrices can reuse them (the
- *           k and v projections after q, up after gate)
+ *           later w2a8_gemm calls on other weight matrices can reuse them
  *   the rest as for w2a8_gemm (same workspace size).
- * This enqueues the two kernels, chained by programmatic dependent launch: on
- * B200 that measured faster than a single launch with quantiser CTAs inside the
- * GEMM grid (see the implementation), so the fusion is one of interface, not of
- * kernels.
- * a, a_scale and y are bitwise what a8_quantize + w2a8_gemm produce.
+ * a and a_scale are bitwise what a8_quantize produces.  y is bitwise what
+ * w2a8_gemm produces when both calls are served by the same kernel; when this
+ * call fuses and w2a8_gemm would take the one-shot kernel for the matrix, the
+ * two differ by fp32 summation order only (both within w2a8_gemm's tolerance,
+ * both repeatable bit for bit).
  */
 int w2a8_linear(const void *x_bf16, int8_t *a, float *a_scale, const uint32_t *packed,
                 const float *w_scale, float *y, int M, int N, int K, int group,

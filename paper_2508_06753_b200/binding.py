@@ -19,6 +19,7 @@ EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
     "w2a8_kernel_for", "w2a8_tensor_core_channels", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
+    "w2a8_gemm_grouped", "w2a8_linear_grouped", "w2a8_grouped_workspace_bytes", "w2a8_grouped_plan",
 ]
 
 _lib = None
@@ -62,8 +63,14 @@ def lib() -> ctypes.CDLL:
         L.w2a8_linear_host_workspace_bytes.argtypes = [i, i, i, i]
         L.w2a8_linear_host.argtypes = [vp, i, i, vp, vp, i, i, vp, vp, sz, vp]
         L.w2a8_gemm_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp]
+        L.w2a8_gemm_grouped.argtypes = [vp, vp, i, vp, vp, vp, vp, i, i, i, vp, sz, vp]
+        L.w2a8_linear_grouped.argtypes = [vp, vp, vp, i, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+        L.w2a8_grouped_workspace_bytes.restype = sz
+        L.w2a8_grouped_workspace_bytes.argtypes = [i, vp, i, i, i]
+        L.w2a8_grouped_plan.argtypes = [i, vp, i, i, i, i]
         for name in ("w2_pack", "a8_quantize", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm",
-                     "w2a8_gemm_partials", "w2a8_linear", "w2a8_linear_host", "w2a8_gemm_static"):
+                     "w2a8_gemm_partials", "w2a8_linear", "w2a8_linear_host", "w2a8_gemm_static",
+                     "w2a8_gemm_grouped", "w2a8_linear_grouped", "w2a8_grouped_plan"):
             getattr(L, name).restype = i
         _lib = L
     return _lib
@@ -248,6 +255,74 @@ def w2a8_linear_host(x_host: torch.Tensor, packed: torch.Tensor, w_scale: torch.
                                   workspace.numel() * workspace.element_size(), _stream(stream)),
            "w2a8_linear_host")
     return y_host
+
+
+FUSE_AUTO, FUSE_OFF, FUSE_ON = -1, 0, 1
+
+
+class Group:
+    """Host-side argument block of the grouped entry points: the arrays of device pointers and of
+    N, built once for a set of weight matrices (and, optionally, outputs) and reused every call."""
+
+    def __init__(self, packed, w_scale, y=None):
+        self.packed, self.w_scale = list(packed), list(w_scale)
+        self.count = len(self.packed)
+        self.N = [int(p.shape[0]) for p in self.packed]
+        self.K = int(self.packed[0].shape[1]) * 16
+        self._pk = (ctypes.c_void_p * self.count)(*[_ptr(p) for p in self.packed])
+        self._sc = (ctypes.c_void_p * self.count)(*[_ptr(s) for s in self.w_scale])
+        self._n = (ctypes.c_int * self.count)(*self.N)
+        self.y = None
+        self._y = None
+        if y is not None:
+            self.bind_outputs(y)
+
+    def bind_outputs(self, y):
+        self.y = list(y)
+        self._y = (ctypes.c_void_p * self.count)(*[_ptr(t) for t in self.y])
+
+
+def w2a8_grouped_workspace_bytes(N, M: int, K: int, group: int) -> int:
+    arr = (ctypes.c_int * len(N))(*[int(n) for n in N])
+    return int(lib().w2a8_grouped_workspace_bytes(len(N), arr, M, K, group))
+
+
+def w2a8_grouped_plan(N, M: int, K: int, group: int, fuse: int = FUSE_AUTO) -> dict:
+    """What a grouped call will do: {'one_launch': bool, 'fused': bool}."""
+    arr = (ctypes.c_int * len(N))(*[int(n) for n in N])
+    r = int(lib().w2a8_grouped_plan(len(N), arr, M, K, group, fuse))
+    _check(r if r < 0 else 0, "w2a8_grouped_plan")
+    return {"one_launch": bool(r & 1), "fused": bool(r & 2)}
+
+
+def w2a8_gemm_grouped(a: torch.Tensor, a_scale: torch.Tensor, grp: Group, group: int,
+                      workspace: torch.Tensor, y=None, stream=None):
+    """y[i] = W2A8(a; matrix i) for the matrices of `grp`; see w2a8_gemm_grouped in include/w2a8.h."""
+    M, K = a.shape
+    if y is not None:
+        grp.bind_outputs(y)
+    elif grp.y is None or grp.y[0].shape[0] != M:
+        grp.bind_outputs([torch.empty((M, n), dtype=torch.float32, device=a.device) for n in grp.N])
+    _check(lib().w2a8_gemm_grouped(_ptr(a), _ptr(a_scale), grp.count, grp._pk, grp._sc, grp._y, grp._n, M, K,
+                                   group, _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                   _stream(stream)), "w2a8_gemm_grouped")
+    return grp.y
+
+
+def w2a8_linear_grouped(x: torch.Tensor, grp: Group, group: int, workspace: torch.Tensor, fuse: int = FUSE_AUTO,
+                        a: torch.Tensor | None = None, a_scale: torch.Tensor | None = None, y=None, stream=None):
+    """bf16 x [M][K] (device) -> y[i] fp32 [M][N_i] for the matrices of `grp`; a / a_scale (optional when the
+    call fuses) receive what a8_quantize would write.  See w2a8_linear_grouped in include/w2a8.h."""
+    M, K = x.shape
+    if y is not None:
+        grp.bind_outputs(y)
+    elif grp.y is None or grp.y[0].shape[0] != M:
+        grp.bind_outputs([torch.empty((M, n), dtype=torch.float32, device=x.device) for n in grp.N])
+    _check(lib().w2a8_linear_grouped(_ptr(x), _ptr(a), _ptr(a_scale), grp.count, grp._pk, grp._sc, grp._y,
+                                     grp._n, M, K, group, fuse, _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream)),
+           "w2a8_linear_grouped")
+    return grp.y
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

@@ -51,6 +51,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                       "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
             if verbose:
                 common[1:1] = ["-Xptxas", "-v"]
+            common += os.environ.get("W2A8_NVCC_FLAGS", "").split()      # e.g. -D switches of the kernels
             # one object per source file, compiled side by side, then one link
             objdir = os.path.join(PKG, "build")
             os.makedirs(objdir, exist_ok=True)

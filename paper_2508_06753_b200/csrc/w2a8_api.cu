@@ -4,6 +4,7 @@
 #include <stdlib.h>
 
 #include "w2a8_common.cuh"
+#include "w2a8_quant.cuh"
 
 namespace w2a8 {
 
@@ -13,6 +14,14 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   bool a16, int ldy);
 size_t decode_workspace_bytes(int M, int N, int K, const ShapeInfo &si);
 size_t decode_workspace_header_bytes(int M, int N, int K, const ShapeInfo &si);
+
+bool gemv_supported(int M, int K, int group);
+bool gemv_preferred(int M, int K, int group, int tiles, int count);
+bool gemv_can_fuse(int M, int K, int group);
+bool gemv_fuse_preferred(int M, int K, int group);
+int launch_gemv(const int8_t *a, const float *a_scale, const void *x_bf16, int8_t *a_out, float *a_scale_out,
+                int count, const uint32_t *const *packed, const float *const *w_scale, float *const *y,
+                const int *N, const int *ldy, int M, int K, int group, cudaStream_t st);
 
 bool prefill_supported(int M, int N, int K, int group);
 bool prefill_preferred(int M, int N, int K, int group);
@@ -100,20 +109,6 @@ w2_pack_kernel(const uint8_t *__restrict__ codes, uint32_t *__restrict__ packed,
 constexpr int kQuantThreads = 256;
 constexpr int kQuantRegThreads = 512;
 
-__device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
-
-__device__ __forceinline__ uint32_t quant4(uint32_t lo, uint32_t hi, float inv) {
-    // lo, hi: two 32-bit words holding four consecutive bf16 values
-    const float x0 = __uint_as_float(lo << 16), x1 = __uint_as_float(lo & 0xFFFF0000u);
-    const float x2 = __uint_as_float(hi << 16), x3 = __uint_as_float(hi & 0xFFFF0000u);
-    int q0 = __float2int_rn(__fmul_rn(x0, inv)), q1 = __float2int_rn(__fmul_rn(x1, inv));
-    int q2 = __float2int_rn(__fmul_rn(x2, inv)), q3 = __float2int_rn(__fmul_rn(x3, inv));
-    q0 = max(-127, min(127, q0)); q1 = max(-127, min(127, q1));
-    q2 = max(-127, min(127, q2)); q3 = max(-127, min(127, q3));
-    return (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) |
-           ((uint32_t)(q3 & 0xFF) << 24);
-}
-
 __global__ void __launch_bounds__(kQuantThreads)
 a8_quantize_kernel(const uint16_t *__restrict__ x, int M, int K, int8_t *__restrict__ a,
                    float *__restrict__ a_scale) {
@@ -156,15 +151,6 @@ a8_quantize_kernel(const uint16_t *__restrict__ x, int M, int K, int8_t *__restr
         o.y = quant4(v.z, v.w, inv);
         ar[i] = o;
     }
-}
-
-__device__ __forceinline__ float quant_scale(uint32_t amax_bits, float *inv_out) {
-    const float amax = bf16_bits_to_float(amax_bits);
-    const float s = __fdiv_rn(amax, 127.0f);
-    float inv = __fdiv_rn(1.0f, s);
-    const bool dead = !(amax > 0.0f) || !(fabsf(inv) <= 3.402823466e38f);
-    *inv_out = dead ? 0.0f : inv;
-    return dead ? 0.0f : s;
 }
 
 // VPT 16-byte vectors per thread, all loaded before the reduction starts.
@@ -451,26 +437,103 @@ int w2a8_gemm_partials(const int8_t *a, const uint32_t *packed, int32_t *partial
 
 static inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 
+// ---- matrices that share their activations --------------------------------------------------
+constexpr int kMaxGroup = 4;
+
+// bit 0: the group runs as one launch of the persistent kernel; bit 1: that launch quantises the
+// activations itself.  fuse: W2A8_FUSE_AUTO / _OFF / _ON.  Negative: error.
+static int grouped_plan(int count, const int *N, int M, int K, int group, int fuse, bool have_x) {
+    if (count < 1 || count > kMaxGroup || !N) return W2A8_ERR_SHAPE;
+    int tiles = 0;
+    for (int i = 0; i < count; ++i) {
+        if (!shape_ok(M, N[i], K, group, nullptr)) return W2A8_ERR_SHAPE;
+        tiles += N[i] / 16;
+    }
+    int plan = 0;
+    if (have_x && fuse != W2A8_FUSE_OFF && gemv_can_fuse(M, K, group) &&
+        (fuse == W2A8_FUSE_ON || gemv_fuse_preferred(M, K, group)))
+        plan = 3;
+    else if (gemv_preferred(M, K, group, tiles, count))
+        plan = 1;
+    return plan;
+}
+
+size_t w2a8_grouped_workspace_bytes(int count, const int *N, int M, int K, int group) {
+    if (count < 1 || count > kMaxGroup || !N) return 0;
+    size_t need = 0;
+    for (int i = 0; i < count; ++i) {
+        const size_t b = w2a8_workspace_bytes(M, N[i], K, group);
+        if (b == 0) return 0;
+        if (b > need) need = b;
+    }
+    return need;
+}
+
+int w2a8_grouped_plan(int count, const int *N, int M, int K, int group, int fuse) {
+    return grouped_plan(count, N, M, K, group, fuse, true);
+}
+
+static int grouped_common(const void *x_bf16, const int8_t *a_in, const float *a_scale_in, int8_t *a, float *a_scale,
+                          int count, const uint32_t *const *packed, const float *const *w_scale, float *const *y,
+                          const int *N, int M, int K, int group, int fuse, void *workspace, size_t workspace_bytes,
+                          void *stream) {
+    if (!packed || !w_scale || !y || !N) return W2A8_ERR_NULL;
+    const int plan = grouped_plan(count, N, M, K, group, fuse, x_bf16 != nullptr);
+    if (plan < 0) return plan;
+    for (int i = 0; i < count; ++i) {
+        if (!packed[i] || !w_scale[i] || !y[i]) return W2A8_ERR_NULL;
+        if (!aligned16(packed[i]) || !aligned16(w_scale[i]) || !aligned16(y[i])) return W2A8_ERR_ALIGN;
+    }
+    if (x_bf16 && !aligned16(x_bf16)) return W2A8_ERR_ALIGN;
+    if ((a && !aligned16(a)) || (a_in && !aligned16(a_in))) return W2A8_ERR_ALIGN;
+    if ((a_scale && (reinterpret_cast<uintptr_t>(a_scale) & 3u)) ||
+        (a_scale_in && (reinterpret_cast<uintptr_t>(a_scale_in) & 3u)))
+        return W2A8_ERR_ALIGN;
+    const size_t need = w2a8_grouped_workspace_bytes(count, N, M, K, group);
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
+    if (int st = check_device()) return st;
+    if (plan == 3)          // one launch: quantise and multiply
+        return launch_gemv(nullptr, nullptr, x_bf16, a, a_scale, count, packed, w_scale, y, N, N, M, K, group,
+                           (cudaStream_t)stream);
+    if (x_bf16) {
+        if (!a || !a_scale) return W2A8_ERR_NULL;    // the quantiser needs somewhere to write
+        if (int st = a8_quantize(x_bf16, M, K, a, a_scale, stream)) return st;
+        a_in = a;
+        a_scale_in = a_scale;
+    }
+    if (plan == 1)          // one launch over all matrices
+        return launch_gemv(a_in, a_scale_in, nullptr, nullptr, nullptr, count, packed, w_scale, y, N, N, M, K, group,
+                           (cudaStream_t)stream);
+    for (int i = 0; i < count; ++i)     // one launch per matrix (same stream, so one workspace serves all)
+        if (int st = w2a8_gemm(a_in, a_scale_in, packed[i], w_scale[i], y[i], M, N[i], K, group, workspace,
+                               workspace_bytes, stream))
+            return st;
+    return W2A8_OK;
+}
+
+int w2a8_gemm_grouped(const int8_t *a, const float *a_scale, int count, const uint32_t *const *packed,
+                      const float *const *w_scale, float *const *y, const int *N, int M, int K, int group,
+                      void *workspace, size_t workspace_bytes, void *stream) {
+    if (!a || !a_scale) return W2A8_ERR_NULL;
+    return grouped_common(nullptr, a, a_scale, nullptr, nullptr, count, packed, w_scale, y, N, M, K, group,
+                          W2A8_FUSE_OFF, workspace, workspace_bytes, stream);
+}
+
+int w2a8_linear_grouped(const void *x_bf16, int8_t *a, float *a_scale, int count, const uint32_t *const *packed,
+                        const float *const *w_scale, float *const *y, const int *N, int M, int K, int group,
+                        int fuse, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!x_bf16) return W2A8_ERR_NULL;
+    if (fuse != W2A8_FUSE_AUTO && fuse != W2A8_FUSE_OFF && fuse != W2A8_FUSE_ON) return W2A8_ERR_SHAPE;
+    return grouped_common(x_bf16, nullptr, nullptr, a, a_scale, count, packed, w_scale, y, N, M, K, group, fuse,
+                          workspace, workspace_bytes, stream);
+}
+
 int w2a8_linear(const void *x_bf16, int8_t *a, float *a_scale, const uint32_t *packed,
                 const float *w_scale, float *y, int M, int N, int K, int group, void *workspace,
                 size_t workspace_bytes, void *stream) {
     if (!x_bf16 || !a || !a_scale || !packed || !w_scale || !y) return W2A8_ERR_NULL;
-    ShapeInfo si;
-    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
-    if (!aligned16(x_bf16) || !aligned16(a) || !aligned16(packed) || !aligned16(y) || !aligned16(w_scale) ||
-        (reinterpret_cast<uintptr_t>(a_scale) & 3u))
-        return W2A8_ERR_ALIGN;
-    const size_t need = w2a8_workspace_bytes(M, N, K, group);
-    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
-    if (int st = check_device()) return st;
-    // Two launches chained by programmatic dependent launch.  A single-launch form (M extra CTAs
-    // of the GEMM grid quantise one token each and publish the rows through flags in the
-    // workspace; the other CTAs request their weights and then poll) was built and measured on
-    // B200 on the gate/up GEMV, back to back: GEMM alone 5.1 us, quantiser launch + GEMM 6.3 us,
-    // single launch 9.0 us -- handing the rows to the other CTAs costs several global round trips
-    // (fence, flag, poll, fence), more than the dependent launch it replaces -- so it was dropped.
-    if (int st = a8_quantize(x_bf16, M, K, a, a_scale, stream)) return st;
-    return w2a8_gemm(a, a_scale, packed, w_scale, y, M, N, K, group, workspace, workspace_bytes, stream);
+    return w2a8_linear_grouped(x_bf16, a, a_scale, 1, &packed, &w_scale, &y, &N, M, K, group, W2A8_FUSE_AUTO,
+                               workspace, workspace_bytes, stream);
 }
 
 size_t w2a8_linear_host_workspace_bytes(int M, int N, int K, int group) {

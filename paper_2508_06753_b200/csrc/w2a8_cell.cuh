@@ -3,9 +3,36 @@
 // (up-convert and int8 multiply-accumulate of Sec. II-C, one scale group at a time).
 #pragma once
 
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "w2a8_common.cuh"
 
 namespace w2a8 {
+
+// Kernel parameters of the one-shot streaming kernel; the cell reads the parity-export and
+// ragged-tail fields from it (unused, and dropped by the compiler, in the full-block instances).
+struct DecodeParams {
+    const int8_t *a;
+    const float *a_scale;
+    const uint32_t *packed;
+    const float *w_scale;
+    float *y;
+    int32_t *partials;
+    float *ws;            // [chunks][M][N] partial outputs (chunks > 1)
+    unsigned *counters;   // [grid.z][tile groups] arrival counters (chunks > 1)
+    int *status;          // device status word (0 = ok)
+    int M, N, K, G, group;
+    int blocks, tail_slices, words_per_row;
+    int chunks, blocks_per_chunk;
+    int cluster;          // chunks > 1 and the chunks of a tile form one thread-block cluster
+    int blocks_per_group; // 256-k blocks per scale group (groups of 256 and more)
+    int s_vec;            // the scales of a cell and channel can be copied as one unit (16/8 B fp32, 8/4 B binary16)
+    int h16;              // w_scale holds IEEE binary16 values (16-bit instances)
+    int a16;              // a holds bf16 activations, a_scale is unused (16-bit-activation instances)
+    int ldy;              // elements between consecutive token rows of y (>= N)
+    int y16;              // 16-bit instances only: y holds bf16 instead of fp32
+};
 
 // ---- PTX wrappers ------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -49,12 +76,26 @@ __device__ __forceinline__ uint4 ld_act16(const int8_t *p) {
     return v;
 }
 
+// The same 16 bytes from a staged copy of the activations in shared memory: `p` carries a 32-bit
+// shared-window address in its low bits (see act_ptr), so pointer arithmetic stays plain adds.
+__device__ __forceinline__ uint4 ld_act16_smem(const int8_t *p) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"((uint32_t)(uintptr_t)p));
+    return v;
+}
+__device__ __forceinline__ const int8_t *act_ptr(uint32_t smem_addr) {
+    return reinterpret_cast<const int8_t *>((uintptr_t)smem_addr);
+}
+
 // One cell: 4 slices x (unpack, 2 MMAs per token slab, promotion at group ends).
 // w0s/w1s: this lane's four words (one per slice) of channels n0+gq and n0+gq+8;
 // sc0/sc1: the cell's scales of the same channels (shared memory, 16 bytes each);
 // brow[mt]: this lane's 16 activation bytes of slice 0 of the cell, token row of slab mt.
 // H16: the scales in shared memory are IEEE binary16 (2 bytes each) instead of fp32.
-template <int MT, int SPP, bool ONE, bool PARTIALS, bool FULL, bool H16>
+// ASMEM: brow[] are shared-memory addresses made by act_ptr (activations staged per CTA).
+template <int MT, int SPP, bool ONE, bool PARTIALS, bool FULL, bool H16, bool ASMEM = false>
 __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32_t (&w0s)[4],
                                              const uint32_t (&w1s)[4], const unsigned char *sc0,
                                              const unsigned char *sc1,
@@ -113,7 +154,7 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
             const bool last = ((s + 1) % SPP) == 0 || s == R - 1;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
-                const uint4 b = ld_act16(brow[mt] + s * kSliceK);
+                const uint4 b = ASMEM ? ld_act16_smem(brow[mt] + s * kSliceK) : ld_act16(brow[mt] + s * kSliceK);
                 if (first) mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, magic);
                 else       mma_s8_16x8x32(D[mt], a0, a1, a2, a3, b.x, b.y, D[mt]);
                 mma_s8_16x8x32(D[mt], a4, a5, a6, a7, b.z, b.w, D[mt]);
@@ -147,6 +188,54 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
                         }
                     }
                 }
+            }
+        }
+    }
+}
+
+// One cell against up to 8 tokens whose activation bytes are already in registers: B[s] holds
+// this lane's 16 bytes of slice s (token row gq of the slab).  A warp that owns the same block of
+// every tile it works on loads them once per launch.  fp32 scales, whole blocks, acc as in
+// compute_cell with MT = 1.
+template <int SPP, bool ONE>
+__device__ __forceinline__ void compute_cell_breg(const uint4 &wa, const uint4 &wb, const unsigned char *sc0,
+                                                  const unsigned char *sc1, const uint4 (&B)[4], float (&acc)[4]) {
+    const uint32_t w0s[4] = {wa.x, wa.y, wa.z, wa.w};
+    const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
+    const int magic[4] = {kMagicInt, kMagicInt, kMagicInt, kMagicInt};
+    float s0s[4 / SPP], s1s[4 / SPP];
+    if constexpr (SPP == 4) {
+        s0s[0] = *reinterpret_cast<const float *>(sc0);
+        s1s[0] = *reinterpret_cast<const float *>(sc1);
+    } else if constexpr (SPP == 2) {
+        const float2 v0 = *reinterpret_cast<const float2 *>(sc0);
+        const float2 v1 = *reinterpret_cast<const float2 *>(sc1);
+        s0s[0] = v0.x; s0s[1] = v0.y; s1s[0] = v1.x; s1s[1] = v1.y;
+    } else {
+        const float4 v0 = *reinterpret_cast<const float4 *>(sc0);
+        const float4 v1 = *reinterpret_cast<const float4 *>(sc1);
+        s0s[0] = v0.x; s0s[1] = v0.y; s0s[2] = v0.z; s0s[3] = v0.w;
+        s1s[0] = v1.x; s1s[1] = v1.y; s1s[2] = v1.z; s1s[3] = v1.w;
+    }
+    int D[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        const uint32_t w0 = w0s[s], w1 = w1s[s];
+        const uint32_t a0 = lane_codes(w0, 0), a1 = lane_codes(w1, 0);
+        const uint32_t a2 = lane_codes(w0, 1), a3 = lane_codes(w1, 1);
+        const uint32_t a4 = lane_codes(w0, 2), a5 = lane_codes(w1, 2);
+        const uint32_t a6 = lane_codes(w0, 3), a7 = lane_codes(w1, 3);
+        if ((s % SPP) == 0) mma_s8_16x8x32_pure(D, a0, a1, a2, a3, B[s].x, B[s].y, magic);
+        else                mma_s8_16x8x32_pure(D, a0, a1, a2, a3, B[s].x, B[s].y, D);
+        mma_s8_16x8x32_pure(D, a4, a5, a6, a7, B[s].z, B[s].w, D);
+        if (((s + 1) % SPP) == 0) {
+            const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
+            if constexpr (ONE) {
+                acc[0] = fmaf(s0, __int_as_float(D[0]) - kMagicFloat, acc[0]);
+                acc[2] = fmaf(s1, __int_as_float(D[2]) - kMagicFloat, acc[2]);
+            } else {
+                promote2(acc[0], acc[1], D[0], D[1], s0);
+                promote2(acc[2], acc[3], D[2], D[3], s1);
             }
         }
     }

@@ -59,27 +59,6 @@ constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kRelaxedCtasPerSm = 7;
 constexpr int kRound = 4;                      // landing slots (cells) per warp
 
-struct DecodeParams {
-    const int8_t *a;
-    const float *a_scale;
-    const uint32_t *packed;
-    const float *w_scale;
-    float *y;
-    int32_t *partials;
-    float *ws;            // [chunks][M][N] partial outputs (chunks > 1)
-    unsigned *counters;   // [grid.z][tile groups] arrival counters (chunks > 1)
-    int *status;          // device status word (0 = ok)
-    int M, N, K, G, group;
-    int blocks, tail_slices, words_per_row;
-    int chunks, blocks_per_chunk;
-    int cluster;          // chunks > 1 and the chunks of a tile form one thread-block cluster
-    int blocks_per_group; // 256-k blocks per scale group (groups of 256 and more)
-    int s_vec;            // the scales of a cell and channel can be copied as one unit (16/8 B fp32, 8/4 B binary16)
-    int h16;              // w_scale holds IEEE binary16 values (16-bit instances)
-    int a16;              // a holds bf16 activations, a_scale is unused (16-bit-activation instances)
-    int ldy;              // elements between consecutive token rows of y (>= N)
-    int y16;              // 16-bit instances only: y holds bf16 instead of fp32
-};
 
 // The same cell for 16-bit activations and no activation quantiser (the alternative kernel of
 // Sec. II): the codes become the bf16 values q - 2 (exact), the activations are the caller's
@@ -486,6 +465,10 @@ w2a8_decode_kernel(const DecodeParams p) {
 
 // ---- host side -----------------------------------------------------------------
 int env_int(const char *name, int dflt);
+bool gemv_preferred(int M, int K, int group, int tiles, int count);
+int launch_gemv(const int8_t *a, const float *a_scale, const void *x_bf16, int8_t *a_out, float *a_scale_out,
+                int count, const uint32_t *const *packed, const float *const *w_scale, float *const *y,
+                const int *N, const int *ldy, int M, int K, int group, cudaStream_t st);
 
 struct DecodePlan {
     int mt, tg, ring, chunks, blocks_per_chunk, slabs, groups, s_vec, cluster;
@@ -711,6 +694,14 @@ int launch_decode(const int8_t *a, const float *a_scale, const uint32_t *packed,
                   bool a16, int ldy) {
     if ((h16 || a16) && partials) return W2A8_ERR_SHAPE;
     if (h16 && a16) return W2A8_ERR_SHAPE;
+    // few tokens, whole blocks, fp32 scales, int8 activations, and a problem small enough to be
+    // bound by latency: the persistent kernel
+    if (!h16 && !a16 && !partials && gemv_preferred(M, K, group, N / 16, 1)) {
+        const uint32_t *pk[1] = {packed};
+        const float *sc[1] = {reinterpret_cast<const float *>(w_scale)};
+        float *yy[1] = {reinterpret_cast<float *>(y)};
+        return launch_gemv(a, a_scale, nullptr, nullptr, nullptr, 1, pk, sc, yy, &N, &ldy, M, K, group, st);
+    }
     const DecodePlan pl = decode_plan(M, N, K, si, h16 || a16);
     DecodeParams p;
     p.a = a; p.a_scale = a_scale; p.packed = packed; p.w_scale = reinterpret_cast<const float *>(w_scale);

@@ -2,6 +2,8 @@
 reference: fp32 results within 1e-4 * max|row|; bf16 results bit-equal to the round-to-nearest-even
 of the fp32 result the same kernel produces, and within one bf16 step of the reference's bf16 where
 the two fp32 values straddle a rounding boundary."""
+import os
+
 import numpy as np
 import pytest
 
@@ -45,8 +47,18 @@ def _check(torch, b, oracle, M, N, K, group, seed, ternary=False, frac=0.0, sel=
     s_h_dev = _dev(torch, s_h.view(np.int16)).view(torch.float16)
     y32 = b.w2a8_gemm_h16(a, s_a, packed, s_h_dev, g, ws)
     y16 = b.w2a8_gemm_h16(a, s_a, packed, s_h_dev, g, ws, out_dtype=torch.bfloat16)
-    # the fp32-scale entry on the widened scales: the same arithmetic, so the same bits
-    y_wide = b.w2a8_gemm(a, s_a, packed, s_h_dev.float(), g, ws)
+    # the fp32-scale entry on the widened scales, through the same kernel (the 16-bit entry is
+    # served by the one-shot streaming kernel, never by the persistent one): the same arithmetic in
+    # the same order, so the same bits
+    had = os.environ.get("W2A8_GEMV")
+    os.environ["W2A8_GEMV"] = "0"
+    try:
+        y_wide = b.w2a8_gemm(a, s_a, packed, s_h_dev.float(), g, ws)
+    finally:
+        if had is None:
+            os.environ.pop("W2A8_GEMV", None)
+        else:
+            os.environ["W2A8_GEMV"] = had
     torch.cuda.synchronize()
     assert b.w2a8_workspace_status(ws) == 0
     assert y16.dtype == torch.bfloat16 and y32.dtype == torch.float32

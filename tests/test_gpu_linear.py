@@ -51,12 +51,23 @@ def test_linear_matches_two_calls_and_reference(gpu, oracle, M, N, K, group):
     ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
     a2, s2 = b.a8_quantize(x)
     y2 = b.w2a8_gemm(a2, s2, packed, s_w_d, g, ws)
+    # When the operator quantises inside the persistent kernel, w2a8_gemm may still pick the
+    # one-shot kernel for the same matrix: a, a_scale are the same bits either way, y the same
+    # bits when the kernel is the same and within the tolerance otherwise.
+    plan = b.w2a8_grouped_plan([N], M, K, g)
+    same_kernel = not plan["fused"] or b.w2a8_grouped_plan([N], M, K, g, b.FUSE_OFF)["one_launch"]
+    y_first = None
     for call in range(3):
         y, a, s = b.w2a8_linear(x, packed, s_w_d, g, ws)
         torch.cuda.synchronize()
         assert b.w2a8_workspace_status(ws) == 0
         assert torch.equal(a, a2) and torch.equal(s, s2), call
-        assert torch.equal(y, y2), call
+        if same_kernel:
+            assert torch.equal(y, y2), call
+        else:
+            assert (y - y2).abs().max() <= TOL * y2.abs().max(), call
+        y_first = y.clone() if y_first is None else y_first
+        assert torch.equal(y, y_first), "repeated calls must be bitwise equal"
     y3 = b.w2a8_gemm(a, s, packed, s_w_d, g, ws)    # a plain call on the same workspace afterwards
     assert torch.equal(y3, y2)
     a_ref, s_ref = oracle.quantize(bits)
