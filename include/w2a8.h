@@ -130,9 +130,10 @@ int w2a8_workspace_status(const void *workspace, void *stream);
  * (tcgen05, 128 x 128 output tiles) when there are enough output tiles for it
  * to be the faster one (M * N above about 0.95 million per round of 148
  * tiles); everything else takes a memory-bound streaming kernel (weights
- * read once per slab of up to 32 tokens): the one-shot kernel, or, for problems
- * of at most 128 tiles of 16 channels with K % 256 == 0 and at most 32 tokens,
- * the persistent one.  w2a8_kernel_for reports tensor-core or streaming.
+ * read once per slab of up to 32 tokens): the one-shot kernel when the problem
+ * is about one wave of its CTAs, the persistent one (at most 32 tokens,
+ * K % 256 == 0) for small matrices with K <= 4096 and for problems of more
+ * than one wave.  w2a8_kernel_for reports tensor-core or streaming.
  * A problem given to the tensor-core kernel may leave its last (at most
  * eight) 128-channel tiles to the streaming kernel, as a second launch on the
  * same stream (w2a8_tensor_core_channels); the result does not depend on it
@@ -258,7 +259,10 @@ size_t w2a8_grouped_workspace_bytes(int count, const int *N, int M, int K, int g
  *                   at most 8 tokens, K % 256 == 0 and rows that fit shared
  *                   memory; where it is not possible this behaves like _OFF.
  *   W2A8_FUSE_AUTO  _ON when the rows a CTA has to scan are small (M * K up to
- *                   32768 values; W2A8_FUSE_MAX_ELEMS in the environment), else _OFF
+ *                   8192 values; W2A8_FUSE_MAX_ELEMS in the environment), else _OFF:
+ *                   on B200 the separate quantiser launch hides behind the weight
+ *                   prefetch of the launch that follows it, so fusing only saves a
+ *                   launch on the host and costs device time from two tokens on
  *   x_bf16     [M][K] bf16 bit patterns, DEVICE
  *   a, a_scale DEVICE buffers that receive what a8_quantize would write; they may
  *              be NULL when the call fuses (then nothing is written), and must
@@ -319,6 +323,17 @@ size_t w2a8_linear_host_workspace_bytes(int M, int N, int K, int group);
 int w2a8_linear_host(const void *x_host, int M, int K, const uint32_t *packed,
                      const float *w_scale, int N, int group, float *y_host,
                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * w2a8_read_probe -- measurement aid, not part of the method (the paper's
+ * counterpart is the bandwidth roofline of Sec. II-E, which needs the machine's
+ * attainable read bandwidth): one kernel that reads `bytes` bytes of `buffer`
+ * (DEVICE, 16-byte aligned) with plain 128-bit loads on `stream` and does
+ * nothing else.  Timed by the caller over a buffer larger than L2, it gives the
+ * read-only ceiling a streaming kernel on this device can be compared with.
+ * `sink` is a DEVICE word the kernel may add to (it practically never does).
+ */
+int w2a8_read_probe(const void *buffer, size_t bytes, unsigned *sink, void *stream);
 
 /*
  * w2a8_gemm_static -- w2a8_gemm without a workspace argument.  (The paper has no

@@ -20,6 +20,7 @@ EXPORTS = [
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
     "w2a8_kernel_for", "w2a8_tensor_core_channels", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
     "w2a8_gemm_grouped", "w2a8_linear_grouped", "w2a8_grouped_workspace_bytes", "w2a8_grouped_plan",
+    "w2a8_read_probe",
 ]
 
 _lib = None
@@ -68,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.w2a8_grouped_workspace_bytes.restype = sz
         L.w2a8_grouped_workspace_bytes.argtypes = [i, vp, i, i, i]
         L.w2a8_grouped_plan.argtypes = [i, vp, i, i, i, i]
+        L.w2a8_read_probe.argtypes = [vp, sz, vp, vp]
+        L.w2a8_read_probe.restype = i
         for name in ("w2_pack", "a8_quantize", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm",
                      "w2a8_gemm_partials", "w2a8_linear", "w2a8_linear_host", "w2a8_gemm_static",
                      "w2a8_gemm_grouped", "w2a8_linear_grouped", "w2a8_grouped_plan"):
@@ -323,6 +326,12 @@ def w2a8_linear_grouped(x: torch.Tensor, grp: Group, group: int, workspace: torc
                                      workspace.numel() * workspace.element_size(), _stream(stream)),
            "w2a8_linear_grouped")
     return grp.y
+
+
+def w2a8_read_probe(buffer: torch.Tensor, sink: torch.Tensor, stream=None):
+    """Enqueue one read-only pass over `buffer` (see w2a8_read_probe in include/w2a8.h)."""
+    _check(lib().w2a8_read_probe(_ptr(buffer), buffer.numel() * buffer.element_size(), _ptr(sink),
+                                 _stream(stream)), "w2a8_read_probe")
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

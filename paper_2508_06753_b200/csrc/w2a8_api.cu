@@ -206,6 +206,28 @@ a8_quantize_reg_kernel(const uint16_t *__restrict__ x, int M, int K, int8_t *__r
 }
 
 
+// ---- read-bandwidth probe ----------------------------------------------------------
+// Plain 128-bit loads of a buffer, summed so that nothing can be dropped: what this device
+// delivers to a kernel that only reads, measured with the library's own launch path.
+__global__ void __launch_bounds__(512)
+w2a8_read_probe_kernel(const uint4 *__restrict__ src, size_t nvec, unsigned *__restrict__ out) {
+    unsigned acc = 0;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // four independent loads in flight per thread and trip
+    for (; i + 3 * stride < nvec; i += 4 * stride) {
+        const uint4 v0 = __ldcs(src + i), v1 = __ldcs(src + i + stride);
+        const uint4 v2 = __ldcs(src + i + 2 * stride), v3 = __ldcs(src + i + 3 * stride);
+        acc += (v0.x ^ v0.y ^ v0.z ^ v0.w) + (v1.x ^ v1.y ^ v1.z ^ v1.w) + (v2.x ^ v2.y ^ v2.z ^ v2.w) +
+               (v3.x ^ v3.y ^ v3.z ^ v3.w);
+    }
+    for (; i < nvec; i += stride) {
+        const uint4 v = __ldcs(src + i);
+        acc += v.x ^ v.y ^ v.z ^ v.w;
+    }
+    if (acc == 0x9E3779B9u) atomicAdd(out, acc);     // practically never: keeps the loads alive
+}
+
 }  // namespace w2a8
 
 // ====================================================================== C ABI ==
@@ -324,6 +346,16 @@ static bool takes_tensor_core_kernel(int M, int N, int K, int group) {
 static int tensor_core_channels(int M, int N, int K, int group) {
     if (env_int("W2A8_PREFILL", 1) == 2 || env_int("W2A8_PF_SPLIT", 1) == 0) return N;
     return prefill_channel_split(M, N, K, group);
+}
+
+int w2a8_read_probe(const void *buffer, size_t bytes, unsigned *sink, void *stream) {
+    if (!buffer || !sink) return W2A8_ERR_NULL;
+    if (!aligned16(buffer) || bytes < 16) return W2A8_ERR_ALIGN;
+    if (int st = check_device()) return st;
+    const int ctas = sm_count() * 4;
+    cudaError_t e = launch_kernel(w2a8_read_probe_kernel, dim3(ctas), dim3(512), 0, (cudaStream_t)stream, false,
+                                  reinterpret_cast<const uint4 *>(buffer), bytes / 16, sink);
+    return e == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
 
 int w2a8_kernel_for(int M, int N, int K, int group) {

@@ -193,13 +193,14 @@ __device__ __forceinline__ void compute_cell(const DecodeParams &p, const uint32
     }
 }
 
-// One cell against up to 8 tokens whose activation bytes are already in registers: B[s] holds
-// this lane's 16 bytes of slice s (token row gq of the slab).  A warp that owns the same block of
+// One cell against 8 * MT tokens whose activation bytes are already in registers: B[mt][s] holds
+// this lane's 16 bytes of slice s (token row gq of slab mt).  A warp that owns the same block of
 // every tile it works on loads them once per launch.  fp32 scales, whole blocks, acc as in
-// compute_cell with MT = 1.
-template <int SPP, bool ONE>
+// compute_cell.
+template <int MT, int SPP, bool ONE>
 __device__ __forceinline__ void compute_cell_breg(const uint4 &wa, const uint4 &wb, const unsigned char *sc0,
-                                                  const unsigned char *sc1, const uint4 (&B)[4], float (&acc)[4]) {
+                                                  const unsigned char *sc1, const uint4 (&B)[MT][4],
+                                                  float (&acc)[MT][4]) {
     const uint32_t w0s[4] = {wa.x, wa.y, wa.z, wa.w};
     const uint32_t w1s[4] = {wb.x, wb.y, wb.z, wb.w};
     const int magic[4] = {kMagicInt, kMagicInt, kMagicInt, kMagicInt};
@@ -217,7 +218,7 @@ __device__ __forceinline__ void compute_cell_breg(const uint4 &wa, const uint4 &
         s0s[0] = v0.x; s0s[1] = v0.y; s0s[2] = v0.z; s0s[3] = v0.w;
         s1s[0] = v1.x; s1s[1] = v1.y; s1s[2] = v1.z; s1s[3] = v1.w;
     }
-    int D[4];
+    int D[MT][4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
         const uint32_t w0 = w0s[s], w1 = w1s[s];
@@ -225,17 +226,25 @@ __device__ __forceinline__ void compute_cell_breg(const uint4 &wa, const uint4 &
         const uint32_t a2 = lane_codes(w0, 1), a3 = lane_codes(w1, 1);
         const uint32_t a4 = lane_codes(w0, 2), a5 = lane_codes(w1, 2);
         const uint32_t a6 = lane_codes(w0, 3), a7 = lane_codes(w1, 3);
-        if ((s % SPP) == 0) mma_s8_16x8x32_pure(D, a0, a1, a2, a3, B[s].x, B[s].y, magic);
-        else                mma_s8_16x8x32_pure(D, a0, a1, a2, a3, B[s].x, B[s].y, D);
-        mma_s8_16x8x32_pure(D, a4, a5, a6, a7, B[s].z, B[s].w, D);
-        if (((s + 1) % SPP) == 0) {
-            const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
-            if constexpr (ONE) {
-                acc[0] = fmaf(s0, __int_as_float(D[0]) - kMagicFloat, acc[0]);
-                acc[2] = fmaf(s1, __int_as_float(D[2]) - kMagicFloat, acc[2]);
-            } else {
-                promote2(acc[0], acc[1], D[0], D[1], s0);
-                promote2(acc[2], acc[3], D[2], D[3], s1);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            if ((s % SPP) == 0) mma_s8_16x8x32_pure(D[mt], a0, a1, a2, a3, B[mt][s].x, B[mt][s].y, magic);
+            else                mma_s8_16x8x32_pure(D[mt], a0, a1, a2, a3, B[mt][s].x, B[mt][s].y, D[mt]);
+            mma_s8_16x8x32_pure(D[mt], a4, a5, a6, a7, B[mt][s].z, B[mt][s].w, D[mt]);
+            if (((s + 1) % SPP) == 0) {
+                const float s0 = s0s[s / SPP], s1 = s1s[s / SPP];
+                if constexpr (ONE) {
+                    acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
+                    acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
+                } else if constexpr (MT == 1) {
+                    promote2(acc[mt][0], acc[mt][1], D[mt][0], D[mt][1], s0);
+                    promote2(acc[mt][2], acc[mt][3], D[mt][2], D[mt][3], s1);
+                } else {
+                    acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
+                    acc[mt][1] = fmaf(s0, __int_as_float(D[mt][1]) - kMagicFloat, acc[mt][1]);
+                    acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
+                    acc[mt][3] = fmaf(s1, __int_as_float(D[mt][3]) - kMagicFloat, acc[mt][3]);
+                }
             }
         }
     }

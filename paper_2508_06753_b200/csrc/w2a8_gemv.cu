@@ -79,11 +79,11 @@ struct GemvParams {
 
 // MT: 8-token slabs per virtual tile; SPP: 64-k slices per scale group (capped at 4); ONE: a single
 // token; ASMEM: activations staged in shared memory (copied, or quantised here when p.x is set);
-// BCACHE: one block per K-lane, one slab, MT = 1: activation fragments live in registers.
+// BCACHE: one block per K-lane and all tokens in one tile (M <= 8 * MT): activation fragments live
+// in registers.
 template <int MT, int SPP, bool ONE, bool ASMEM, bool BCACHE>
 __global__ void __launch_bounds__(kGvThreads, 1)
 w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
-    static_assert(!BCACHE || MT == 1, "register-resident activations need a single slab");
     constexpr int SPB = 4 / SPP;                  // scales per block and channel
     constexpr int kRed = ONE ? 16 : MT * 128;     // sums a K-lane parks per tile
     extern __shared__ __align__(128) unsigned char smem[];
@@ -249,11 +249,15 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
         if constexpr (ASMEM) return act_ptr(act_u32 + row * p.act_stride + kb * kBlockK + t * 16);
         else                 return p.a + (size_t)row * p.K + kb * kBlockK + t * 16;
     };
-    uint4 B[4];
+    uint4 B[MT][4];
     if constexpr (BCACHE) {
-        const int8_t *src = act_at(min(gq, p.M - 1), b0);
 #pragma unroll
-        for (int s = 0; s < 4; ++s) B[s] = ASMEM ? ld_act16_smem(src + s * kSliceK) : ld_act16(src + s * kSliceK);
+        for (int mt = 0; mt < MT; ++mt) {
+            const int8_t *src = act_at(min(8 * mt + gq, p.M - 1), b0);
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+                B[mt][s] = ASMEM ? ld_act16_smem(src + s * kSliceK) : ld_act16(src + s * kSliceK);
+        }
     }
 
     // ---- compute side ---------------------------------------------------------------------
@@ -286,8 +290,12 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
                         const uint4 wa = *reinterpret_cast<const uint4 *>(wslots + u * kGvWSlot);
                         const uint4 wb = *reinterpret_cast<const uint4 *>(wslots + u * kGvWSlot + 32 * 16);
                         const unsigned char *sc0 = sslots + u * kGvSSlot + gq * 16;
-                        float acc[1][4] = {{0.f, 0.f, 0.f, 0.f}};
-                        compute_cell_breg<SPP, ONE>(wa, wb, sc0, sc0 + 8 * 16, B, acc[0]);
+                        float acc[MT][4];
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+                        compute_cell_breg<MT, SPP, ONE>(wa, wb, sc0, sc0 + 8 * 16, B, acc);
                         park(li + u * TG, acc);
                         __syncwarp();                             // every lane has read the slot
                         if (q_li < nt_cta) request(u);
@@ -376,17 +384,38 @@ bool gemv_supported(int M, int K, int group) {
 }
 
 // Whether the persistent kernel is expected to beat the one-shot streaming kernel (one launch per
-// matrix) on `count` matrices of `tiles` 16-channel tiles in all.  Measured on B200 (us per call,
-// back to back, group 64, K = 4096; one-shot / persistent): 64 tiles 2.4 / 2.0; 256 tiles 3.0 /
-// 3.3; q|k|v, 384 tiles in three matrices, 7.8 / 3.9; 896 tiles 4.95 / 6.3; gate|up, 1792 tiles in
-// two matrices, 9.9 / 9.7 at one token and 10.6 / 11.4 at four.  So: very small problems, and
-// groups of matrices that are latency-bound one by one.  W2A8_GEMV=2: whenever it serves the
-// shape; W2A8_GEMV=0: never.
+// matrix) on `count` matrices of `tiles` 16-channel tiles in all.  Measured on B200 (us per call
+// incl. the quantiser launch, back to back over rotating weight copies; one-shot / persistent):
+//   Llama-3-8B linears, group 64, M = 1, 4, 8, 16 tokens
+//     q|k|v  4096 x (4096+1024+1024):   8.9 / 5.2    9.3 / 5.3    9.9 / 5.8   11.4 / 12.9
+//     o      4096 x 4096:               4.7 / 4.7    5.2 / 4.8    5.2 / 5.2    6.1 / 11.4
+//     gate   4096 x 14336 (alone):      5.0 / 6.2
+//     gate|up 4096 x (14336+14336):    11.7 / 10.9  12.4 / 12.9  13.2 / 13.1  19.2 / 24.6
+//     down   14336 x 4096:              7.4 / 8.3    8.2 / 10.0   8.3 / 10.4  14.3 / 12.9
+//   Llama-3-70B linears, group 128, M = 1, 8, 32 tokens
+//     q|k|v  8192 x (8192+1024+1024):  13.4 / 10.3  14.8 / 12.4  31.9 / 28.8
+//     o      8192 x 8192:               8.4 / 9.3    9.3 / 10.3  23.7 / 23.7
+//     gate|up 8192 x (28672+28672):    47.2 / 33.0  55.7 / 49.0   140 / 142
+//     down   28672 x 8192:             27.8 / 23.2  32.0 / 29.7  80.7 / 64.6
+// The one-shot kernel is at its best when the whole problem is one wave of its CTAs (8 per SM, 16
+// cells of one 16-channel tile x one 256-k block each); the persistent kernel is ahead on groups
+// of matrices that are latency-bound one by one, on problems of more than one such wave, and
+// where a K-lane is a single block so that the activation fragments stay in registers (K <= 4096,
+// at most 16 tokens) unless the problem is a single matrix near the one-wave size.  (The table was
+// taken before the register-resident form existed for 9 .. 16 tokens.)
+// W2A8_GEMV=2: whenever it serves the shape; W2A8_GEMV=0: never.
 bool gemv_preferred(int M, int K, int group, int tiles, int count) {
     if (!gemv_supported(M, K, group)) return false;
     if (env_int("W2A8_GEMV", 1) == 2) return true;
-    if (tiles <= 128) return true;
-    return count >= 2 && tiles <= 640;
+    const long long blocks = K / kBlockK, cells = (long long)tiles * blocks;
+    const long long one_wave = (long long)sm_count() * 8 * 16;          // cells the one-shot kernel holds at once
+    if (M <= 8) {
+        if (count >= 2 || cells > one_wave) return true;
+        return blocks <= 16 && cells <= 8192;
+    }
+    // two slabs of 8 tokens per tile: ahead with register-resident activations (up to 16 tokens,
+    // K <= 4096) and on long rows
+    return (M <= 16 && blocks <= 16) || blocks >= 32;
 }
 
 // The kernel can quantise the activations itself for this many tokens and this K.
@@ -395,12 +424,17 @@ bool gemv_can_fuse(int M, int K, int group) {
     return (size_t)M * (K + kGvActPad) <= (size_t)(kGvMaxSmem - kGvRingBytes - 2 * kGvPartBytes);
 }
 
-// The paper exposes "abs-max inside the GEMM or in a kernel of its own" as a knob (Sec. II-D) and
-// finds the fused form ahead for GEMV-sized problems only.  Here every CTA repeats the abs-max,
-// so the rule is by the bytes a CTA has to scan: M * K bf16 values.
+// The paper exposes the abs-max scales "inside the GEMM or in a kernel of their own" as a knob
+// (Sec. II-D) and finds the fused form ahead for GEMV-sized problems only.  Here every CTA repeats
+// the abs-max, so the rule is by the values a CTA has to scan, M * K.  Measured on B200 (us per
+// call, fused / quantiser launch + persistent kernel): one token, K = 4096: 5.2 / 5.2 (q|k|v), 4.7 /
+// 4.7 (o), 11.0 / 10.9 (gate|up); one token, K = 14336: 9.1 / 8.3; four tokens, K = 4096: 7.6 / 5.3;
+// eight: 11.0 / 5.8.  Under programmatic dependent launch the quantiser launch hides behind the
+// weight prefetch of the kernel that follows it, so fusing gains nothing on the device even for
+// one token and loses from two tokens on; what it saves is one launch on the host.
 bool gemv_fuse_preferred(int M, int K, int group) {
     if (!gemv_can_fuse(M, K, group)) return false;
-    return (long long)M * K <= (long long)env_int("W2A8_FUSE_MAX_ELEMS", 32768);
+    return (long long)M * K <= (long long)env_int("W2A8_FUSE_MAX_ELEMS", 8192);
 }
 
 static GemvPlan gemv_plan(int M, int K, int tiles, const ShapeInfo &si, bool fused) {
@@ -412,7 +446,7 @@ static GemvPlan gemv_plan(int M, int K, int tiles, const ShapeInfo &si, bool fus
     const int ks = si.blocks >= 16 ? 16 : si.blocks >= 8 ? 8 : 4;
     pl.ks_shift = ks == 16 ? 4 : ks == 8 ? 3 : 2;
     pl.tg = kGvWarps / ks;
-    pl.bcache = pl.mt == 1 && pl.slabs == 1 && si.blocks == ks && env_int("W2A8_GEMV_BCACHE", 1) != 0;
+    pl.bcache = pl.slabs == 1 && si.blocks == ks && env_int("W2A8_GEMV_BCACHE", 1) != 0;
     pl.vtiles = tiles * pl.slabs;
     const int sms = sm_count();
     pl.grid = pl.vtiles < sms ? pl.vtiles : sms;
@@ -449,11 +483,9 @@ static cudaError_t launch_gemv_inst(const GemvParams &p, const GemvPlan &pl, cud
 
 template <int MT, int SPP, bool ONE>
 static cudaError_t launch_gemv_act(const GemvParams &p, const GemvPlan &pl, cudaStream_t st) {
-    if constexpr (MT == 1) {
-        if (pl.bcache)
-            return pl.asmem ? launch_gemv_inst<1, SPP, ONE, true, true>(p, pl, st)
-                            : launch_gemv_inst<1, SPP, ONE, false, true>(p, pl, st);
-    }
+    if (pl.bcache)
+        return pl.asmem ? launch_gemv_inst<MT, SPP, ONE, true, true>(p, pl, st)
+                        : launch_gemv_inst<MT, SPP, ONE, false, true>(p, pl, st);
     return pl.asmem ? launch_gemv_inst<MT, SPP, ONE, true, false>(p, pl, st)
                     : launch_gemv_inst<MT, SPP, ONE, false, false>(p, pl, st);
 }
