@@ -38,7 +38,9 @@ NOMINAL_HBM_GBS = 8000.0
 # 4096x14336, M=1, group-64 GEMM (ncu capture of one launch); the algorithmic bytes of that
 # launch are 18,411,524.
 NCU_TRAFFIC_BYTES_GATE_M1 = 18_378_752
-NCU_TRAFFIC_BYTES_GATEUP_M1 = None      # filled from the ncu capture of the grouped launch
+# the same for one grouped launch of the persistent kernel on gate|up, 4096x(14336+14336), M=1:
+# 36,818,948 algorithmic bytes, 36,736,256 read from DRAM (the activations come from L2), 0 written
+NCU_TRAFFIC_BYTES_GATEUP_M1 = 36_736_256
 
 
 # --------------------------------------------------------------------- accounting
