@@ -95,6 +95,63 @@ def test_argument_errors_are_detected_on_the_host(lib):
     assert lib.w2a8_workspace_status(None, None) == NULLP
 
 
+def test_grouped_entry_points_reject_bad_arguments_on_the_host(lib):
+    buf = ctypes.create_string_buffer(1 << 16)
+    p = (ctypes.addressof(buf) + 15) // 16 * 16
+    NULLP, SHAPE, ALIGN, WS = -1, -2, -3, -4
+    vp2 = (ctypes.c_void_p * 2)(p, p)
+    n2 = (ctypes.c_int * 2)(16, 32)
+    bad_n = (ctypes.c_int * 2)(16, 24)
+    null2 = (ctypes.c_void_p * 2)(p, None)
+    odd2 = (ctypes.c_void_p * 2)(p, p + 8)
+    big = 1 << 15
+    assert lib.w2a8_gemm_grouped(None, p, 2, vp2, vp2, vp2, n2, 1, 256, 64, p, big, None) == NULLP
+    assert lib.w2a8_gemm_grouped(p, p, 2, None, vp2, vp2, n2, 1, 256, 64, p, big, None) == NULLP
+    assert lib.w2a8_gemm_grouped(p, p, 2, null2, vp2, vp2, n2, 1, 256, 64, p, big, None) == NULLP
+    assert lib.w2a8_gemm_grouped(p, p, 0, vp2, vp2, vp2, n2, 1, 256, 64, p, big, None) == SHAPE
+    assert lib.w2a8_gemm_grouped(p, p, 5, vp2, vp2, vp2, n2, 1, 256, 64, p, big, None) == SHAPE
+    assert lib.w2a8_gemm_grouped(p, p, 2, vp2, vp2, vp2, bad_n, 1, 256, 64, p, big, None) == SHAPE
+    assert lib.w2a8_gemm_grouped(p, p, 2, vp2, vp2, vp2, n2, 1, 256, 96, p, big, None) == SHAPE
+    assert lib.w2a8_gemm_grouped(p, p, 2, vp2, odd2, vp2, n2, 1, 256, 64, p, big, None) == ALIGN
+    assert lib.w2a8_gemm_grouped(p, p, 2, vp2, vp2, vp2, n2, 1, 256, 64, None, 0, None) == WS
+    assert lib.w2a8_linear_grouped(None, p, p, 2, vp2, vp2, vp2, n2, 1, 256, 64, -1, p, big, None) == NULLP
+    assert lib.w2a8_linear_grouped(p, p, p, 2, vp2, vp2, vp2, n2, 1, 256, 64, 7, p, big, None) == SHAPE
+    assert lib.w2a8_linear_grouped(p + 2, p, p, 2, vp2, vp2, vp2, n2, 1, 256, 64, 1, p, big, None) == ALIGN
+    assert lib.w2a8_linear_grouped(p, p, p, 2, vp2, vp2, vp2, n2, 1, 256, 64, 0, p, 8, None) == WS
+    assert lib.w2a8_grouped_workspace_bytes(2, n2, 1, 256, 64) >= 256
+    assert lib.w2a8_grouped_workspace_bytes(2, bad_n, 1, 256, 64) == 0
+    assert lib.w2a8_grouped_workspace_bytes(0, n2, 1, 256, 64) == 0
+    assert lib.w2a8_grouped_plan(2, bad_n, 1, 256, 64, -1) == SHAPE
+    assert lib.w2a8_read_probe(None, 1 << 20, p, None) == NULLP
+    assert lib.w2a8_read_probe(p + 4, 1 << 20, p, None) == ALIGN
+
+
+def test_grouped_plan_needs_no_gpu(lib, monkeypatch):
+    """Which kernel a group of matrices gets and whether the quantiser goes inside is host logic:
+    pinned on the linear groups of the benchmark layer (148 SMs assumed when no device is present)."""
+    from paper_2508_06753_b200 import binding as b
+    for name in ("W2A8_GEMV", "W2A8_FUSE_MAX_ELEMS", "W2A8_CHUNKS", "W2A8_TG", "W2A8_RING", "W2A8_MT",
+                 "W2A8_CLUSTER", "W2A8_MIN_WARPS", "W2A8_RELAX"):
+        monkeypatch.delenv(name, raising=False)
+    qkv, gateup = [4096, 1024, 1024], [14336, 14336]
+    assert b.w2a8_grouped_plan(qkv, 1, 4096, 64) == {"one_launch": True, "fused": True}
+    assert b.w2a8_grouped_plan(qkv, 4, 4096, 64) == {"one_launch": True, "fused": False}
+    assert b.w2a8_grouped_plan(qkv, 16, 4096, 64) == {"one_launch": True, "fused": False}
+    assert b.w2a8_grouped_plan(gateup, 4, 4096, 64) == {"one_launch": True, "fused": False}
+    assert b.w2a8_grouped_plan([14336], 1, 4096, 64, b.FUSE_OFF) == {"one_launch": False, "fused": False}
+    assert b.w2a8_grouped_plan([4096], 1, 14336, 64) == {"one_launch": False, "fused": False}      # down
+    assert b.w2a8_grouped_plan([4096], 16, 14336, 64) == {"one_launch": True, "fused": False}
+    assert b.w2a8_grouped_plan([8192], 1, 28672, 128) == {"one_launch": True, "fused": False}      # 70B down
+    assert b.w2a8_grouped_plan(qkv, 4, 4096, 64, b.FUSE_ON) == {"one_launch": True, "fused": True}
+    assert b.w2a8_grouped_plan(qkv, 16, 4096, 64, b.FUSE_ON)["fused"] is False                     # too many tokens
+    assert b.w2a8_grouped_plan([48, 32], 3, 1600, 64) == {"one_launch": False, "fused": False}     # ragged K
+    assert b.w2a8_grouped_plan(qkv, 64, 4096, 64) == {"one_launch": False, "fused": False}
+    monkeypatch.setenv("W2A8_GEMV", "0")
+    assert b.w2a8_grouped_plan(qkv, 1, 4096, 64) == {"one_launch": False, "fused": False}
+    monkeypatch.setenv("W2A8_GEMV", "2")
+    assert b.w2a8_grouped_plan([14336], 1, 4096, 64, b.FUSE_OFF)["one_launch"] is True
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     from paper_2508_06753_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)
