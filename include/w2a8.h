@@ -187,8 +187,10 @@ int w2a8_gemm_h16(const int8_t* a, const float* a_scale, const uint32_t* packed,
  * scale), this build applies it to the group sum, which is exact for all four
  * code values and keeps fp32 scales.  The result differs from the exact sum by
  * fp32 summation error only (of the order sqrt(K) * 2^-24 relative to the
- * magnitude of the terms).  The streaming kernel serves every M (there is no
- * tensor-memory variant of this entry); it is meant for few tokens.
+ * magnitude of the terms).  Few tokens take the streaming kernel (`mma.sync`
+ * bf16); shapes the tensor-core path takes (see w2a8_gemm) run on the 16-bit
+ * tensor-core kernel: tcgen05 kind::f16 with bf16 operands and fp32 accumulators
+ * in tensor memory, the group scale applied when an accumulator is drained.
  */
 int w2a16_gemm(const void* x_bf16, const uint32_t* packed, const float* w_scale, float* y,
                int M, int N, int K, int group, void* workspace, size_t workspace_bytes, void* stream);
@@ -201,6 +203,17 @@ int w2a16_gemm(const void* x_bf16, const uint32_t* packed, const float* w_scale,
  * and measured.)
  */
 int w2a8_kernel_for(int M, int N, int K, int group);
+
+/*
+ * Which tensor-core kernel serves w2a8_gemm / w2a8_gemm_partials for a shape the
+ * tensor-core path takes: 8 = the int8 kernel (tcgen05 kind::i8, int32
+ * accumulators), 16 = the 16-bit kernel (kind::f16 on a bf16 copy of the int8
+ * activations made by a small kernel in front; every product and partial sum is
+ * an integer below 2^24, so the fp32 accumulators hold the same exact group sums
+ * and no int32 -> float conversion is needed), 0 = the shape goes to a streaming
+ * kernel.  W2A8_TC_KIND=8 / 16 in the environment forces one.  Host only.
+ */
+int w2a8_tensor_core_kind(int M, int N, int K, int group);
 
 /*
  * How many of the N output channels the tensor-core kernel computes for this

@@ -20,7 +20,7 @@ EXPORTS = [
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
     "w2a8_kernel_for", "w2a8_tensor_core_channels", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
     "w2a8_gemm_grouped", "w2a8_linear_grouped", "w2a8_grouped_workspace_bytes", "w2a8_grouped_plan",
-    "w2a8_read_probe",
+    "w2a8_read_probe", "w2a8_tensor_core_kind",
 ]
 
 _lib = None
@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.w2a8_grouped_workspace_bytes.restype = sz
         L.w2a8_grouped_workspace_bytes.argtypes = [i, vp, i, i, i]
         L.w2a8_grouped_plan.argtypes = [i, vp, i, i, i, i]
+        L.w2a8_tensor_core_kind.argtypes = [i, i, i, i]
+        L.w2a8_tensor_core_kind.restype = i
         L.w2a8_read_probe.argtypes = [vp, sz, vp, vp]
         L.w2a8_read_probe.restype = i
         for name in ("w2_pack", "a8_quantize", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm",
@@ -172,6 +174,13 @@ def w2a8_kernel_for(M: int, N: int, K: int, group: int) -> str:
     r = int(lib().w2a8_kernel_for(M, N, K, group))
     _check(r if r < 0 else 0, "w2a8_kernel_for")
     return "tensor_core" if r == 1 else "streaming"
+
+
+def w2a8_tensor_core_kind(M: int, N: int, K: int, group: int) -> int:
+    """8 (int8 kernel), 16 (16-bit kernel on a bf16 copy of the activations) or 0 (streaming)."""
+    r = int(lib().w2a8_tensor_core_kind(M, N, K, group))
+    _check(r if r < 0 else 0, "w2a8_tensor_core_kind")
+    return r
 
 
 def w2a8_tensor_core_channels(M: int, N: int, K: int, group: int) -> int:

@@ -29,6 +29,12 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
                    void *y, int32_t *partials, int M, int N, int K, int group, int *status,
                    cudaStream_t st, bool h16, bool y16, int ldy);
 int prefill_channel_split(int M, int N, int K, int group);
+bool prefill_f16_supported(int M, int N, int K, int group);
+size_t prefill_f16_scratch_bytes(int M, int K);
+int launch_prefill_f16(const void *x_bf16, const float *a_scale, const uint32_t *packed, const float *w_scale,
+                       float *y, int32_t *partials, int M, int N, int K, int group, int *status, cudaStream_t st,
+                       int ldy);
+int launch_a8_to_bf16(const int8_t *a, void *scratch, int M, int K, cudaStream_t st);
 
 int env_int(const char *name, int dflt) {
     const char *v = getenv(name);
@@ -298,7 +304,10 @@ int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, voi
 static bool takes_tensor_core_kernel(int M, int N, int K, int group);
 static int tensor_core_channels(int M, int N, int K, int group);
 
-size_t w2a8_workspace_bytes(int M, int N, int K, int group) {
+static bool tensor_core_kind_is_16(int M, int N, int K, int group);
+
+// Workspace of the kernels themselves (status word, split-K counters and partial outputs).
+static size_t kernel_workspace_bytes(int M, int N, int K, int group) {
     ShapeInfo si;
     if (!shape_ok(M, N, K, group, &si)) return 0;
     size_t need = decode_workspace_bytes(M, N, K, si);
@@ -311,6 +320,15 @@ size_t w2a8_workspace_bytes(int M, int N, int K, int group) {
             if (r > need) need = r;
         }
     }
+    return (need + 255) / 256 * 256;
+}
+
+size_t w2a8_workspace_bytes(int M, int N, int K, int group) {
+    size_t need = kernel_workspace_bytes(M, N, K, group);
+    if (need == 0) return 0;
+    // the 16-bit tensor-core kernel reads the int8 activations from a bf16 copy kept behind that
+    if (takes_tensor_core_kernel(M, N, K, group) && tensor_core_kind_is_16(M, N, K, group))
+        need += prefill_f16_scratch_bytes(M, K);
     return need;
 }
 
@@ -358,6 +376,26 @@ int w2a8_read_probe(const void *buffer, size_t bytes, unsigned *sink, void *stre
     return e == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
 
+// Which tensor-core kernel serves the int8 entries for a shape the tensor-core path takes: the int8
+// kernel (kind::i8, int32 accumulators, conversion in the drain) or the 16-bit one (kind::f16 on a
+// bf16 copy of the activations, fp32 accumulators holding the same exact integers).
+// W2A8_TC_KIND=8 / 16 forces one.
+static bool tensor_core_kind_is_16(int M, int N, int K, int group) {
+    if (!prefill_f16_supported(M, N, K, group)) return false;
+    if ((long long)254 * group >= (1ll << 24)) return false;      // fp32 must hold the group sums exactly
+    const int forced = env_int("W2A8_TC_KIND", 0);
+    if (forced == 8) return false;
+    if (forced == 16) return true;
+    return false;
+}
+
+int w2a8_tensor_core_kind(int M, int N, int K, int group) {
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
+    if (!takes_tensor_core_kernel(M, N, K, group)) return 0;
+    return tensor_core_kind_is_16(M, N, K, group) ? 16 : 8;
+}
+
 int w2a8_kernel_for(int M, int N, int K, int group) {
     ShapeInfo si;
     if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
@@ -397,21 +435,38 @@ size_t gemm_header_bytes(int M, int N, int K, int group) {
 int gemm_dispatch(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
                   void *y, int32_t *partials, int M, int N, int K, int group, const ShapeInfo &si,
                   void *workspace, void *stream, bool h16, bool y16, bool a16) {
-    if (!a16 && takes_tensor_core_kernel(M, N, K, group)) {
+    const bool tc16 = !h16 && prefill_f16_supported(M, N, K, group) && takes_tensor_core_kernel(M, N, K, group) &&
+                      (a16 || tensor_core_kind_is_16(M, N, K, group));
+    if (tc16 || (!a16 && takes_tensor_core_kernel(M, N, K, group))) {
         // The tensor-core kernel takes the first n_tc channels; when a last round of a few tiles
         // would cost a whole round, the remaining channel tiles go to the streaming kernel in a
         // second launch (rows of the packed matrix and of the scales are independent; both kernels
         // write their own columns of y).  The parity export is never split.
         const int n_tc = partials ? N : tensor_core_channels(M, N, K, group);
-        int st = launch_prefill(a, a_scale, packed, w_scale, y, partials, M, n_tc, K, group,
+        int st;
+        if (tc16) {
+            // 16-bit operands: the caller's bf16 activations as they are (a16), or a bf16 copy of
+            // the int8 activations kept behind the kernels' own workspace
+            const void *x = a;
+            if (!a16) {
+                void *copy = reinterpret_cast<char *>(workspace) + kernel_workspace_bytes(M, N, K, group);
+                if (int e = launch_a8_to_bf16(a, copy, M, K, (cudaStream_t)stream)) return e;
+                x = copy;
+            }
+            st = launch_prefill_f16(x, a16 ? nullptr : a_scale, packed, reinterpret_cast<const float *>(w_scale),
+                                    reinterpret_cast<float *>(y), partials, M, n_tc, K, group,
+                                    reinterpret_cast<int *>(workspace), (cudaStream_t)stream, N);
+        } else {
+            st = launch_prefill(a, a_scale, packed, w_scale, y, partials, M, n_tc, K, group,
                                 reinterpret_cast<int *>(workspace), (cudaStream_t)stream, h16, y16, N);
+        }
         ShapeInfo rest;
         if (st != W2A8_OK || n_tc >= N || !shape_ok(M, N - n_tc, K, group, &rest)) return st;
         const size_t scale_bytes = h16 ? 2 : 4, y_bytes = (h16 && y16) ? 2 : 4;
         return launch_decode(a, a_scale, packed + (size_t)n_tc * si.words_per_row,
                              reinterpret_cast<const char *>(w_scale) + (size_t)n_tc * si.G * scale_bytes,
                              reinterpret_cast<char *>(y) + (size_t)n_tc * y_bytes, nullptr, M, N - n_tc, K,
-                             group, rest, workspace, (cudaStream_t)stream, h16, y16, false, N);
+                             group, rest, workspace, (cudaStream_t)stream, h16, y16, a16, N);
     }
     return launch_decode(a, a_scale, packed, w_scale, y, partials, M, N, K, group, si, workspace,
                          (cudaStream_t)stream, h16, y16, a16, N);

@@ -44,8 +44,8 @@ CASES = [
     (32, 256, 8192, 128, False, 0.01),
     (1, 256, 8192, 64, True, 0.0),          # split-K inside a cluster
     (1, 16, 28672, 128, False, 0.01),       # longest K of any configuration
-    (70, 48, 768, 128, False, 0.0),         # many tokens: still the streaming kernel
-    (96, 256, 1024, 64, False, 0.0),        # a shape the int8 entry would give to the tensor-core kernel
+    (70, 48, 768, 128, False, 0.0),         # many tokens, a shape the tensor-core kernel does not tile
+    (96, 256, 1024, 64, False, 0.0),        # too few output tiles for the tensor-core kernel to pay
 ]
 
 
@@ -120,6 +120,81 @@ def test_a16_full_size_gate_sampled(gpu, oracle, M):
     err = np.abs(y[:, sel].astype(np.float64) - ref).max(axis=1)
     assert (err <= TOL * np.abs(ref).max(axis=1)).all()
     assert np.isfinite(y).all()
+
+
+TC_CASES = [
+    # M, N, K, group (0 = K): shapes of the tensor-core kernel's own parity list
+    (128, 128, 256, 64), (64, 128, 512, 64), (300, 256, 1024, 64), (256, 384, 2048, 128), (130, 128, 1024, 256),
+    (200, 256, 1536, 512), (257, 128, 1280, 0), (640, 4096, 512, 64), (200, 19200, 256, 128),
+]
+
+
+@pytest.mark.parametrize("M,N,K,group", TC_CASES)
+def test_a16_tensor_core_kernel(gpu, oracle, monkeypatch, M, N, K, group):
+    """Many tokens: the 16-bit tensor-core kernel (tcgen05 kind::f16, bf16 operands, fp32 accumulators
+    in tensor memory), forced for small shapes the dispatch rule would stream."""
+    torch, b = gpu
+    monkeypatch.setenv("W2A8_PREFILL", "2")
+    g = K if group == 0 else group
+    assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
+    codes, s_w = synth.make_linear(5 * M + N + K, K, N, g)
+    bits = synth.activations_bf16(M + K, M, K, 0.01)
+    packed = b.w2_pack(_dev(torch, codes))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    x = _bf16_dev(torch, bits)
+    y = b.w2a16_gemm(x, packed, _dev(torch, s_w), g, ws)
+    y2 = b.w2a16_gemm(x, packed, _dev(torch, s_w), g, ws)
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    assert torch.equal(y, y2)
+    ref = oracle.gemm_a16(bits, codes, s_w, g)
+    err = np.abs(y.cpu().numpy().astype(np.float64) - ref.astype(np.float64)).max(axis=1)
+    assert (err <= TOL * np.abs(ref).max(axis=1)).all(), float((err / (TOL * np.abs(ref).max(axis=1))).max())
+    # and the streaming kernel on the same problem agrees within the same tolerance
+    monkeypatch.setenv("W2A8_PREFILL", "0")
+    y_st = b.w2a16_gemm(x, packed, _dev(torch, s_w), g, ws)
+    assert (y - y_st).abs().max() <= 2 * TOL * y.abs().max()
+
+
+@pytest.mark.parametrize("M,N,K,group", [(128, 128, 1024, 64), (192, 256, 2048, 128), (96, 128, 15104 - 256 * 3 + 256, 0)])
+def test_a16_tensor_core_exact_on_integers(gpu, monkeypatch, M, N, K, group):
+    """Integer activations and unit scales through the tensor-core kernel: the integer matrix
+    product, bit for bit."""
+    torch, b = gpu
+    monkeypatch.setenv("W2A8_PREFILL", "2")
+    g = K if group == 0 else group
+    rng = np.random.default_rng(M + N + K)
+    xi = rng.integers(-127, 128, size=(M, K))
+    codes = rng.integers(0, 4, size=(N, K), dtype=np.uint8)
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    x = _dev(torch, xi.astype(np.float32)).to(torch.bfloat16)
+    y = b.w2a16_gemm(x, b.w2_pack(_dev(torch, codes)), torch.ones((N, K // g), dtype=torch.float32, device="cuda"),
+                     g, ws)
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    want = xi @ (codes.astype(np.int64) - 2).T
+    assert np.abs(want).max() < 2 ** 24
+    assert np.array_equal(y.cpu().numpy().astype(np.int64), want)
+
+
+def test_a16_full_size_prefill_sampled_rows(gpu, oracle):
+    """The prefill configuration's gate matrix at M = 2048 through w2a16_gemm as dispatched by
+    default (tensor-core kernel plus the streamed last channel tile), on sampled token rows."""
+    torch, b = gpu
+    M, K, N, g = 2048, 4096, 14336, 64
+    assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
+    codes, s_w = synth.make_linear(4100, K, N, g)
+    bits = synth.activations_bf16(4101, M, K)
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    y = b.w2a16_gemm(_bf16_dev(torch, bits), b.w2_pack(_dev(torch, codes)), _dev(torch, s_w), g, ws)
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    rows = sorted(set([0, 127, 1024, 1151, M - 128, M - 1] + [int(r) for r in np.random.default_rng(3).integers(0, M, 26)]))
+    ref = oracle.gemm_a16(bits[rows], codes, s_w, g)
+    got = y[torch.tensor(rows, device="cuda")].cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref).max(axis=1)
+    assert (err <= TOL * np.abs(ref).max(axis=1)).all()
+    assert bool(torch.isfinite(y).all())
 
 
 def test_a16_argument_errors(gpu):

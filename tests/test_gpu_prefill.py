@@ -47,11 +47,17 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("kind", [8, 16])
 @pytest.mark.parametrize("M,N,K,group", CASES)
-def test_prefill_against_reference(gpu, oracle, M, N, K, group):
+def test_prefill_against_reference(gpu, oracle, monkeypatch, M, N, K, group, kind):
+    """Both tensor-core kernels behind w2a8_gemm: the int8 one (kind::i8, int32 accumulators) and
+    the 16-bit one (kind::f16 on a bf16 copy of the int8 activations, fp32 accumulators that hold the
+    same integers): exact int32 group sums from either."""
     torch, b = gpu
+    monkeypatch.setenv("W2A8_TC_KIND", str(kind))
     g = K if group == 0 else group
     assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
+    assert b.w2a8_tensor_core_kind(M, N, K, g) == kind
     codes, s_w = synth.make_linear(7 * M + N + K, K, N, g)
     bits = synth.activations_bf16(M + K, M, K)
     packed = b.w2_pack(_dev(torch, codes))
