@@ -1007,6 +1007,49 @@ def prefill_probe(device, peaks, Ms=(512, 2048, 8192), reps=5):
                          "frac_of_measured_int8_sustained": tops / int8_peak_sustained,
                          "status": b.w2a8_workspace_status(ws)})
         del packed, s_w_d, ws
+    # The 16-bit tensor-core kernel (tcgen05 kind::f16, the alternative kernel of Sec. II) on the
+    # same gate/up problem: behind w2a16_gemm (bf16 activations as they are) and behind w2a8_gemm
+    # (W2A8_TC_KIND=16: bf16 copy of the int8 activations, copy kernel included in the time)
+    alt = []
+    name, K, N = cfg["shapes"][0]
+    g = synth.config_group(cfg, K)
+    codes, s_w = synth.make_linear(synth.shape_seed(cfg, 0), K, N, g)
+    packed = b.w2_pack(torch.from_numpy(codes).to(device))
+    s_w_d = torch.from_numpy(s_w).to(device)
+    del codes
+    saved_kind = os.environ.get("W2A8_TC_KIND")
+    for M in Ms:
+        bits = synth.activations_bf16(cfg["seed"] + 7 + M, M, K)
+        x = torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+        a, s_a = b.a8_quantize(x)
+        y = torch.empty((M, N), dtype=torch.float32, device=device)
+        row = {"shape": f"{K}x{N}", "M": M, "group": g}
+        for label, kind in (("w2a16_gemm", None), ("w2a8_gemm_kind16", "16")):
+            if kind is None:
+                os.environ.pop("W2A8_TC_KIND", None)
+            else:
+                os.environ["W2A8_TC_KIND"] = kind
+            ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g), device=device)
+            fn = (lambda: b.w2a16_gemm(x, packed, s_w_d, g, ws, y)) if kind is None else \
+                 (lambda: b.w2a8_gemm(a, s_a, packed, s_w_d, g, ws, y))
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            row[label] = {"ms": ms, "tops": 2.0 * M * N * K / (ms * 1e-3) / 1e12, "status": b.w2a8_workspace_status(ws)}
+            del ws
+        alt.append(row)
+    if saved_kind is None:
+        os.environ.pop("W2A8_TC_KIND", None)
+    else:
+        os.environ["W2A8_TC_KIND"] = saved_kind
+    del packed, s_w_d
     # library int8 GEMM on the same device as a second, directly measured denominator
     lib_int8 = None
     try:
@@ -1030,7 +1073,9 @@ def prefill_probe(device, peaks, Ms=(512, 2048, 8192), reps=5):
     return {"unit": "int8 TOPS", "peak_measured_burst": int8_peak_burst,
             "peak_measured_sustained": int8_peak_sustained,
             "peak_note": "measured cuBLAS bf16 peak x 2 (nominal int8 : bf16 ratio); nominal dense int8 4500",
-            "library_int8_gemm": lib_int8, "rows": rows, "by_group_m2048": by_group}
+            "library_int8_gemm": lib_int8, "rows": rows, "by_group_m2048": by_group,
+            "kind_f16_kernel": {"what": "16-bit tensor-core kernel (tcgen05 kind::f16, fp32 accumulators, no conversion "
+                                        "in the drain): op/s counted as for the int8 kernel", "rows": alt}}
 
 
 def run_kernel_profile(args):

@@ -236,14 +236,9 @@ __device__ __forceinline__ void compute_cell_breg(const uint4 &wa, const uint4 &
                 if constexpr (ONE) {
                     acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
                     acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
-                } else if constexpr (MT == 1) {
+                } else {
                     promote2(acc[mt][0], acc[mt][1], D[mt][0], D[mt][1], s0);
                     promote2(acc[mt][2], acc[mt][3], D[mt][2], D[mt][3], s1);
-                } else {
-                    acc[mt][0] = fmaf(s0, __int_as_float(D[mt][0]) - kMagicFloat, acc[mt][0]);
-                    acc[mt][1] = fmaf(s0, __int_as_float(D[mt][1]) - kMagicFloat, acc[mt][1]);
-                    acc[mt][2] = fmaf(s1, __int_as_float(D[mt][2]) - kMagicFloat, acc[mt][2]);
-                    acc[mt][3] = fmaf(s1, __int_as_float(D[mt][3]) - kMagicFloat, acc[mt][3]);
                 }
             }
         }
