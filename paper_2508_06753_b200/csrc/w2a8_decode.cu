@@ -299,6 +299,21 @@ w2a8_decode_kernel(const DecodeParams p) {
     }
     pdl_wait();
 
+    // The token scale of the outputs this thread will store is only needed by the epilogue, at the
+    // very end of the critical path of a short launch: fetch it now.  Output element e of the CTA
+    // (see `locate` below) belongs to token row_of(e).
+    constexpr int kOutPerThread = ONE ? 1 : TG * MT;          // = ceil(kElems / kDecodeThreads)
+    float tok_scale[kOutPerThread];
+    if constexpr (!PARTIALS && !A16) {
+#pragma unroll
+        for (int j = 0; j < kOutPerThread; ++j) {
+            const int e = threadIdx.x + j * kDecodeThreads;
+            const int el = e & 31, ei = (e >> 5) % (MT * 4);
+            const int mm = ONE ? 0 : m0 + 8 * (ei >> 2) + 2 * (el & 3) + (ei & 1);
+            tok_scale[j] = mm < p.M ? p.a_scale[mm] * (1.0f / kCodeGain) : 0.f;
+        }
+    }
+
     float acc[MT][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
@@ -398,8 +413,8 @@ w2a8_decode_kernel(const DecodeParams p) {
         };
 
         // final value of y[mm][nn]: fp32, or (16-bit instances, on request) rounded to bf16
-        auto store_y = [&](int mm, int nn, float v) {
-            if constexpr (!A16) v *= p.a_scale[mm] * (1.0f / kCodeGain);   // bf16 weights carry no gain
+        auto store_y = [&](int mm, int nn, float v, float scale) {
+            if constexpr (!A16) v *= scale;                                // bf16 weights carry no gain
             if constexpr (H16) {
                 if (p.y16) {
                     reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)mm * p.ldy + nn] = __float2bfloat16_rn(v);
@@ -410,9 +425,11 @@ w2a8_decode_kernel(const DecodeParams p) {
         };
 
         if (p.chunks == 1) {
-            for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
+#pragma unroll
+            for (int j = 0; j < kOutPerThread; ++j) {
+                const int e = threadIdx.x + j * kDecodeThreads;
                 int mm, nn;
-                if (locate(e, mm, nn)) store_y(mm, nn, cta_sum(e));
+                if (e < kElems && locate(e, mm, nn)) store_y(mm, nn, cta_sum(e), tok_scale[j]);
             }
         } else if (p.cluster) {
             // ---- split-K inside a thread-block cluster: the chunks of a tile are the CTAs of one
@@ -428,12 +445,14 @@ w2a8_decode_kernel(const DecodeParams p) {
             }
             cluster_sync();
             if (rank != 0) return;
-            for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
+#pragma unroll
+            for (int j = 0; j < kOutPerThread; ++j) {
+                const int e = threadIdx.x + j * kDecodeThreads;
                 int mm, nn;
-                if (locate(e, mm, nn)) {
+                if (e < kElems && locate(e, mm, nn)) {
                     float v = 0.f;
                     for (int ch = 0; ch < p.chunks; ++ch) v += recv[ch * kElems + e];
-                    store_y(mm, nn, v);
+                    store_y(mm, nn, v, tok_scale[j]);
                 }
             }
         } else {
@@ -450,12 +469,14 @@ w2a8_decode_kernel(const DecodeParams p) {
             __syncthreads();
             if (!is_last) return;
             __threadfence();
-            for (int e = threadIdx.x; e < kElems; e += kDecodeThreads) {
+#pragma unroll
+            for (int j = 0; j < kOutPerThread; ++j) {
+                const int e = threadIdx.x + j * kDecodeThreads;
                 int mm, nn;
-                if (locate(e, mm, nn)) {
+                if (e < kElems && locate(e, mm, nn)) {
                     float v = 0.f;
                     for (int ch = 0; ch < p.chunks; ++ch) v += __ldcg(p.ws + ch * MN + (size_t)mm * p.N + nn);
-                    store_y(mm, nn, v);
+                    store_y(mm, nn, v, tok_scale[j]);
                 }
             }
             if (threadIdx.x == 0) *counter = 0u;   // leave the workspace reusable

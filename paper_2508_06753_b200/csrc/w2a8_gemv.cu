@@ -88,7 +88,7 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
     constexpr int kRed = ONE ? 16 : MT * 128;     // sums a K-lane parks per tile
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ uint32_t wmax[kGvMaxFuseM][kGvWarps];
-    __shared__ float s_scale[kGvMaxFuseM];
+    __shared__ float s_scale[kGvMaxTokens];     // token scales: written here, read by the epilogue
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, t = lane & 3;
     const int TG = p.tg, KS = 1 << p.ks_shift;
@@ -183,6 +183,9 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
         if (r == 0) pdl_launch_dependents();
     }
     pdl_wait();
+    // The token scales are only needed by the epilogue, at the very end of the critical path of a
+    // short launch: fetch them now (the first CTA barrier orders them before their use).
+    if (!(ASMEM && p.x != nullptr) && threadIdx.x < p.M) s_scale[threadIdx.x] = p.a_scale[threadIdx.x];
 
     // ---- activations into shared memory (ASMEM) ---------------------------------------
     if constexpr (ASMEM) {
@@ -241,7 +244,6 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
         __syncthreads();
     }
     const uint32_t act_u32 = smem_u32(act);
-    const bool own_scales = ASMEM && p.x != nullptr;
 
     // This lane's activation bytes of block kb, token row `row` (MMA column gq of a slab).  Token
     // columns of an MMA are independent and columns beyond M are never stored: they read the last row.
@@ -355,11 +357,16 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
                 nn = (el >> 2) + 8 * ((ei & 3) >> 1);
             }
             if (mm >= p.M) continue;
+            // all K-lane sums of the output are fetched first (independent loads), then added in
+            // lane order: the order, and with it the bits of y, does not depend on anything else
             const float *src = rpart + li * KS * kRed + r;
+            float part[kGvWarps];
+#pragma unroll
+            for (int k2 = 0; k2 < kGvWarps; ++k2) part[k2] = k2 < KS ? src[k2 * kRed] : 0.f;
             float v = 0.f;
-            for (int k2 = 0; k2 < KS; ++k2) v += src[k2 * kRed];
-            const float sa = own_scales ? s_scale[mm] : p.a_scale[mm];
-            ow.y[(size_t)mm * ow.ldy + nn] = v * (sa * (1.0f / kCodeGain));
+#pragma unroll
+            for (int k2 = 0; k2 < kGvWarps; ++k2) v += part[k2];
+            ow.y[(size_t)mm * ow.ldy + nn] = v * (s_scale[mm] * (1.0f / kCodeGain));
         }
     }
 }
