@@ -338,6 +338,21 @@ int w2a8_linear_host(const void *x_host, int M, int K, const uint32_t *packed,
                      void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * w2a8_linear_grouped_host -- w2a8_linear_host for `count` (1 .. 4) matrices
+ * that share their activations: x is brought to the device and quantised once,
+ * then the group runs as in w2a8_gemm_grouped and every y_host[i] ([M][N[i]]
+ * fp32, HOST) receives its result.  packed, w_scale, N, y_host are HOST arrays of
+ * `count` entries; the entries of packed and w_scale are DEVICE pointers, those of
+ * y_host HOST pointers.  Zero-copy rule, workspace initialisation and
+ * asynchronous completion as for w2a8_linear_host; workspace size from
+ * w2a8_linear_grouped_host_workspace_bytes.
+ */
+size_t w2a8_linear_grouped_host_workspace_bytes(int count, const int *N, int M, int K, int group);
+int w2a8_linear_grouped_host(const void *x_host, int M, int K, int count, const uint32_t *const *packed,
+                             const float *const *w_scale, const int *N, int group, float *const *y_host,
+                             void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * w2a8_read_probe -- measurement aid, not part of the method (the paper's
  * counterpart is the bandwidth roofline of Sec. II-E, which needs the machine's
  * attainable read bandwidth): one kernel that reads `bytes` bytes of `buffer`

@@ -21,6 +21,7 @@ EXPORTS = [
     "w2a8_kernel_for", "w2a8_tensor_core_channels", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
     "w2a8_gemm_grouped", "w2a8_linear_grouped", "w2a8_grouped_workspace_bytes", "w2a8_grouped_plan",
     "w2a8_read_probe", "w2a8_tensor_core_kind",
+    "w2a8_linear_grouped_host", "w2a8_linear_grouped_host_workspace_bytes",
 ]
 
 _lib = None
@@ -69,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.w2a8_grouped_workspace_bytes.restype = sz
         L.w2a8_grouped_workspace_bytes.argtypes = [i, vp, i, i, i]
         L.w2a8_grouped_plan.argtypes = [i, vp, i, i, i, i]
+        L.w2a8_linear_grouped_host_workspace_bytes.restype = sz
+        L.w2a8_linear_grouped_host_workspace_bytes.argtypes = [i, vp, i, i, i]
+        L.w2a8_linear_grouped_host.argtypes = [vp, i, i, i, vp, vp, vp, i, vp, vp, sz, vp]
+        L.w2a8_linear_grouped_host.restype = i
         L.w2a8_tensor_core_kind.argtypes = [i, i, i, i]
         L.w2a8_tensor_core_kind.restype = i
         L.w2a8_read_probe.argtypes = [vp, sz, vp, vp]
@@ -335,6 +340,23 @@ def w2a8_linear_grouped(x: torch.Tensor, grp: Group, group: int, workspace: torc
                                      workspace.numel() * workspace.element_size(), _stream(stream)),
            "w2a8_linear_grouped")
     return grp.y
+
+
+def w2a8_linear_grouped_host_workspace_bytes(N, M: int, K: int, group: int) -> int:
+    arr = (ctypes.c_int * len(N))(*[int(n) for n in N])
+    return int(lib().w2a8_linear_grouped_host_workspace_bytes(len(N), arr, M, K, group))
+
+
+def w2a8_linear_grouped_host(x_host: torch.Tensor, grp: Group, group: int, y_host, workspace: torch.Tensor,
+                             stream=None):
+    """Host bf16 x [M][K] -> host fp32 y_host[i] [M][N_i] for the matrices of `grp` (device); x is
+    brought over and quantised once.  See w2a8_linear_grouped_host in include/w2a8.h."""
+    M, K = x_host.shape
+    ys = (ctypes.c_void_p * grp.count)(*[_ptr(t) for t in y_host])
+    _check(lib().w2a8_linear_grouped_host(_ptr(x_host), M, K, grp.count, grp._pk, grp._sc, grp._n, group, ys,
+                                          _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                          _stream(stream)), "w2a8_linear_grouped_host")
+    return y_host
 
 
 def w2a8_read_probe(buffer: torch.Tensor, sink: torch.Tensor, stream=None):

@@ -681,4 +681,57 @@ int w2a8_linear_host(const void *x_host, int M, int K, const uint32_t *packed,
     return W2A8_OK;
 }
 
+size_t w2a8_linear_grouped_host_workspace_bytes(int count, const int *N, int M, int K, int group) {
+    const size_t g = w2a8_grouped_workspace_bytes(count, N, M, K, group);
+    if (g == 0) return 0;
+    size_t need = up256(g) + up256((size_t)M * K * 2) + up256((size_t)M * K) + up256((size_t)M * 4);
+    for (int i = 0; i < count; ++i) need += up256((size_t)M * N[i] * 4);
+    return need;
+}
+
+int w2a8_linear_grouped_host(const void *x_host, int M, int K, int count, const uint32_t *const *packed,
+                             const float *const *w_scale, const int *N, int group, float *const *y_host,
+                             void *workspace, size_t workspace_bytes, void *stream) {
+    if (!x_host || !packed || !w_scale || !N || !y_host) return W2A8_ERR_NULL;
+    const size_t need = w2a8_linear_grouped_host_workspace_bytes(count, N, M, K, group);
+    if (need == 0) return W2A8_ERR_SHAPE;
+    if (!workspace || workspace_bytes < need || !aligned16(workspace)) return W2A8_ERR_WORKSPACE;
+    for (int i = 0; i < count; ++i)
+        if (!y_host[i]) return W2A8_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    char *p = reinterpret_cast<char *>(workspace);
+    const size_t gemm_ws = w2a8_grouped_workspace_bytes(count, N, M, K, group);
+    void *ws = p;                     p += up256(gemm_ws);
+    void *x_dev = p;                  p += up256((size_t)M * K * 2);
+    int8_t *a = (int8_t *)p;          p += up256((size_t)M * K);
+    float *a_scale = (float *)p;      p += up256((size_t)M * 4);
+    float *y_dev[kMaxGroup];
+    for (int i = 0; i < count; ++i) { y_dev[i] = (float *)p; p += up256((size_t)M * N[i] * 4); }
+    // As in w2a8_linear_host: with few tokens and page-locked, mapped buffers the quantiser reads x
+    // over the bus itself -- once for the whole group -- and the GEMMs store straight to the host
+    // buffers; otherwise staged copies.  The quantiser always runs as a launch of its own here:
+    // inside the GEMM launch every CTA would fetch x over the bus.
+    static const int zero_copy_max = env_int("W2A8_ZEROCOPY_MAX", kDecodeMaxZeroCopyTokens);
+    const void *x_map = (M <= zero_copy_max) ? mapped_device_pointer(x_host) : nullptr;
+    float *y_map[kMaxGroup];
+    bool direct = x_map != nullptr && aligned16(x_map);
+    for (int i = 0; i < count && direct; ++i) {
+        y_map[i] = reinterpret_cast<float *>(mapped_device_pointer(y_host[i]));
+        direct = y_map[i] != nullptr && aligned16(y_map[i]);
+    }
+    if (direct) {
+        if (int s = a8_quantize(x_map, M, K, a, a_scale, stream)) return s;
+        return w2a8_gemm_grouped(a, a_scale, count, packed, w_scale, y_map, N, M, K, group, ws, gemm_ws, stream);
+    }
+    if (cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return W2A8_ERR_CUDA;
+    if (int s = a8_quantize(x_dev, M, K, a, a_scale, stream)) return s;
+    if (int s = w2a8_gemm_grouped(a, a_scale, count, packed, w_scale, y_dev, N, M, K, group, ws, gemm_ws, stream))
+        return s;
+    for (int i = 0; i < count; ++i)
+        if (cudaMemcpyAsync(y_host[i], y_dev[i], (size_t)M * N[i] * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return W2A8_ERR_CUDA;
+    return W2A8_OK;
+}
+
 }  // extern "C"

@@ -122,6 +122,11 @@ def test_grouped_entry_points_reject_bad_arguments_on_the_host(lib):
     assert lib.w2a8_grouped_workspace_bytes(2, bad_n, 1, 256, 64) == 0
     assert lib.w2a8_grouped_workspace_bytes(0, n2, 1, 256, 64) == 0
     assert lib.w2a8_grouped_plan(2, bad_n, 1, 256, 64, -1) == SHAPE
+    assert lib.w2a8_linear_grouped_host(None, 1, 256, 2, vp2, vp2, n2, 64, vp2, p, big, None) == NULLP
+    assert lib.w2a8_linear_grouped_host(p, 1, 256, 2, vp2, vp2, bad_n, 64, vp2, p, big, None) == SHAPE
+    assert lib.w2a8_linear_grouped_host(p, 1, 256, 2, vp2, vp2, n2, 64, null2, p, 1 << 20, None) == NULLP
+    assert lib.w2a8_linear_grouped_host(p, 1, 256, 2, vp2, vp2, n2, 64, vp2, p, 16, None) == WS
+    assert lib.w2a8_linear_grouped_host_workspace_bytes(2, n2, 1, 256, 64) > lib.w2a8_grouped_workspace_bytes(2, n2, 1, 256, 64)
     assert lib.w2a8_read_probe(None, 1 << 20, p, None) == NULLP
     assert lib.w2a8_read_probe(p + 4, 1 << 20, p, None) == ALIGN
 

@@ -302,6 +302,31 @@ def test_linear_host_end_to_end(gpu, oracle, M, pinned):
         assert ok, worst
 
 
+@pytest.mark.parametrize("M,pinned", [(1, True), (4, True), (16, True), (4, False), (40, True)])
+def test_linear_grouped_host_end_to_end(gpu, oracle, M, pinned):
+    """q|k|v-like group with host buffers in and out: x crosses the bus once, every y lands in its
+    host buffer; zero-copy for few tokens in page-locked buffers, staged copies otherwise."""
+    torch, b = gpu
+    K, Ns, g = 4096, [1024, 256, 256], 64
+    mats = [synth.make_linear(300 + i, K, n, g) for i, n in enumerate(Ns)]
+    bits = synth.activations_bf16(301, M, K)
+    grp = b.Group([b.w2_pack(_dev(torch, c)) for c, _ in mats], [_dev(torch, s) for _, s in mats])
+    x_host = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+    ys = [torch.empty((M, n), dtype=torch.float32) for n in Ns]
+    if pinned:
+        x_host, ys = x_host.pin_memory(), [y.pin_memory() for y in ys]
+    ws = b.new_workspace(b.w2a8_linear_grouped_host_workspace_bytes(Ns, M, K, g))
+    a_ref, s_ref = oracle.quantize(bits)
+    for _ in range(2):
+        for y in ys:
+            y.zero_()
+        b.w2a8_linear_grouped_host(x_host, grp, g, ys, ws)
+        torch.cuda.synchronize()
+        for (codes, s_w), y in zip(mats, ys):
+            ok, worst = _row_err_ok(y.numpy(), oracle.gemm(a_ref, s_ref, codes, s_w, g))
+            assert ok, worst
+
+
 def test_pdl_off_matches(gpu, oracle):
     # the same library with plain launches, in a child process (the switch is read once)
     import subprocess
