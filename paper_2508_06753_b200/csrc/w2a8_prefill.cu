@@ -18,7 +18,8 @@
 // Per 64-k group (or whatever the scale group is) an MMA thread issues K = 32 steps
 // into one of four accumulator buffers (all 512 TMEM columns).  MMA and drain hand
 // buffers over in units of two consecutive groups (a barrier round trip costs as much
-// as the MMAs of a 64-k group); two threads share the issuing, one unit slot each.
+// as the MMAs of a 64-k group); two threads share the issuing, one unit slot each, in
+// straight-line code per stage (the kernel is specialised on the slices per group).
 // Eight "drain" warps (two per TMEM lane quarter, 64 token columns each) read finished
 // buffers with tcgen05.ld, software-pipelined in 32-column halves, convert to fp32 and
 // accumulate scale * value in registers with packed fp32 FMAs.  Stage slots and units
@@ -28,6 +29,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+
+#include <type_traits>
 
 #include "w2a8_tc.cuh"
 
@@ -61,7 +64,7 @@ struct PrefillParams {
 };
 
 // H16: w_scale points at IEEE binary16 values; the result is fp32 or, with p.y16, bf16.
-template <bool PARTIALS, bool H16>
+template <bool PARTIALS, bool H16, int DPS>
 __global__ void __launch_bounds__(kPfThreads, 1)
 w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillParams p) {
     extern __shared__ unsigned char pf_smem_raw[];
@@ -108,60 +111,116 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
 
     if (warp < 2) {
         // ===== MMA issuers (one thread in each of warps 0 and 1) =========================
-        // Issuing is scalar work of a single thread and costs several hundred cycles per
-        // group, so two threads share it.  The hand-off unit between MMA and drain is two
-        // consecutive scale groups (two accumulator buffers, one barrier pair): a barrier
-        // round trip costs a few hundred cycles, as much as the MMAs of a 64-k group, so
-        // halving their number matters.  Thread `mma_id` owns the units with that parity.
-        // Descriptors are a base plus compile-time offsets, bookkeeping uses counters (no
-        // division), the four slices of a stage are unrolled.
+        // The hand-off unit between MMA and drain is two consecutive scale groups (two
+        // accumulator buffers, one barrier pair); thread w owns the units of parity w.
+        // A lone thread runs a dependent instruction every several cycles, so the cost of
+        // issuing is the number of scalar instructions between two MMAs: with loop-carried
+        // bookkeeping and 64-bit descriptor arithmetic one thread issued an MMA every ~200
+        // cycles (measured with producers and drain switched off: 1.3-1.5 POPS for the pair),
+        // three times the 64 cycles the MMA takes.  Written as straight-line code per stage --
+        // the kernel is specialised on the slices per group (DPS = 1, 2, or 0 for groups of
+        // whole stages), K-step offsets are immediates added to the low descriptor word --
+        // the same pair issues at the tensor pipe's rate (3.2-3.3 POPS in that test).
         if (lane == 0) {
-            const int mma_id = warp;
-            constexpr uint32_t idesc = pf_instr_desc(kPfBM, kPfBN);
+            const int w = warp;             // this thread's unit slot: accumulator buffers 2 w and 2 w + 1
             const uint64_t a_desc0 = pf_smem_desc(smem_base);
             const uint64_t b_desc0 = pf_smem_desc(smem_base + 2 * kPfHalfBytes);
+            // Only the low word of a descriptor (start address / 16) changes from step to step
+            const uint32_t a_lo0 = (uint32_t)a_desc0, a_hi = (uint32_t)(a_desc0 >> 32);
+            const uint32_t b_lo0 = (uint32_t)b_desc0, b_hi = (uint32_t)(b_desc0 >> 32);
+            const uint32_t acc_empty_bar = pf_smem_u32(&bar_acc_empty[w]), acc_full_bar = pf_smem_u32(&bar_acc_full[w]);
+            const uint32_t t0 = tmem_base + 2 * w * kPfBN;
             int s = 0;
+            uint32_t so = 0;                // stage offset in 16-byte units
             uint32_t full_parity = 0;
-            int unit0 = 0;                  // units of the tiles before this one
             bool ok = true;
-            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
-                int pos = 0;                // 64-k slices already issued in the current group
-                int group_idx = 0;          // scale groups of this tile completed so far
-                for (int it = 0; it < nstages && ok; ++it) {
-                    ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
-                    if (!ok) break;
-                    pf_tc_fence_after();
-                    const uint64_t stage_off = (uint64_t)((uint32_t)(s * kPfStageBytes) >> 4);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        // unit u: accumulator buffers 2 (u % 2) and 2 (u % 2) + 1
-                        const int u = unit0 + (group_idx >> 1), slot = u & 1;
-                        const bool mine = slot == mma_id;
-                        const int buf = 2 * slot + (group_idx & 1);
-                        if (mine && pos == 0 && (group_idx & 1) == 0 && u >= kPfUnits) {
-                            // the drain warps must have emptied this unit's previous groups
-                            ok = pf_wait(pf_smem_u32(&bar_acc_empty[slot]), ((u >> 1) - 1) & 1, abort_flag);
+            // K step j of a stage (j = 0..7: 64-k slice j / 2, half j % 2 of it) into buffer 2 w + b
+            auto step = [&](auto jc, int b, uint32_t accumulate) {
+                constexpr int j = decltype(jc)::value;
+                constexpr uint32_t koff = ((j >> 2) & 1) * (kPfHalfBytes >> 4) + (j & 3) * 2;
+                const uint64_t ad = ((uint64_t)a_hi << 32) | (a_lo0 + so + koff);
+                const uint64_t bd = ((uint64_t)b_hi << 32) | (b_lo0 + so + koff);
+                pf_mma_i8(t0 + b * kPfBN, ad, bd, pf_instr_desc(kPfBM, kPfBN), accumulate);
+            };
+            auto next_stage = [&]() {
+                pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
+                so += kPfStageBytes >> 4;
+                if (++s == kPfStages) { s = 0; so = 0; full_parity ^= 1u; }
+            };
+            using J0 = std::integral_constant<int, 0>; using J1 = std::integral_constant<int, 1>;
+            using J2 = std::integral_constant<int, 2>; using J3 = std::integral_constant<int, 3>;
+            using J4 = std::integral_constant<int, 4>; using J5 = std::integral_constant<int, 5>;
+            using J6 = std::integral_constant<int, 6>; using J7 = std::integral_constant<int, 7>;
+            if constexpr (DPS == 1) {
+                // 64-k groups: a stage holds two units; ngroups is a multiple of four, so every
+                // tile starts on an even unit and thread w always takes slices 2 w and 2 w + 1.
+                int c = 0;                  // units this thread has issued so far
+                for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                    for (int it = 0; it < nstages && ok; ++it, ++c) {
+                        ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
+                        if (!ok) break;
+                        if (c >= 1) {       // the drain warps must have emptied the unit issued before
+                            ok = pf_wait(acc_empty_bar, (uint32_t)(c - 1) & 1u, abort_flag);
                             if (!ok) break;
-                            pf_tc_fence_after();
                         }
-                        if (mine) {
-#pragma unroll
-                            for (int ks = 0; ks < 2; ++ks) {
-                                constexpr int kHalf16 = kPfHalfBytes >> 4;
-                                const uint64_t off = stage_off + (uint64_t)((q >> 1) * kHalf16 + ((q & 1) * 2 + ks) * 2);
-                                pf_mma_i8(tmem_base + buf * kPfBN, a_desc0 + off, b_desc0 + off, idesc,
-                                          (pos == 0 && ks == 0) ? 0u : 1u);
+                        pf_tc_fence_after();
+                        if (w == 0) { step(J0{}, 0, 0u); step(J1{}, 0, 1u); step(J2{}, 1, 0u); step(J3{}, 1, 1u); }
+                        else        { step(J4{}, 0, 0u); step(J5{}, 0, 1u); step(J6{}, 1, 0u); step(J7{}, 1, 1u); }
+                        pf_mma_commit(acc_full_bar);
+                        next_stage();
+                    }
+                }
+            } else if constexpr (DPS == 2) {
+                // 128-k groups: a stage is one unit; the two threads take alternate stages
+                int u = 0;                  // unit (= stage) index across tiles
+                for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                    for (int it = 0; it < nstages && ok; ++it, ++u) {
+                        ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
+                        if (!ok) break;
+                        if ((u & 1) == w) {
+                            if (u >= kPfUnits) {
+                                ok = pf_wait(acc_empty_bar, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                                if (!ok) break;
                             }
+                            pf_tc_fence_after();
+                            step(J0{}, 0, 0u); step(J1{}, 0, 1u); step(J2{}, 0, 1u); step(J3{}, 0, 1u);
+                            step(J4{}, 1, 0u); step(J5{}, 1, 1u); step(J6{}, 1, 1u); step(J7{}, 1, 1u);
+                            pf_mma_commit(acc_full_bar);
                         }
-                        if (++pos == dps) {
+                        next_stage();
+                    }
+                }
+            } else {
+                // groups of whole stages (a multiple of 256 k): all eight steps of a stage go to
+                // one buffer; unit = two consecutive groups (the last unit of a tile may hold one)
+                const int spg = dps >> 2;   // stages per group
+                int unit0 = 0;              // units of the tiles before this one
+                for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
+                    int group_idx = 0, pos = 0;     // group of this tile, stage inside the group
+                    for (int it = 0; it < nstages && ok; ++it) {
+                        ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
+                        if (!ok) break;
+                        const int u = unit0 + (group_idx >> 1);
+                        const bool mine = (u & 1) == w;
+                        if (mine) {
+                            if (pos == 0 && (group_idx & 1) == 0 && u >= kPfUnits) {
+                                ok = pf_wait(acc_empty_bar, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                                if (!ok) break;
+                            }
+                            pf_tc_fence_after();
+                            const int b = group_idx & 1;
+                            step(J0{}, b, pos == 0 ? 0u : 1u);
+                            step(J1{}, b, 1u); step(J2{}, b, 1u); step(J3{}, b, 1u);
+                            step(J4{}, b, 1u); step(J5{}, b, 1u); step(J6{}, b, 1u); step(J7{}, b, 1u);
+                        }
+                        if (++pos == spg) {
                             pos = 0;
                             const bool unit_done = (group_idx & 1) == 1 || group_idx == ngroups - 1;
-                            if (mine && unit_done) pf_mma_commit(pf_smem_u32(&bar_acc_full[slot]));
+                            if (mine && unit_done) pf_mma_commit(acc_full_bar);
                             ++group_idx;
                         }
+                        next_stage();
                     }
-                    pf_mma_commit(pf_smem_u32(&bar_empty[s]));   // stage can be refilled once these MMAs are done
-                    if (++s == kPfStages) { s = 0; full_parity ^= 1u; }
                 }
             }
         }
@@ -440,15 +499,22 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
     const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
     const int sms = sm_count();
     dim3 grid((unsigned)(tiles < sms ? tiles : sms));   // persistent CTAs, one per SM
-    static PerDeviceFlags configured[3];
+    static PerDeviceFlags configured[9];
     auto launch = [&](auto kernel, int slot) -> bool {
         if (allow_dynamic_smem(kernel, configured[slot], (int)smem) != cudaSuccess) return false;
         kernel<<<grid, kPfThreads, smem, st>>>(map, p);
         return true;
     };
-    const bool launched = partials ? launch(w2a8_prefill_kernel<true, false>, 1)
-                        : h16      ? launch(w2a8_prefill_kernel<false, true>, 2)
-                                   : launch(w2a8_prefill_kernel<false, false>, 0);
+    // The MMA-issuing code is specialised on the 64-k slices per scale group: 1, 2, or whole stages (0)
+    auto launch_dps = [&](auto partials_c, auto h16_c, int slot0) -> bool {
+        constexpr bool P = decltype(partials_c)::value, H = decltype(h16_c)::value;
+        if (group == 64) return launch(w2a8_prefill_kernel<P, H, 1>, slot0);
+        if (group == 128) return launch(w2a8_prefill_kernel<P, H, 2>, slot0 + 1);
+        return launch(w2a8_prefill_kernel<P, H, 0>, slot0 + 2);
+    };
+    const bool launched = partials ? launch_dps(std::true_type{}, std::false_type{}, 3)
+                        : h16      ? launch_dps(std::false_type{}, std::true_type{}, 6)
+                                   : launch_dps(std::false_type{}, std::false_type{}, 0);
     if (!launched) return W2A8_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }

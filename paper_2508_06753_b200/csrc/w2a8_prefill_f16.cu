@@ -18,6 +18,8 @@
 // exact int32 sums of the int8 kernel, bit for bit.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "w2a8_tc.cuh"
 
 namespace w2a8 {
@@ -87,7 +89,7 @@ __device__ __forceinline__ void hf_unpack_word(uint32_t w, uint4 &lo, uint4 &hi)
     hi = make_uint4(r[4], r[5], r[6], r[7]);
 }
 
-template <bool PARTIALS>
+template <bool PARTIALS, int DPS>
 __global__ void __launch_bounds__(kHfThreads, 1)
 w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams p) {
     extern __shared__ unsigned char hf_smem_raw[];
@@ -148,52 +150,92 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
                 }
             }
         }
-        // ===== MMA issuers: thread `mma_id` owns the hand-off units of that parity ===========
+        // ===== MMA issuers: thread w owns the hand-off units of parity w ======================
+        // Straight-line code per stage (see the int8 kernel: the issue rate of a lone thread is
+        // set by the scalar instructions between two MMAs): specialised on the 64-k slices per
+        // group (DPS = 1, 2, or 0 for groups of whole 256-k blocks), K-step offsets as immediates
+        // on the low descriptor word.  A stage is two 64-k sub-tiles of four K = 16 steps each.
         if (warp < 2 && lane == 0) {
-            const int mma_id = warp;
-            constexpr uint32_t idesc = pf_instr_desc_bf16(kHfBM, kHfBN);
+            const int w = warp;
             const uint64_t a_desc0 = pf_smem_desc(smem_base);
             const uint64_t b_desc0 = pf_smem_desc(smem_base + 2 * kHfHalfBytes);
+            const uint32_t a_lo0 = (uint32_t)a_desc0, a_hi = (uint32_t)(a_desc0 >> 32);
+            const uint32_t b_lo0 = (uint32_t)b_desc0, b_hi = (uint32_t)(b_desc0 >> 32);
+            const uint32_t acc_empty_bar = pf_smem_u32(&bar_acc_empty[w]), acc_full_bar = pf_smem_u32(&bar_acc_full[w]);
+            const uint32_t t0 = tmem_base + 2 * w * kHfBN;
             int s = 0;
+            uint32_t so = 0;                // stage offset in 16-byte units
             uint32_t full_parity = 0;
-            int unit0 = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
-                int pos = 0;                // 64-k slices already issued in the current group
-                int group_idx = 0;
-                for (int it = 0; it < nstages && ok; ++it) {
-                    ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
-                    if (!ok) break;
-                    pf_tc_fence_after();
-                    const uint64_t stage_off = (uint64_t)((uint32_t)(s * kHfStageBytes) >> 4);
-#pragma unroll
-                    for (int q = 0; q < 2; ++q) {          // the two 64-k sub-tiles of the stage
-                        const int u = unit0 + (group_idx >> 1), slot = u & 1;
-                        const bool mine = slot == mma_id;
-                        const int buf = 2 * slot + (group_idx & 1);
-                        if (mine && pos == 0 && (group_idx & 1) == 0 && u >= kHfUnits) {
-                            ok = pf_wait(pf_smem_u32(&bar_acc_empty[slot]), ((u >> 1) - 1) & 1, abort_flag);
-                            if (!ok) break;
-                            pf_tc_fence_after();
-                        }
-                        if (mine) {
-#pragma unroll
-                            for (int ks = 0; ks < 4; ++ks) {       // K = 16 per instruction: 32 bytes of the row
-                                constexpr int kHalf16 = kHfHalfBytes >> 4;
-                                const uint64_t off = stage_off + (uint64_t)(q * kHalf16 + ks * 2);
-                                pf_mma_f16(tmem_base + buf * kHfBN, a_desc0 + off, b_desc0 + off, idesc,
-                                           (pos == 0 && ks == 0) ? 0u : 1u);
+            // K step j of a stage (j = 0..7: sub-tile j / 4, step j % 4 of it) into buffer 2 w + b
+            auto step = [&](auto jc, int b, uint32_t accumulate) {
+                constexpr int j = decltype(jc)::value;
+                constexpr uint32_t koff = (j >> 2) * (kHfHalfBytes >> 4) + (j & 3) * 2;
+                const uint64_t ad = ((uint64_t)a_hi << 32) | (a_lo0 + so + koff);
+                const uint64_t bd = ((uint64_t)b_hi << 32) | (b_lo0 + so + koff);
+                pf_mma_f16(t0 + b * kHfBN, ad, bd, pf_instr_desc_bf16(kHfBM, kHfBN), accumulate);
+            };
+            auto next_stage = [&]() {
+                pf_mma_commit(pf_smem_u32(&bar_empty[s]));
+                so += kHfStageBytes >> 4;
+                if (++s == kHfStages) { s = 0; so = 0; full_parity ^= 1u; }
+            };
+            using J0 = std::integral_constant<int, 0>; using J1 = std::integral_constant<int, 1>;
+            using J2 = std::integral_constant<int, 2>; using J3 = std::integral_constant<int, 3>;
+            using J4 = std::integral_constant<int, 4>; using J5 = std::integral_constant<int, 5>;
+            using J6 = std::integral_constant<int, 6>; using J7 = std::integral_constant<int, 7>;
+            if constexpr (DPS == 1) {
+                // 64-k groups: a stage is one unit (two groups); the threads take alternate stages
+                int u = 0;                  // unit (= stage) index across tiles
+                for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                    for (int it = 0; it < nstages && ok; ++it, ++u) {
+                        ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
+                        if (!ok) break;
+                        if ((u & 1) == w) {
+                            if (u >= kHfUnits) {
+                                ok = pf_wait(acc_empty_bar, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                                if (!ok) break;
                             }
+                            pf_tc_fence_after();
+                            step(J0{}, 0, 0u); step(J1{}, 0, 1u); step(J2{}, 0, 1u); step(J3{}, 0, 1u);
+                            step(J4{}, 1, 0u); step(J5{}, 1, 1u); step(J6{}, 1, 1u); step(J7{}, 1, 1u);
+                            pf_mma_commit(acc_full_bar);
                         }
-                        if (++pos == dps) {
+                        next_stage();
+                    }
+                }
+            } else {
+                // groups of one stage (DPS == 2) or of whole 256-k blocks (two stages each): all
+                // eight steps of a stage go to one buffer; unit = two consecutive groups (the
+                // last unit of a tile may hold one)
+                const int spg = dps >> 1;   // stages per group
+                int unit0 = 0;              // units of the tiles before this one
+                for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
+                    int group_idx = 0, pos = 0;     // group of this tile, stage inside the group
+                    for (int it = 0; it < nstages && ok; ++it) {
+                        ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
+                        if (!ok) break;
+                        const int u = unit0 + (group_idx >> 1);
+                        const bool mine = (u & 1) == w;
+                        if (mine) {
+                            if (pos == 0 && (group_idx & 1) == 0 && u >= kHfUnits) {
+                                ok = pf_wait(acc_empty_bar, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                                if (!ok) break;
+                            }
+                            pf_tc_fence_after();
+                            const int b = group_idx & 1;
+                            step(J0{}, b, (DPS == 2 || pos == 0) ? 0u : 1u);
+                            step(J1{}, b, 1u); step(J2{}, b, 1u); step(J3{}, b, 1u);
+                            step(J4{}, b, 1u); step(J5{}, b, 1u); step(J6{}, b, 1u); step(J7{}, b, 1u);
+                        }
+                        if (DPS == 2 || ++pos == spg) {
                             pos = 0;
                             const bool unit_done = (group_idx & 1) == 1 || group_idx == ngroups - 1;
-                            if (mine && unit_done) pf_mma_commit(pf_smem_u32(&bar_acc_full[slot]));
+                            if (mine && unit_done) pf_mma_commit(acc_full_bar);
                             ++group_idx;
                         }
+                        next_stage();
                     }
-                    pf_mma_commit(pf_smem_u32(&bar_empty[s]));
-                    if (++s == kHfStages) { s = 0; full_parity ^= 1u; }
                 }
             }
         }
@@ -417,13 +459,20 @@ int launch_prefill_f16(const void *x_bf16, const float *a_scale, const uint32_t 
     const long long tiles = (long long)(N / kHfBM) * ((M + kHfBN - 1) / kHfBN);
     const int sms = sm_count();
     dim3 grid((unsigned)(tiles < sms ? tiles : sms));
-    static PerDeviceFlags configured[2];
+    static PerDeviceFlags configured[6];
     auto launch = [&](auto kernel, int slot) -> bool {
         if (allow_dynamic_smem(kernel, configured[slot], (int)smem) != cudaSuccess) return false;
         kernel<<<grid, kHfThreads, smem, st>>>(map, p);
         return true;
     };
-    const bool launched = partials ? launch(w2a16_prefill_kernel<true>, 1) : launch(w2a16_prefill_kernel<false>, 0);
+    // the MMA-issuing code is specialised on the 64-k slices per scale group: 1, 2, or whole blocks (0)
+    auto launch_dps = [&](auto partials_c, int slot0) -> bool {
+        constexpr bool P = decltype(partials_c)::value;
+        if (group == 64) return launch(w2a16_prefill_kernel<P, 1>, slot0);
+        if (group == 128) return launch(w2a16_prefill_kernel<P, 2>, slot0 + 1);
+        return launch(w2a16_prefill_kernel<P, 0>, slot0 + 2);
+    };
+    const bool launched = partials ? launch_dps(std::true_type{}, 3) : launch_dps(std::false_type{}, 0);
     if (!launched) return W2A8_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
