@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
 w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillParams p) {
     extern __shared__ unsigned char pf_smem_raw[];
     __shared__ __align__(8) unsigned long long bar_full[kPfStages], bar_empty[kPfStages];
-    __shared__ __align__(8) unsigned long long bar_acc_full[kPfUnits], bar_acc_empty[kPfUnits];
+    __shared__ __align__(8) unsigned long long bar_acc_full[kPfUnits], bar_acc_empty[kPfAccBufs];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     volatile int *abort_flag = &abort_flag_s;
@@ -96,10 +96,10 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             pf_mbar_init(pf_smem_u32(&bar_full[s]), kPfUnpackWarps + 1);
             pf_mbar_init(pf_smem_u32(&bar_empty[s]), 2);      // one tcgen05.commit per MMA-issuing thread
         }
-        for (int b = 0; b < kPfUnits; ++b) {
-            pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);   // tcgen05.commit
-            pf_mbar_init(pf_smem_u32(&bar_acc_empty[b]), 8);  // one arrive per drain warp
-        }
+        for (int b = 0; b < kPfUnits; ++b) pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);   // tcgen05.commit
+        // buffers are handed back one by one (one arrive per drain warp): the MMAs of a unit's
+        // first group start while the drain warps are still reading its second buffer
+        for (int b = 0; b < kPfAccBufs; ++b) pf_mbar_init(pf_smem_u32(&bar_acc_empty[b]), 8);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         pf_fence_proxy_async();
     }
@@ -128,7 +128,8 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             // Only the low word of a descriptor (start address / 16) changes from step to step
             const uint32_t a_lo0 = (uint32_t)a_desc0, a_hi = (uint32_t)(a_desc0 >> 32);
             const uint32_t b_lo0 = (uint32_t)b_desc0, b_hi = (uint32_t)(b_desc0 >> 32);
-            const uint32_t acc_empty_bar = pf_smem_u32(&bar_acc_empty[w]), acc_full_bar = pf_smem_u32(&bar_acc_full[w]);
+            const uint32_t acc_empty_bar0 = pf_smem_u32(&bar_acc_empty[2 * w]), acc_empty_bar1 = pf_smem_u32(&bar_acc_empty[2 * w + 1]);
+            const uint32_t acc_full_bar = pf_smem_u32(&bar_acc_full[w]);
             const uint32_t t0 = tmem_base + 2 * w * kPfBN;
             int s = 0;
             uint32_t so = 0;                // stage offset in 16-byte units
@@ -159,13 +160,17 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     for (int it = 0; it < nstages && ok; ++it, ++c) {
                         ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
                         if (!ok) break;
-                        if (c >= 1) {       // the drain warps must have emptied the unit issued before
-                            ok = pf_wait(acc_empty_bar, (uint32_t)(c - 1) & 1u, abort_flag);
-                            if (!ok) break;
-                        }
+                        // each buffer must have been read out by the drain warps since its last use
+                        if (c >= 1) ok = pf_wait(acc_empty_bar0, (uint32_t)(c - 1) & 1u, abort_flag);
+                        if (!ok) break;
                         pf_tc_fence_after();
-                        if (w == 0) { step(J0{}, 0, 0u); step(J1{}, 0, 1u); step(J2{}, 1, 0u); step(J3{}, 1, 1u); }
-                        else        { step(J4{}, 0, 0u); step(J5{}, 0, 1u); step(J6{}, 1, 0u); step(J7{}, 1, 1u); }
+                        if (w == 0) { step(J0{}, 0, 0u); step(J1{}, 0, 1u); }
+                        else        { step(J4{}, 0, 0u); step(J5{}, 0, 1u); }
+                        if (c >= 1) ok = pf_wait(acc_empty_bar1, (uint32_t)(c - 1) & 1u, abort_flag);
+                        if (!ok) break;
+                        pf_tc_fence_after();
+                        if (w == 0) { step(J2{}, 1, 0u); step(J3{}, 1, 1u); }
+                        else        { step(J6{}, 1, 0u); step(J7{}, 1, 1u); }
                         pf_mma_commit(acc_full_bar);
                         next_stage();
                     }
@@ -178,12 +183,13 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
                         if (!ok) break;
                         if ((u & 1) == w) {
-                            if (u >= kPfUnits) {
-                                ok = pf_wait(acc_empty_bar, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
-                                if (!ok) break;
-                            }
+                            if (u >= kPfUnits) ok = pf_wait(acc_empty_bar0, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                            if (!ok) break;
                             pf_tc_fence_after();
                             step(J0{}, 0, 0u); step(J1{}, 0, 1u); step(J2{}, 0, 1u); step(J3{}, 0, 1u);
+                            if (u >= kPfUnits) ok = pf_wait(acc_empty_bar1, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                            if (!ok) break;
+                            pf_tc_fence_after();
                             step(J4{}, 1, 0u); step(J5{}, 1, 1u); step(J6{}, 1, 1u); step(J7{}, 1, 1u);
                             pf_mma_commit(acc_full_bar);
                         }
@@ -195,6 +201,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 // one buffer; unit = two consecutive groups (the last unit of a tile may hold one)
                 const int spg = dps >> 2;   // stages per group
                 int unit0 = 0;              // units of the tiles before this one
+                int uses0 = 0, uses1 = 0;   // groups this thread has put into its first / second buffer
                 for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
                     int group_idx = 0, pos = 0;     // group of this tile, stage inside the group
                     for (int it = 0; it < nstages && ok; ++it) {
@@ -203,12 +210,14 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         const int u = unit0 + (group_idx >> 1);
                         const bool mine = (u & 1) == w;
                         if (mine) {
-                            if (pos == 0 && (group_idx & 1) == 0 && u >= kPfUnits) {
-                                ok = pf_wait(acc_empty_bar, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                            const int b = group_idx & 1;
+                            if (pos == 0) {     // a new group: its buffer must have been read out since its last use
+                                const int uses = b ? uses1 : uses0;
+                                if (uses >= 1) ok = pf_wait(b ? acc_empty_bar1 : acc_empty_bar0, (uint32_t)(uses - 1) & 1u, abort_flag);
                                 if (!ok) break;
+                                if (b) ++uses1; else ++uses0;
                             }
                             pf_tc_fence_after();
-                            const int b = group_idx & 1;
                             step(J0{}, b, pos == 0 ? 0u : 1u);
                             step(J1{}, b, 1u); step(J2{}, b, 1u); step(J3{}, b, 1u);
                             step(J4{}, b, 1u); step(J5{}, b, 1u); step(J6{}, b, 1u); step(J7{}, b, 1u);
@@ -228,12 +237,17 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         // ===== unpack warps: packed words -> int8 lanes, K-major, 128-byte swizzle =====
         constexpr int kUnits = 512 / (32 * kPfUnpackWarps);   // 16-byte units per thread and stage
         const int ut = (warp - 2) * 32 + lane;
+        // Unit u: 16 bytes of packed words (word t = u % 4 of the four slices) of one row.  The eight
+        // lanes whose 16-byte stores share a shared-memory wavefront take rows that differ by four:
+        // under the 128-byte swizzle (chunk ^= row % 8) their two groups of four chunks are then the
+        // two halves of a 128-byte row, one store per bank (consecutive rows would share a half).
+        auto unit_row = [](int u) { return (u >> 5) * 8 + ((u >> 2) & 1) * 4 + ((u >> 3) & 3); };
         auto request = [&](uint4 (&w)[kUnits], int tile, int it) {
             const int n0 = (tile / tiles_m) * kPfBM;
 #pragma unroll
             for (int i = 0; i < kUnits; ++i) {
                 const int u = ut + 32 * kPfUnpackWarps * i;   // unit: row = u / 4, quarter t = u % 4
-                const int r = u >> 2, t = u & 3;
+                const int r = unit_row(u), t = u & 3;
                 w[i] = __ldg(reinterpret_cast<const uint4 *>(p.packed + (size_t)(n0 + r) * p.words_per_row +
                                                              16 * it + 4 * t));
             }
@@ -267,7 +281,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
 #pragma unroll
                 for (int i = 0; i < kUnits; ++i) {
                     const int u = ut + 32 * kPfUnpackWarps * i;
-                    const int r = u >> 2, t = u & 3;
+                    const int r = unit_row(u), t = u & 3;
                     const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
 #pragma unroll
                     for (int sl = 0; sl < 4; ++sl) {    // slice sl: k = 64 sl + 16 t .. + 15 of this block
@@ -374,11 +388,11 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         for (int j = 0; j < 32; j += 2) pf_fma2(acc[j], acc[j + 1], (float)v0[j], (float)v0[j + 1], sc);
                     }
                     pf_tmem_ld_wait();                     // second half is in v1
-                    if ((gi & 1) == 1 || gi == ngroups - 1) {
-                        // all of this warp's share of the unit (two groups) has been read: hand it back
+                    {
+                        // all of this warp's share of the buffer has been read: hand it back
                         pf_tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[unit & 1]));
+                        if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[buf]));
                     }
                     if (gi + 1 < ngroups) {                // request the first half of the next group
                         const int nunit = unit0 + ((gi + 1) >> 1);

@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(kHfThreads, 1)
 w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams p) {
     extern __shared__ unsigned char hf_smem_raw[];
     __shared__ __align__(8) unsigned long long bar_full[kHfStages], bar_empty[kHfStages];
-    __shared__ __align__(8) unsigned long long bar_acc_full[kHfUnits], bar_acc_empty[kHfUnits];
+    __shared__ __align__(8) unsigned long long bar_acc_full[kHfUnits], bar_acc_empty[kHfAccBufs];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     volatile int *abort_flag = &abort_flag_s;
@@ -115,10 +115,9 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
             pf_mbar_init(pf_smem_u32(&bar_full[s]), kHfUnpackWarps + 1);   // unpack warps + the TMA producer
             pf_mbar_init(pf_smem_u32(&bar_empty[s]), 2);                   // one commit per MMA-issuing thread
         }
-        for (int b = 0; b < kHfUnits; ++b) {
-            pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);
-            pf_mbar_init(pf_smem_u32(&bar_acc_empty[b]), 8);
-        }
+        for (int b = 0; b < kHfUnits; ++b) pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);
+        // buffers are handed back one by one (one arrive per drain warp)
+        for (int b = 0; b < kHfAccBufs; ++b) pf_mbar_init(pf_smem_u32(&bar_acc_empty[b]), 8);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         pf_fence_proxy_async();
     }
@@ -161,7 +160,8 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
             const uint64_t b_desc0 = pf_smem_desc(smem_base + 2 * kHfHalfBytes);
             const uint32_t a_lo0 = (uint32_t)a_desc0, a_hi = (uint32_t)(a_desc0 >> 32);
             const uint32_t b_lo0 = (uint32_t)b_desc0, b_hi = (uint32_t)(b_desc0 >> 32);
-            const uint32_t acc_empty_bar = pf_smem_u32(&bar_acc_empty[w]), acc_full_bar = pf_smem_u32(&bar_acc_full[w]);
+            const uint32_t acc_empty_bar0 = pf_smem_u32(&bar_acc_empty[2 * w]), acc_empty_bar1 = pf_smem_u32(&bar_acc_empty[2 * w + 1]);
+            const uint32_t acc_full_bar = pf_smem_u32(&bar_acc_full[w]);
             const uint32_t t0 = tmem_base + 2 * w * kHfBN;
             int s = 0;
             uint32_t so = 0;                // stage offset in 16-byte units
@@ -192,12 +192,14 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
                         ok = pf_wait(pf_smem_u32(&bar_full[s]), full_parity, abort_flag);
                         if (!ok) break;
                         if ((u & 1) == w) {
-                            if (u >= kHfUnits) {
-                                ok = pf_wait(acc_empty_bar, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
-                                if (!ok) break;
-                            }
+                            // each buffer must have been read out by the drain warps since its last use
+                            if (u >= kHfUnits) ok = pf_wait(acc_empty_bar0, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                            if (!ok) break;
                             pf_tc_fence_after();
                             step(J0{}, 0, 0u); step(J1{}, 0, 1u); step(J2{}, 0, 1u); step(J3{}, 0, 1u);
+                            if (u >= kHfUnits) ok = pf_wait(acc_empty_bar1, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                            if (!ok) break;
+                            pf_tc_fence_after();
                             step(J4{}, 1, 0u); step(J5{}, 1, 1u); step(J6{}, 1, 1u); step(J7{}, 1, 1u);
                             pf_mma_commit(acc_full_bar);
                         }
@@ -210,6 +212,7 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
                 // last unit of a tile may hold one)
                 const int spg = dps >> 1;   // stages per group
                 int unit0 = 0;              // units of the tiles before this one
+                int uses0 = 0, uses1 = 0;   // groups this thread has put into its first / second buffer
                 for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
                     int group_idx = 0, pos = 0;     // group of this tile, stage inside the group
                     for (int it = 0; it < nstages && ok; ++it) {
@@ -218,12 +221,14 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
                         const int u = unit0 + (group_idx >> 1);
                         const bool mine = (u & 1) == w;
                         if (mine) {
-                            if (pos == 0 && (group_idx & 1) == 0 && u >= kHfUnits) {
-                                ok = pf_wait(acc_empty_bar, (uint32_t)((u >> 1) - 1) & 1u, abort_flag);
+                            const int b = group_idx & 1;
+                            if (pos == 0) {     // a new group: its buffer must have been read out since its last use
+                                const int uses = b ? uses1 : uses0;
+                                if (uses >= 1) ok = pf_wait(b ? acc_empty_bar1 : acc_empty_bar0, (uint32_t)(uses - 1) & 1u, abort_flag);
                                 if (!ok) break;
+                                if (b) ++uses1; else ++uses0;
                             }
                             pf_tc_fence_after();
-                            const int b = group_idx & 1;
                             step(J0{}, b, (DPS == 2 || pos == 0) ? 0u : 1u);
                             step(J1{}, b, 1u); step(J2{}, b, 1u); step(J3{}, b, 1u);
                             step(J4{}, b, 1u); step(J5{}, b, 1u); step(J6{}, b, 1u); step(J7{}, b, 1u);
@@ -348,10 +353,10 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
                             pf_fma2(acc[j], acc[j + 1], __int_as_float(v0[j]), __int_as_float(v0[j + 1]), sc);
                     }
                     pf_tmem_ld_wait();                     // second half is in v1
-                    if ((gi & 1) == 1 || gi == ngroups - 1) {
+                    {   // this warp's share of the buffer has been read: hand it back
                         pf_tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[unit & 1]));
+                        if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_acc_empty[buf]));
                     }
                     if (gi + 1 < ngroups) {                // request the first half of the next group
                         const int nunit = unit0 + ((gi + 1) >> 1);
