@@ -385,7 +385,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         }
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) pf_fma2(acc[j], acc[j + 1], (float)v0[j], (float)v0[j + 1], sc);
+                        for (int j = 0; j < 32; j += 2) pf_cvt_fma2<DPS == 1 || DPS == 2>(acc[j], acc[j + 1], v0[j], v0[j + 1], sc);
                     }
                     pf_tmem_ld_wait();                     // second half is in v1
                     {
@@ -397,7 +397,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     if (gi + 1 < ngroups) {                // request the first half of the next group
                         const int nunit = unit0 + ((gi + 1) >> 1);
                         if (((gi + 1) & 1) == 0) {         // it opens a new unit: wait for its MMAs
-                            ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[nunit & 1]), (nunit >> 1) & 1, abort_flag);
+                            ok = pf_wait(pf_smem_u32(&bar_acc_full[nunit & 1]), (nunit >> 1) & 1, abort_flag);   // all lanes poll: no broadcast step
                             if (!ok) break;
                             pf_tc_fence_after();
                         }
@@ -412,7 +412,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; j += 2)
-                            pf_fma2(acc[32 + j], acc[32 + j + 1], (float)v1[j], (float)v1[j + 1], sc);
+                            pf_cvt_fma2<DPS == 1 || DPS == 2>(acc[32 + j], acc[32 + j + 1], v1[j], v1[j + 1], sc);
                     }
                 }
             }

@@ -95,6 +95,28 @@ __device__ __forceinline__ void pf_fma2(float &acc0, float &acc1, float x0, floa
         "mov.b64 {%0, %1}, c;\n\t}"
         : "+f"(acc0), "+f"(acc1) : "f"(x0), "f"(x1), "f"(sc));
 }
+// (acc0, acc1) += (float(d0), float(d1)) * sc for int32 d0, d1.  MAGIC (|d| < 2^22 only): the
+// float is built as bits(d + 0x4B400000) = 12582912 + d (exact: below 2^24 in magnitude, one unit
+// in the last place is 1) and the offset is taken off again by one packed subtraction, which is
+// exact too: the result equals float(d) bit for bit, from full-rate integer and float
+// instructions instead of the int-to-float conversion, which issues at a quarter of their rate.
+template <bool MAGIC>
+__device__ __forceinline__ void pf_cvt_fma2(float &acc0, float &acc1, int d0, int d1, float sc) {
+    if constexpr (MAGIC) {
+        const float x0 = __int_as_float(d0 + 0x4B400000), x1 = __int_as_float(d1 + 0x4B400000);
+        asm("{\n\t.reg .b64 a, b, c, m;\n\t"
+            "mov.b64 a, {%2, %3};\n\t"
+            "mov.b64 m, {%5, %5};\n\t"
+            "add.rn.f32x2 a, a, m;\n\t"
+            "mov.b64 b, {%4, %4};\n\t"
+            "mov.b64 c, {%0, %1};\n\t"
+            "fma.rn.f32x2 c, a, b, c;\n\t"
+            "mov.b64 {%0, %1}, c;\n\t}"
+            : "+f"(acc0), "+f"(acc1) : "f"(x0), "f"(x1), "f"(sc), "f"(-12582912.0f));
+    } else {
+        pf_fma2(acc0, acc1, (float)d0, (float)d1, sc);
+    }
+}
 __device__ __forceinline__ void pf_tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major [rows][128 B] tile stored with the
