@@ -36,8 +36,15 @@
 
 namespace w2a8 {
 
-constexpr int kPfUnpackWarps = 2;
-constexpr int kPfThreads = 32 * (2 + kPfUnpackWarps + 8);   // warps: 2 MMA issuers, unpack (+TMA), 8 drain
+// Two warp layouts (template parameter UW = unpack warps):
+//   UW = 2: 12 warps -- 2 MMA issuers, 2 unpack warps (lane 0 of the first also issues the TMA
+//           loads), 8 drain warps; every thread has the same 168 registers.
+//   UW = 4: 16 warps in four warpgroups whose registers are re-balanced at entry (setmaxnreg):
+//           warps 0-3 two MMA issuers, the TMA producer, one spare (56 registers per thread);
+//           warps 4-7 unpack (104); warps 8-15 drain (176).
+__host__ __device__ constexpr int pf_threads(int uw) { return uw == 4 ? 512 : 384; }
+__host__ __device__ constexpr int pf_first_unpack(int uw) { return uw == 4 ? 4 : 2; }
+__host__ __device__ constexpr int pf_first_drain(int uw) { return uw == 4 ? 8 : 4; }
 constexpr int kPfDrainCols = 64;         // token columns per drain warp (two warps share a lane quarter)
 constexpr int kPfBM = 128;               // channels per tile (UMMA M)
 constexpr int kPfBN = 128;               // tokens per tile (UMMA N)
@@ -64,8 +71,13 @@ struct PrefillParams {
 };
 
 // H16: w_scale points at IEEE binary16 values; the result is fp32 or, with p.y16, bf16.
-template <bool PARTIALS, bool H16, int DPS>
-__global__ void __launch_bounds__(kPfThreads, 1)
+template <int N>
+__device__ __forceinline__ void pf_setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void pf_setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+template <bool PARTIALS, bool H16, int DPS, int UW>
+__global__ void __launch_bounds__(pf_threads(UW), 1)
 w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillParams p) {
     extern __shared__ unsigned char pf_smem_raw[];
     __shared__ __align__(8) unsigned long long bar_full[kPfStages], bar_empty[kPfStages];
@@ -93,7 +105,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         abort_flag_s = 0;
         for (int s = 0; s < kPfStages; ++s) {
             // one arrive per unpack warp + the TMA producer's arrive with its transaction bytes
-            pf_mbar_init(pf_smem_u32(&bar_full[s]), kPfUnpackWarps + 1);
+            pf_mbar_init(pf_smem_u32(&bar_full[s]), UW + 1);
             pf_mbar_init(pf_smem_u32(&bar_empty[s]), 2);      // one tcgen05.commit per MMA-issuing thread
         }
         for (int b = 0; b < kPfUnits; ++b) pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);   // tcgen05.commit
@@ -109,7 +121,32 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     pf_tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp < 2) {
+    constexpr int kFirstUnpack = pf_first_unpack(UW), kFirstDrain = pf_first_drain(UW);
+    if (warp < kFirstUnpack) {
+        if constexpr (UW == 4) {
+            pf_setmaxnreg_dec<56>();
+            if (warp == 2 && lane == 0) {
+                // ===== TMA producer: activations, 128 tokens x 256 k per stage ===============
+                int s = 0, round = 0;
+                for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+                    const int m0 = (tile % tiles_m) * kPfBN;
+                    bool ok = true;
+                    for (int it = 0; it < nstages; ++it) {
+                        if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t bar = pf_smem_u32(&bar_full[s]);
+                        const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
+                        pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
+                        pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
+                        pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
+                        if (++s == kPfStages) { s = 0; ++round; }
+                    }
+                    if (!ok) break;
+                }
+            }
+        }
         // ===== MMA issuers (one thread in each of warps 0 and 1) =========================
         // The hand-off unit between MMA and drain is two consecutive scale groups (two
         // accumulator buffers, one barrier pair); thread w owns the units of parity w.
@@ -121,7 +158,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         // the kernel is specialised on the slices per group (DPS = 1, 2, or 0 for groups of
         // whole stages), K-step offsets are immediates added to the low descriptor word --
         // the same pair issues at the tensor pipe's rate (3.2-3.3 POPS in that test).
-        if (lane == 0) {
+        if (warp < 2 && lane == 0) {
             const int w = warp;             // this thread's unit slot: accumulator buffers 2 w and 2 w + 1
             const uint64_t a_desc0 = pf_smem_desc(smem_base);
             const uint64_t b_desc0 = pf_smem_desc(smem_base + 2 * kPfHalfBytes);
@@ -233,10 +270,11 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 }
             }
         }
-    } else if (warp < 2 + kPfUnpackWarps) {
+    } else if (warp < kFirstDrain) {
+        if constexpr (UW == 4) pf_setmaxnreg_dec<104>();
         // ===== unpack warps: packed words -> int8 lanes, K-major, 128-byte swizzle =====
-        constexpr int kUnits = 512 / (32 * kPfUnpackWarps);   // 16-byte units per thread and stage
-        const int ut = (warp - 2) * 32 + lane;
+        constexpr int kUnits = 512 / (32 * UW);   // 16-byte units per thread and stage
+        const int ut = (warp - kFirstUnpack) * 32 + lane;
         // Unit u: 16 bytes of packed words (word t = u % 4 of the four slices) of one row.  The eight
         // lanes whose 16-byte stores share a shared-memory wavefront take rows that differ by four:
         // under the 128-byte swizzle (chunk ^= row % 8) their two groups of four chunks are then the
@@ -246,7 +284,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             const int n0 = (tile / tiles_m) * kPfBM;
 #pragma unroll
             for (int i = 0; i < kUnits; ++i) {
-                const int u = ut + 32 * kPfUnpackWarps * i;   // unit: row = u / 4, quarter t = u % 4
+                const int u = ut + 32 * UW * i;
                 const int r = unit_row(u), t = u & 3;
                 w[i] = __ldg(reinterpret_cast<const uint4 *>(p.packed + (size_t)(n0 + r) * p.words_per_row +
                                                              16 * it + 4 * t));
@@ -269,7 +307,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     ok = false;
                     break;
                 }
-                if (warp == 2 && lane == 0) {
+                if (UW == 2 && warp == 2 && lane == 0) {
                     // this lane is also the TMA producer: activations, 128 tokens x 256 k per stage
                     const uint32_t bar = pf_smem_u32(&bar_full[s]);
                     const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
@@ -280,7 +318,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 unsigned char *a_stage = smem_gen + s * kPfStageBytes;
 #pragma unroll
                 for (int i = 0; i < kUnits; ++i) {
-                    const int u = ut + 32 * kPfUnpackWarps * i;
+                    const int u = ut + 32 * UW * i;
                     const int r = unit_row(u), t = u & 3;
                     const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
 #pragma unroll
@@ -301,7 +339,8 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     } else {
         // ===== drain warps: TMEM -> registers, fp32 accumulate with the group scale ======
         const int q4 = warp & 3;                    // TMEM lane quarter this warp may access
-        const int col0 = ((warp - 2 - kPfUnpackWarps) >> 2) * kPfDrainCols;   // first token column of this warp
+        if constexpr (UW == 4) pf_setmaxnreg_inc<176>();
+        const int col0 = ((warp - kFirstDrain) >> 2) * kPfDrainCols;   // first token column of this warp
         const int ch = q4 * 32 + lane;              // channel inside the tile = TMEM lane
         const uint32_t tlane = tmem_base + ((uint32_t)(q4 * 32) << 16) + col0;
         bool ok = true;
@@ -442,6 +481,18 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
 }
 
 // ---- host side -----------------------------------------------------------------------
+int env_int(const char *name, int dflt);
+
+// Unpack warps (warp layout) by scale group; W2A8_PF_UNPACK_WARPS = 2 or 4 overrides.
+int prefill_unpack_warps(int group) {
+    const int forced = env_int("W2A8_PF_UNPACK_WARPS", 0);
+    if (forced == 2 || forced == 4) return forced;
+    // Measured on B200 (4096 -> 14336, 2048 tokens, POPS with 2 / 4 unpack warps): group 64: 717 / 637;
+    // 128: 946 / 1006; 256: 1105 / 1328; K: 1130 / 1455.  With 64-k groups the drain warps are the
+    // bottleneck and two more warps competing for their issue slots cost more than a faster unpack
+    // gains; from 128 up the unpack is.
+    return group >= 128 ? 4 : 2;
+}
 bool prefill_supported(int M, int N, int K, int group) {
     if (M < 64) return false;
     if (N % kPfBM != 0 || K % kPfBK != 0) return false;
@@ -513,22 +564,30 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
     const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
     const int sms = sm_count();
     dim3 grid((unsigned)(tiles < sms ? tiles : sms));   // persistent CTAs, one per SM
-    static PerDeviceFlags configured[9];
-    auto launch = [&](auto kernel, int slot) -> bool {
+    static PerDeviceFlags configured[15];
+    auto launch = [&](auto kernel, int slot, int threads) -> bool {
         if (allow_dynamic_smem(kernel, configured[slot], (int)smem) != cudaSuccess) return false;
-        kernel<<<grid, kPfThreads, smem, st>>>(map, p);
+        kernel<<<grid, threads, smem, st>>>(map, p);
         return true;
     };
-    // The MMA-issuing code is specialised on the 64-k slices per scale group: 1, 2, or whole stages (0)
-    auto launch_dps = [&](auto partials_c, auto h16_c, int slot0) -> bool {
+    // The MMA-issuing code is specialised on the 64-k slices per scale group: 1, 2, or whole stages
+    // (0); the warp layout on the number of unpack warps (the parity export keeps the 12-warp one).
+    const int uw = prefill_unpack_warps(group);
+    auto launch_dps = [&](auto partials_c, auto h16_c, auto uw_c, int slot0) -> bool {
         constexpr bool P = decltype(partials_c)::value, H = decltype(h16_c)::value;
-        if (group == 64) return launch(w2a8_prefill_kernel<P, H, 1>, slot0);
-        if (group == 128) return launch(w2a8_prefill_kernel<P, H, 2>, slot0 + 1);
-        return launch(w2a8_prefill_kernel<P, H, 0>, slot0 + 2);
+        constexpr int U = decltype(uw_c)::value;
+        if (group == 64) return launch(w2a8_prefill_kernel<P, H, 1, U>, slot0, pf_threads(U));
+        if (group == 128) return launch(w2a8_prefill_kernel<P, H, 2, U>, slot0 + 1, pf_threads(U));
+        return launch(w2a8_prefill_kernel<P, H, 0, U>, slot0 + 2, pf_threads(U));
     };
-    const bool launched = partials ? launch_dps(std::true_type{}, std::false_type{}, 3)
-                        : h16      ? launch_dps(std::false_type{}, std::true_type{}, 6)
-                                   : launch_dps(std::false_type{}, std::false_type{}, 0);
+    using U2 = std::integral_constant<int, 2>;
+    using U4 = std::integral_constant<int, 4>;
+    const bool launched =
+        partials ? launch_dps(std::true_type{}, std::false_type{}, U2{}, 3)
+        : h16    ? (uw == 4 ? launch_dps(std::false_type{}, std::true_type{}, U4{}, 12)
+                            : launch_dps(std::false_type{}, std::true_type{}, U2{}, 6))
+                 : (uw == 4 ? launch_dps(std::false_type{}, std::false_type{}, U4{}, 9)
+                            : launch_dps(std::false_type{}, std::false_type{}, U2{}, 0));
     if (!launched) return W2A8_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
