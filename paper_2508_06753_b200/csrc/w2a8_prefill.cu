@@ -105,7 +105,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         abort_flag_s = 0;
         for (int s = 0; s < kPfStages; ++s) {
             // one arrive per unpack warp + the TMA producer's arrive with its transaction bytes
-            pf_mbar_init(pf_smem_u32(&bar_full[s]), UW + 1);
+            pf_mbar_init(pf_smem_u32(&bar_full[s]), 2 + 1);   // the two unpack warps of a team + the TMA producer
             pf_mbar_init(pf_smem_u32(&bar_empty[s]), 2);      // one tcgen05.commit per MMA-issuing thread
         }
         for (int b = 0; b < kPfUnits; ++b) pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);   // tcgen05.commit
@@ -273,8 +273,13 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     } else if (warp < kFirstDrain) {
         if constexpr (UW == 4) pf_setmaxnreg_dec<104>();
         // ===== unpack warps: packed words -> int8 lanes, K-major, 128-byte swizzle =====
-        constexpr int kUnits = 512 / (32 * UW);   // 16-byte units per thread and stage
-        const int ut = (warp - kFirstUnpack) * 32 + lane;
+        // Teams of two warps; team j fills stages j, j + kTeams, ... (numbered across tiles).  With
+        // two teams a stage's fixed costs -- the wait for the slot, the proxy fence, the arrive --
+        // overlap the other team's unpack instead of adding to every stage.
+        constexpr int kTeams = UW / 2;
+        constexpr int kUnits = 8;                   // 16-byte units per thread and stage
+        const int team = (warp - kFirstUnpack) >> 1;
+        const int ut = ((warp - kFirstUnpack) & 1) * 32 + lane;
         // Unit u: 16 bytes of packed words (word t = u % 4 of the four slices) of one row.  The eight
         // lanes whose 16-byte stores share a shared-memory wavefront take rows that differ by four:
         // under the 128-byte swizzle (chunk ^= row % 8) their two groups of four chunks are then the
@@ -284,57 +289,60 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             const int n0 = (tile / tiles_m) * kPfBM;
 #pragma unroll
             for (int i = 0; i < kUnits; ++i) {
-                const int u = ut + 32 * UW * i;
+                const int u = ut + 64 * i;
                 const int r = unit_row(u), t = u & 3;
                 w[i] = __ldg(reinterpret_cast<const uint4 *>(p.packed + (size_t)(n0 + r) * p.words_per_row +
                                                              16 * it + 4 * t));
             }
         };
+        auto advance = [&](int &tile, int &it) {    // the next stage in the order the CTA walks them
+            if (++it == nstages) { it = 0; tile += gridDim.x; }
+        };
+        int tile = blockIdx.x, it = 0;
+        for (int j = 0; j < team; ++j) advance(tile, it);
+        int s = team, round = 0;                    // slot and use count of the slot for this team's stage
         uint4 w_nxt[kUnits];
-        if ((int)blockIdx.x < ntiles) request(w_nxt, blockIdx.x, 0);
-        int s = 0, round = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
-            const int m0 = (tile % tiles_m) * kPfBN;
-            for (int it = 0; it < nstages; ++it) {
-                uint4 w[kUnits];
+        if (tile < ntiles) request(w_nxt, tile, it);
+        while (tile < ntiles) {
+            uint4 w[kUnits];
 #pragma unroll
-                for (int i = 0; i < kUnits; ++i) w[i] = w_nxt[i];
-                // next stage's words in flight (possibly the first stage of the next tile)
-                if (it + 1 < nstages) request(w_nxt, tile, it + 1);
-                else if (tile + (int)gridDim.x < ntiles) request(w_nxt, tile + gridDim.x, 0);
-                if (round > 0 && !pf_wait_warp(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                if (UW == 2 && warp == 2 && lane == 0) {
-                    // this lane is also the TMA producer: activations, 128 tokens x 256 k per stage
-                    const uint32_t bar = pf_smem_u32(&bar_full[s]);
-                    const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
-                    pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
-                    pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
-                    pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
-                }
-                unsigned char *a_stage = smem_gen + s * kPfStageBytes;
+            for (int i = 0; i < kUnits; ++i) w[i] = w_nxt[i];
+            // the words of this team's next stage in flight (possibly in the next tile)
+            int tile_nxt = tile, it_nxt = it;
 #pragma unroll
-                for (int i = 0; i < kUnits; ++i) {
-                    const int u = ut + 32 * UW * i;
-                    const int r = unit_row(u), t = u & 3;
-                    const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
-#pragma unroll
-                    for (int sl = 0; sl < 4; ++sl) {    // slice sl: k = 64 sl + 16 t .. + 15 of this block
-                        uint4 v;
-                        v.x = lane_codes(ws[sl], 0); v.y = lane_codes(ws[sl], 1);
-                        v.z = lane_codes(ws[sl], 2); v.w = lane_codes(ws[sl], 3);
-                        const int chunk = (4 * (sl & 1) + t) ^ (r & 7);
-                        *reinterpret_cast<uint4 *>(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16) = v;
-                    }
-                }
-                pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
-                __syncwarp();
-                if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full[s]));
-                if (++s == kPfStages) { s = 0; ++round; }
+            for (int j = 0; j < kTeams; ++j) advance(tile_nxt, it_nxt);
+            if (tile_nxt < ntiles) request(w_nxt, tile_nxt, it_nxt);
+            if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
+            if (UW == 2 && warp == kFirstUnpack && lane == 0) {
+                // this lane is also the TMA producer: activations, 128 tokens x 256 k per stage
+                const int m0 = (tile % tiles_m) * kPfBN;
+                const uint32_t bar = pf_smem_u32(&bar_full[s]);
+                const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
+                pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
+                pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
+                pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
             }
+            unsigned char *a_stage = smem_gen + s * kPfStageBytes;
+#pragma unroll
+            for (int i = 0; i < kUnits; ++i) {
+                const int u = ut + 64 * i;
+                const int r = unit_row(u), t = u & 3;
+                const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) {    // slice sl: k = 64 sl + 16 t .. + 15 of this block
+                    uint4 v;
+                    v.x = lane_codes(ws[sl], 0); v.y = lane_codes(ws[sl], 1);
+                    v.z = lane_codes(ws[sl], 2); v.w = lane_codes(ws[sl], 3);
+                    const int chunk = (4 * (sl & 1) + t) ^ (r & 7);
+                    *reinterpret_cast<uint4 *>(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16) = v;
+                }
+            }
+            pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
+            __syncwarp();
+            if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full[s]));
+            tile = tile_nxt; it = it_nxt;
+            s += kTeams;
+            if (s >= kPfStages) { s -= kPfStages; ++round; }
         }
     } else {
         // ===== drain warps: TMEM -> registers, fp32 accumulate with the group scale ======

@@ -274,7 +274,7 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
                     if (it + 2 < nstages) request(w_nxt, tile, (it >> 1) + 1);
                     else if (tile + (int)gridDim.x < ntiles) request(w_nxt, tile + gridDim.x, 0);
                 }
-                if (round > 0 && !pf_wait_warp(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) {
+                if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) {
                     ok = false;
                     break;
                 }
@@ -361,7 +361,7 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
                     if (gi + 1 < ngroups) {                // request the first half of the next group
                         const int nunit = unit0 + ((gi + 1) >> 1);
                         if (((gi + 1) & 1) == 0) {
-                            ok = pf_wait_warp(pf_smem_u32(&bar_acc_full[nunit & 1]), (nunit >> 1) & 1, abort_flag);
+                            ok = pf_wait(pf_smem_u32(&bar_acc_full[nunit & 1]), (nunit >> 1) & 1, abort_flag);
                             if (!ok) break;
                             pf_tc_fence_after();
                         }
