@@ -30,8 +30,7 @@ int env_int(const char *name, int dflt);
 //   warps 0-3   two MMA issuers, the TMA producer, one spare       (56 registers per thread)
 //   warps 4-7   unpack                                             (104)
 //   warps 8-15  drain: 64 fp32 accumulators + 64 staged values     (176)
-constexpr int kHfUnpackWarps = 4;
-constexpr int kHfFirstUnpackWarp = 4;
+constexpr int kHfFirstUnpackWarp = 4;    // four unpack warps: two teams of two
 constexpr int kHfFirstDrainWarp = 8;
 constexpr int kHfThreads = 32 * 16;
 constexpr int kHfDrainCols = 64;         // token columns per drain warp (two warps share a lane quarter)
@@ -112,7 +111,7 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         for (int s = 0; s < kHfStages; ++s) {
-            pf_mbar_init(pf_smem_u32(&bar_full[s]), kHfUnpackWarps + 1);   // unpack warps + the TMA producer
+            pf_mbar_init(pf_smem_u32(&bar_full[s]), 2 + 1);   // the two unpack warps of a team + the TMA producer
             pf_mbar_init(pf_smem_u32(&bar_empty[s]), 2);                   // one commit per MMA-issuing thread
         }
         for (int b = 0; b < kHfUnits; ++b) pf_mbar_init(pf_smem_u32(&bar_acc_full[b]), 1);
@@ -247,57 +246,58 @@ w2a16_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const HfParams
     } else if (warp < kHfFirstDrainWarp) {
         hf_setmaxnreg_dec<104>();
         // ===== unpack warps: packed words -> bf16 values, K-major, 128-byte swizzle =========
-        // A thread owns four 16-byte units of every block (row r = u / 4, quarter t = u % 4); a
-        // unit holds word t of each of the block's four slices, two of which belong to a stage.
-        constexpr int kUnits = 512 / (32 * kHfUnpackWarps);
-        const int ut = (warp - kHfFirstUnpackWarp) * 32 + lane;
-        auto request = [&](uint4 (&w)[kUnits], int tile, int blk) {
+        // Two teams of two warps; a stage is half a 256-k block, so team j fills every stage of
+        // parity j: slices 2 j and 2 j + 1 of each block.  A stage's fixed costs (the wait for the
+        // slot, the proxy fence, the arrive) overlap the other team's unpack.  A thread owns eight
+        // units of a stage (row r = u / 4, quarter t = u % 4): word t of the stage's two slices.
+        constexpr int kUnits = 8;
+        const int team = (warp - kHfFirstUnpackWarp) >> 1;
+        const int ut = ((warp - kHfFirstUnpackWarp) & 1) * 32 + lane;
+        auto request = [&](uint2 (&w)[kUnits], int tile, int blk) {
             const int n0 = (tile / tiles_m) * kHfBM;
 #pragma unroll
             for (int i = 0; i < kUnits; ++i) {
-                const int u = ut + 32 * kHfUnpackWarps * i;
+                const int u = ut + 64 * i;
                 const int r = u >> 2, t = u & 3;
-                w[i] = __ldg(reinterpret_cast<const uint4 *>(p.packed + (size_t)(n0 + r) * p.words_per_row +
-                                                             16 * blk + 4 * t));
+                w[i] = __ldg(reinterpret_cast<const uint2 *>(p.packed + (size_t)(n0 + r) * p.words_per_row +
+                                                             16 * blk + 4 * t + 2 * team));
             }
         };
-        uint4 w_cur[kUnits], w_nxt[kUnits];
-        if ((int)blockIdx.x < ntiles) request(w_nxt, blockIdx.x, 0);
-        int s = 0, round = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
-            for (int it = 0; it < nstages; ++it) {
-                if ((it & 1) == 0) {
+        const int nblocks = nstages >> 1;
+        int tile = blockIdx.x, blk = 0;
+        int s = team, round = 0;                    // slot and use count of the slot for this team's stage
+        uint2 w_nxt[kUnits];
+        if (tile < ntiles) request(w_nxt, tile, 0);
+        while (tile < ntiles) {
+            uint2 w_cur[kUnits];
 #pragma unroll
-                    for (int i = 0; i < kUnits; ++i) w_cur[i] = w_nxt[i];
-                    // next block's words in flight (possibly the first block of the next tile)
-                    if (it + 2 < nstages) request(w_nxt, tile, (it >> 1) + 1);
-                    else if (tile + (int)gridDim.x < ntiles) request(w_nxt, tile + gridDim.x, 0);
-                }
-                if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                unsigned char *a_stage = smem_gen + s * kHfStageBytes;
+            for (int i = 0; i < kUnits; ++i) w_cur[i] = w_nxt[i];
+            // next block's words in flight (possibly the first block of the next tile)
+            int tile_nxt = tile, blk_nxt = blk + 1;
+            if (blk_nxt == nblocks) { blk_nxt = 0; tile_nxt += gridDim.x; }
+            if (tile_nxt < ntiles) request(w_nxt, tile_nxt, blk_nxt);
+            if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
+            unsigned char *a_stage = smem_gen + s * kHfStageBytes;
 #pragma unroll
-                for (int i = 0; i < kUnits; ++i) {
-                    const int u = ut + 32 * kHfUnpackWarps * i;
-                    const int r = u >> 2, t = u & 3;
-                    const uint32_t ws[2] = {(it & 1) ? w_cur[i].z : w_cur[i].x, (it & 1) ? w_cur[i].w : w_cur[i].y};
+            for (int i = 0; i < kUnits; ++i) {
+                const int u = ut + 64 * i;
+                const int r = u >> 2, t = u & 3;
+                const uint32_t ws[2] = {w_cur[i].x, w_cur[i].y};
 #pragma unroll
-                    for (int sl = 0; sl < 2; ++sl) {    // slice sl of the stage: k = 64 sl + 16 t .. + 15
-                        uint4 lo, hi;
-                        hf_unpack_word(ws[sl], lo, hi);
-                        unsigned char *row = a_stage + sl * kHfHalfBytes + r * 128;
-                        *reinterpret_cast<uint4 *>(row + (((2 * t) ^ (r & 7)) << 4)) = lo;
-                        *reinterpret_cast<uint4 *>(row + (((2 * t + 1) ^ (r & 7)) << 4)) = hi;
-                    }
+                for (int sl = 0; sl < 2; ++sl) {    // slice sl of the stage: k = 64 sl + 16 t .. + 15
+                    uint4 lo, hi;
+                    hf_unpack_word(ws[sl], lo, hi);
+                    unsigned char *row = a_stage + sl * kHfHalfBytes + r * 128;
+                    *reinterpret_cast<uint4 *>(row + (((2 * t) ^ (r & 7)) << 4)) = lo;
+                    *reinterpret_cast<uint4 *>(row + (((2 * t + 1) ^ (r & 7)) << 4)) = hi;
                 }
-                pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
-                __syncwarp();
-                if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full[s]));
-                if (++s == kHfStages) { s = 0; ++round; }
             }
+            pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
+            __syncwarp();
+            if (lane == 0) pf_mbar_arrive(pf_smem_u32(&bar_full[s]));
+            tile = tile_nxt; blk = blk_nxt;
+            s += 2;
+            if (s >= kHfStages) { s -= kHfStages; ++round; }
         }
     } else {
         hf_setmaxnreg_inc<176>();
