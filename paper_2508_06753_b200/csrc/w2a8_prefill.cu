@@ -509,18 +509,27 @@ bool prefill_supported(int M, int N, int K, int group) {
     return true;
 }
 
+// Cost of one round of tiles (one 128 x 128 tile per SM) in seconds per unit of K, by scale group:
+// the drain runs once per group, so larger groups are cheaper.  From the kernel's measured rates on
+// B200 at 4096 -> 14336, 2048 tokens (12 rounds): group 64: 717 TOPS = 6.8 ns per k and round (the
+// rule keeps the 7 ns it was fitted with), 128: 1021 = 4.8, 256: 1356 = 3.6, K: 1657 = 2.9.
+static double prefill_round_seconds_per_k(int group) {
+    return group <= 64 ? 7.0e-9 : group <= 128 ? 4.8e-9 : group <= 256 ? 3.6e-9 : 3.0e-9;
+}
+constexpr double kStreamSecondsPerMac = 8.0e-15;    // streaming kernel, per token x weight
+
 // Whether the tensor-core kernel is expected to beat the streaming kernel on a shape it supports.
 // Its grid is one CTA per 128 x 128 output tile (at most one per SM), each walking all of K, so a
-// problem with few tiles leaves most SMs idle: on B200 a round of tiles takes about 7 ns per unit
-// of K, the streaming kernel about 8e-15 s per token x weight, which crosses at M * N of about
-// 0.95 million per round (measured: 14336x4096 at M = 128: 94 us against 66 us streaming; at
+// problem with few tiles leaves most SMs idle.  At group 64 the two cost models cross at M * N of
+// about 0.95 million per round (measured: 14336x4096 at M = 128: 94 us against 66 us streaming; at
 // M = 256: 97 against 127; 4096x4096 at M = 64: 31 against 11).
 bool prefill_preferred(int M, int N, int K, int group) {
-    (void)K; (void)group;
+    (void)K;
     const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
     const long long sms = sm_count();
     const long long rounds = (tiles + sms - 1) / sms;
-    return (long long)M * N > rounds * 950000ll;
+    const double per_round = 950000.0 * prefill_round_seconds_per_k(group) / 7.0e-9;
+    return (double)M * (double)N > (double)rounds * per_round;
 }
 
 // How many of the N channels the tensor-core kernel should take when the rest may go to the
@@ -530,15 +539,15 @@ bool prefill_preferred(int M, int N, int K, int group) {
 // streaming kernel can remove that round.  Same cost model as prefill_preferred, plus 2 us for
 // the extra launch.  Returns a multiple of 128 in (0, N].
 int prefill_channel_split(int M, int N, int K, int group) {
-    (void)group;
     const int ct = N / kPfBM, tiles_m = (M + kPfBN - 1) / kPfBN;
     const long long sms = sm_count();
+    const double round_s = prefill_round_seconds_per_k(group) * K;
     double best = 1e30;
     int best_ct = ct;
     for (int c = ct; c >= 1 && c >= ct - 8; --c) {
         const long long rounds = ((long long)c * tiles_m + sms - 1) / sms;
-        double t = (double)rounds * K * 7.0e-9;
-        if (c < ct) t += 2.0e-6 + 8.0e-15 * (double)M * (double)(ct - c) * kPfBM * (double)K;
+        double t = (double)rounds * round_s;
+        if (c < ct) t += 2.0e-6 + kStreamSecondsPerMac * (double)M * (double)(ct - c) * kPfBM * (double)K;
         if (t < best * 0.97) { best = t; best_ct = c; }      // a split has to pay by 3 % or more
     }
     return best_ct * kPfBM;
