@@ -1081,6 +1081,49 @@ def prefill_probe(device, peaks, Ms=(512, 2048, 8192), reps=5):
     else:
         os.environ["W2A8_TC_KIND"] = saved_kind
     del packed, s_w_d
+    # Few output tiles (64-256 tokens on the 8B layer's matrices): the tensor-core kernel with K split
+    # over the otherwise idle SMs, next to the same kernel unsplit and to the streaming kernel
+    few = []
+    saved = {k: os.environ.get(k) for k in ("W2A8_PREFILL", "W2A8_PF_KSPLIT")}
+
+    def set_env(**kv):
+        for k, v in kv.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+    for (K, N) in ((4096, 4096), (14336, 4096), (4096, 14336)):
+        g = 64
+        codes, s_w = synth.make_linear(synth.shape_seed(cfg, 0) + K + N, K, N, g)
+        packed = b.w2_pack(torch.from_numpy(codes).to(device))
+        s_w_d = torch.from_numpy(s_w).to(device)
+        del codes
+        for M in (64, 128, 256):
+            bits = synth.activations_bf16(cfg["seed"] + 11 + M, M, K)
+            x = torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+            a, s_a = b.a8_quantize(x)
+            y = torch.empty((M, N), dtype=torch.float32, device=device)
+            row = {"shape": f"{K}x{N}", "M": M, "group": g}
+            for label, env in (("default", dict(W2A8_PREFILL=None, W2A8_PF_KSPLIT=None)),
+                               ("tensor_core_unsplit", dict(W2A8_PREFILL="2", W2A8_PF_KSPLIT="1")),
+                               ("streaming", dict(W2A8_PREFILL="0", W2A8_PF_KSPLIT=None))):
+                set_env(**env)
+                ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g), device=device)
+                stream = side_stream(torch)
+
+                def body():
+                    for _ in range(4):
+                        b.w2a8_gemm(a, s_a, packed, s_w_d, g, ws, y)
+                run, how = capture(torch, body, stream)          # env switches are read at capture time
+                t = timed_blocks(torch, run, stream, blocks=5, reps=3)
+                torch.cuda.current_stream().wait_stream(stream)
+                row[label] = {"us": t["mean"] / 4 * 1e3, "us_min": t["min"] / 4 * 1e3, "timing": how,
+                              "kernel": b.w2a8_kernel_for(M, N, K, g),
+                              "k_splits": b.w2a8_tensor_core_ksplit(M, N, K, g), "status": b.w2a8_workspace_status(ws)}
+                del ws, run
+            few.append(row)
+        del packed, s_w_d
+    set_env(**saved)
     # library int8 GEMM on the same device as a second, directly measured denominator
     lib_int8 = None
     try:
@@ -1105,6 +1148,7 @@ def prefill_probe(device, peaks, Ms=(512, 2048, 8192), reps=5):
             "peak_measured_sustained": int8_peak_sustained,
             "peak_note": "measured cuBLAS bf16 peak x 2 (nominal int8 : bf16 ratio); nominal dense int8 4500",
             "library_int8_gemm": lib_int8, "rows": rows, "by_group_m2048": by_group,
+            "few_tile_k_split": few,
             "kind_f16_kernel": {"what": "16-bit tensor-core kernel (tcgen05 kind::f16, fp32 accumulators, no conversion "
                                         "in the drain): op/s counted as for the int8 kernel", "rows": alt}}
 

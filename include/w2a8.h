@@ -227,6 +227,21 @@ int w2a8_tensor_core_kind(int M, int N, int K, int group);
 int w2a8_tensor_core_channels(int M, int N, int K, int group);
 
 /*
+ * How many ways the tensor-core kernel splits K for this shape: 0 when the
+ * streaming kernel takes the problem, else 1, 2, 4 or 8.  A problem with few
+ * 128 x 128 output tiles would leave most SMs idle; with a split every tile
+ * becomes that many work items (each a whole number of 256-k blocks and of
+ * scale groups), whose fp32 partial outputs go to the workspace and are added
+ * in split order by a second, small kernel on the same stream -- so the result
+ * does not depend on timing, and differs from the unsplit sum only by the order
+ * of fp32 additions (Sec. II-D: splitting along K to put all cores to work).
+ * w2a8_workspace_bytes covers the partial outputs.  W2A8_PF_KSPLIT = 1, 2, 4, 8
+ * forces a count where it divides the shape.  Host only.  W2A8_ERR_SHAPE for a
+ * shape that is not accepted.
+ */
+int w2a8_tensor_core_ksplit(int M, int N, int K, int group);
+
+/*
  * w2a8_gemm_partials -- parity/debug export of the exact int32 per-group sums
  * P[m][n][gi] computed by the same inner-product code as w2a8_gemm.
  *   partials [M][N][K/group] int32, fully overwritten.

@@ -24,7 +24,9 @@ int launch_gemv(const int8_t *a, const float *a_scale, const void *x_bf16, int8_
                 const int *N, const int *ldy, int M, int K, int group, cudaStream_t st);
 
 bool prefill_supported(int M, int N, int K, int group);
-bool prefill_preferred(int M, int N, int K, int group);
+bool prefill_preferred(int M, int N, int K, int group, bool can_split);
+size_t prefill_workspace_bytes(int M, int N, int K, int group);
+int prefill_ksplit(int M, int N, int K, int group);
 int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
                    void *y, int32_t *partials, int M, int N, int K, int group, int *status,
                    cudaStream_t st, bool h16, bool y16, int ldy);
@@ -302,6 +304,7 @@ int a8_quantize(const void *x_bf16, int M, int K, int8_t *a, float *a_scale, voi
 }
 
 static bool takes_tensor_core_kernel(int M, int N, int K, int group);
+static bool takes_tensor_core_kernel_ex(int M, int N, int K, int group, bool can_split);
 static int tensor_core_channels(int M, int N, int K, int group);
 
 static bool tensor_core_kind_is_16(int M, int N, int K, int group);
@@ -312,6 +315,9 @@ static size_t kernel_workspace_bytes(int M, int N, int K, int group) {
     if (!shape_ok(M, N, K, group, &si)) return 0;
     size_t need = decode_workspace_bytes(M, N, K, si);
     if (takes_tensor_core_kernel(M, N, K, group)) {
+        // partial outputs of a K split of the int8 tensor-core kernel
+        const size_t split = prefill_workspace_bytes(M, N, K, group);
+        if (split > need) need = split;
         // the last channel tiles may be given to the streaming kernel, with a plan of its own
         const int n_tc = tensor_core_channels(M, N, K, group);
         ShapeInfo rest;
@@ -351,12 +357,16 @@ int w2a8_workspace_status(const void *workspace, void *stream) {
 
 // W2A8_PREFILL: 0 = never the tensor-core kernel, 2 = whenever it supports the shape, else
 // (default) when it supports the shape and is expected to be the faster one.
-static bool takes_tensor_core_kernel(int M, int N, int K, int group) {
+static bool takes_tensor_core_kernel_ex(int M, int N, int K, int group, bool can_split) {
     if (!prefill_supported(M, N, K, group)) return false;
     const int mode = env_int("W2A8_PREFILL", 1);
     if (mode == 0) return false;
     if (mode == 2) return true;
-    return prefill_preferred(M, N, K, group);
+    return prefill_preferred(M, N, K, group, can_split);
+}
+// int8 activations: the int8 kernel can split K for problems with few output tiles, the 16-bit one cannot
+static bool takes_tensor_core_kernel(int M, int N, int K, int group) {
+    return takes_tensor_core_kernel_ex(M, N, K, group, !tensor_core_kind_is_16(M, N, K, group));
 }
 
 // Channels the tensor-core kernel takes (the rest, if any, goes to the streaming kernel in a
@@ -408,6 +418,14 @@ int w2a8_tensor_core_channels(int M, int N, int K, int group) {
     return takes_tensor_core_kernel(M, N, K, group) ? tensor_core_channels(M, N, K, group) : 0;
 }
 
+int w2a8_tensor_core_ksplit(int M, int N, int K, int group) {
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
+    if (!takes_tensor_core_kernel(M, N, K, group)) return 0;
+    if (tensor_core_kind_is_16(M, N, K, group)) return 1;
+    return prefill_ksplit(M, N, K, group);
+}
+
 }  // extern "C"
 
 namespace w2a8 {
@@ -435,9 +453,10 @@ size_t gemm_header_bytes(int M, int N, int K, int group) {
 int gemm_dispatch(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
                   void *y, int32_t *partials, int M, int N, int K, int group, const ShapeInfo &si,
                   void *workspace, void *stream, bool h16, bool y16, bool a16) {
-    const bool tc16 = !h16 && prefill_f16_supported(M, N, K, group) && takes_tensor_core_kernel(M, N, K, group) &&
+    const bool takes = a16 ? takes_tensor_core_kernel_ex(M, N, K, group, false) : takes_tensor_core_kernel(M, N, K, group);
+    const bool tc16 = !h16 && takes && prefill_f16_supported(M, N, K, group) &&
                       (a16 || tensor_core_kind_is_16(M, N, K, group));
-    if (tc16 || (!a16 && takes_tensor_core_kernel(M, N, K, group))) {
+    if (tc16 || (!a16 && takes)) {
         // The tensor-core kernel takes the first n_tc channels; when a last round of a few tiles
         // would cost a whole round, the remaining channel tiles go to the streaming kernel in a
         // second launch (rows of the packed matrix and of the scales are independent; both kernels

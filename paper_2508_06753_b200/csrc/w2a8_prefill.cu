@@ -68,6 +68,8 @@ struct PrefillParams {
     int slices_per_group;    // group / 64
     int y16;                 // 16-bit instance only: y holds bf16 instead of fp32
     int ldy;                 // elements between consecutive token rows of y (>= N)
+    int ks_shift;            // log2 of the K splits S: work item = tile * S + split; each split walks K / S
+    float *split_out;        // S > 1: [S][M][N] fp32 partial outputs (summed in split order by a second kernel)
 };
 
 // H16: w_scale points at IEEE binary16 values; the result is fp32 or, with p.y16, bf16.
@@ -76,7 +78,9 @@ __device__ __forceinline__ void pf_setmaxnreg_dec() { asm volatile("setmaxnreg.d
 template <int N>
 __device__ __forceinline__ void pf_setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
-template <bool PARTIALS, bool H16, int DPS, int UW>
+// SPLIT: work items are (tile, K split) pairs; without it the split count is the constant 1 (the
+// general form costs 15 % on the unsplit problem: 596 against 702 TOPS at 2048 tokens, group 64).
+template <bool PARTIALS, bool H16, int DPS, int UW, bool SPLIT>
 __global__ void __launch_bounds__(pf_threads(UW), 1)
 w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillParams p) {
     extern __shared__ unsigned char pf_smem_raw[];
@@ -87,16 +91,21 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     volatile int *abort_flag = &abort_flag_s;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nstages = p.K / kPfBK;        // stages per tile
+    const int ks_shift = SPLIT ? p.ks_shift : 0;
+    const int nsplit = 1 << ks_shift;       // K splits: a work item is one tile over K / nsplit
+    const int nstages = (p.K / kPfBK) >> ks_shift;        // stages per work item
     const int dps = p.slices_per_group;     // 64-k slices between two drains
-    const int ngroups = (p.K / 64) / dps;   // scale groups per tile
+    const int ngroups = ((p.K / 64) >> ks_shift) / dps;   // scale groups per work item
     const int units_per_tile = (ngroups + 1) / 2;
     // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; consecutive tiles share the
     // channel tile and differ in the token tile, so neighbouring CTAs re-use weights from L2.
     // Stage slots and accumulator units are numbered across tiles (the pipeline does not drain
     // between tiles: producers run ahead into the next tile while the drain warps store y).
     const int tiles_m = (p.M + kPfBN - 1) / kPfBN;
-    const int ntiles = (p.N / kPfBM) * tiles_m;
+    const int ntiles = ((p.N / kPfBM) * tiles_m) << ks_shift;   // work items; `tile` below is a work-item index
+    auto item_n0 = [&](int item) { return ((item >> ks_shift) / tiles_m) * kPfBM; };     // first channel
+    auto item_m0 = [&](int item) { return ((item >> ks_shift) % tiles_m) * kPfBN; };     // first token
+    auto item_stage0 = [&](int item) { return (item & (nsplit - 1)) * nstages; };          // first 256-k block
     // stage buffers, 1024-byte aligned (swizzle atom = 8 rows x 128 B)
     const uint32_t smem_base = (pf_smem_u32(pf_smem_raw) + 1023u) & ~1023u;
     unsigned char *smem_gen = pf_smem_raw + (smem_base - pf_smem_u32(pf_smem_raw));
@@ -129,7 +138,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 // ===== TMA producer: activations, 128 tokens x 256 k per stage ===============
                 int s = 0, round = 0;
                 for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-                    const int m0 = (tile % tiles_m) * kPfBN;
+                    const int m0 = item_m0(tile), k0 = item_stage0(tile) * kPfBK;
                     bool ok = true;
                     for (int it = 0; it < nstages; ++it) {
                         if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) {
@@ -139,8 +148,8 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         const uint32_t bar = pf_smem_u32(&bar_full[s]);
                         const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
                         pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
-                        pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
-                        pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
+                        pf_tma_load_2d(dst, &act_map, k0 + it * kPfBK, m0, bar);
+                        pf_tma_load_2d(dst + kPfHalfBytes, &act_map, k0 + it * kPfBK + 128, m0, bar);
                         if (++s == kPfStages) { s = 0; ++round; }
                     }
                     if (!ok) break;
@@ -286,13 +295,13 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         // two halves of a 128-byte row, one store per bank (consecutive rows would share a half).
         auto unit_row = [](int u) { return (u >> 5) * 8 + ((u >> 2) & 1) * 4 + ((u >> 3) & 3); };
         auto request = [&](uint4 (&w)[kUnits], int tile, int it) {
-            const int n0 = (tile / tiles_m) * kPfBM;
+            const int n0 = item_n0(tile), blk = item_stage0(tile) + it;
 #pragma unroll
             for (int i = 0; i < kUnits; ++i) {
                 const int u = ut + 64 * i;
                 const int r = unit_row(u), t = u & 3;
                 w[i] = __ldg(reinterpret_cast<const uint4 *>(p.packed + (size_t)(n0 + r) * p.words_per_row +
-                                                             16 * it + 4 * t));
+                                                             16 * blk + 4 * t));
             }
         };
         auto advance = [&](int &tile, int &it) {    // the next stage in the order the CTA walks them
@@ -315,12 +324,12 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
             if (round > 0 && !pf_wait(pf_smem_u32(&bar_empty[s]), (round - 1) & 1, abort_flag)) break;
             if (UW == 2 && warp == kFirstUnpack && lane == 0) {
                 // this lane is also the TMA producer: activations, 128 tokens x 256 k per stage
-                const int m0 = (tile % tiles_m) * kPfBN;
+                const int m0 = item_m0(tile), k = (item_stage0(tile) + it) * kPfBK;
                 const uint32_t bar = pf_smem_u32(&bar_full[s]);
                 const uint32_t dst = smem_base + s * kPfStageBytes + 2 * kPfHalfBytes;
                 pf_mbar_arrive_expect_tx(bar, 2 * kPfHalfBytes);
-                pf_tma_load_2d(dst, &act_map, it * kPfBK, m0, bar);
-                pf_tma_load_2d(dst + kPfHalfBytes, &act_map, it * kPfBK + 128, m0, bar);
+                pf_tma_load_2d(dst, &act_map, k, m0, bar);
+                pf_tma_load_2d(dst + kPfHalfBytes, &act_map, k + 128, m0, bar);
             }
             unsigned char *a_stage = smem_gen + s * kPfStageBytes;
 #pragma unroll
@@ -354,21 +363,23 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
         bool ok = true;
         int unit0 = 0;                              // units of the tiles before this one
         for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, unit0 += units_per_tile) {
-            const int n = (tile / tiles_m) * kPfBM + ch;
-            const int m0 = (tile % tiles_m) * kPfBN;
+            const int n = item_n0(tile) + ch;
+            const int m0 = item_m0(tile);
+            const int split = tile & (nsplit - 1);
+            const int gbase = split * ngroups;          // first scale group of this work item
             float acc[kPfDrainCols];
 #pragma unroll
             for (int j = 0; j < kPfDrainCols; ++j) acc[j] = 0.f;
             // Scales are fetched eight groups ahead (a drain takes a few hundred cycles, a
             // global load several hundred): a ring of eight, refilled once per eight groups.
-            const float *sc_row = PARTIALS ? nullptr : p.w_scale + (size_t)n * p.G;
-            const unsigned short *sc_row_h = reinterpret_cast<const unsigned short *>(p.w_scale) + (size_t)n * p.G;
+            const float *sc_row = PARTIALS ? nullptr : p.w_scale + (size_t)n * p.G + gbase;
+            const unsigned short *sc_row_h = reinterpret_cast<const unsigned short *>(p.w_scale) + (size_t)n * p.G + gbase;
             // The ring holds what the loads return, untouched: any instruction that reads a
             // loaded register makes the warp wait for that load.  fp32: eight values.  binary16:
             // eight values widened when they are taken out -- fetched as one 16-byte load when the
             // row pitch allows (G % 8 == 0: registers 0..3 hold two scales each), else as eight
             // 16-bit loads into 32-bit registers.
-            const bool vec8 = H16 && (p.G % 8 == 0);
+            const bool vec8 = H16 && (p.G % 8 == 0) && (gbase % 8 == 0);
             uint32_t sc_nxt[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
             auto refill = [&](int g0) {
                 if constexpr (PARTIALS) {
@@ -470,7 +481,8 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     const int m = m0 + col0 + j;
                     if (m < p.M) {
                         const float v = acc[j] * (__ldg(p.a_scale + m) * (1.0f / kCodeGain));
-                        if (H16 && p.y16) reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)m * p.ldy + n] = __float2bfloat16_rn(v);
+                        if (SPLIT)        p.split_out[((size_t)split * p.M + m) * p.N + n] = v;
+                        else if (H16 && p.y16) reinterpret_cast<__nv_bfloat16 *>(p.y)[(size_t)m * p.ldy + n] = __float2bfloat16_rn(v);
                         else              p.y[(size_t)m * p.ldy + n] = v;
                     }
                 }
@@ -485,6 +497,28 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     if (warp == 1) {
         pf_tc_fence_after();
         pf_tmem_dealloc(tmem_base, kPfTmemCols);
+    }
+}
+
+// Sum of the K-split partial outputs in split order (fixed order: the result does not depend on
+// which CTA finished first).  One thread per four consecutive channels.
+__global__ void pf_splitk_reduce_kernel(const float *__restrict__ split_out, void *__restrict__ y, int M, int N,
+                                        int nsplit, int ldy, int y16) {
+    const size_t quads = (size_t)M * (N / 4);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < quads; i += (size_t)gridDim.x * blockDim.x) {
+        const int m = (int)(i / (N / 4)), n = (int)(i % (N / 4)) * 4;
+        float4 acc = __ldcs(reinterpret_cast<const float4 *>(split_out + (size_t)m * N + n));
+        for (int sidx = 1; sidx < nsplit; ++sidx) {
+            const float4 v = __ldcs(reinterpret_cast<const float4 *>(split_out + ((size_t)sidx * M + m) * N + n));
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        if (y16) {
+            __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(y) + (size_t)m * ldy + n;
+            out[0] = __float2bfloat16_rn(acc.x); out[1] = __float2bfloat16_rn(acc.y);
+            out[2] = __float2bfloat16_rn(acc.z); out[3] = __float2bfloat16_rn(acc.w);
+        } else {
+            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(y) + (size_t)m * ldy + n) = acc;
+        }
     }
 }
 
@@ -518,18 +552,59 @@ static double prefill_round_seconds_per_k(int group) {
 }
 constexpr double kStreamSecondsPerMac = 8.0e-15;    // streaming kernel, per token x weight
 
-// Whether the tensor-core kernel is expected to beat the streaming kernel on a shape it supports.
-// Its grid is one CTA per 128 x 128 output tile (at most one per SM), each walking all of K, so a
-// problem with few tiles leaves most SMs idle.  At group 64 the two cost models cross at M * N of
-// about 0.95 million per round (measured: 14336x4096 at M = 128: 94 us against 66 us streaming; at
-// M = 256: 97 against 127; 4096x4096 at M = 64: 31 against 11).
-bool prefill_preferred(int M, int N, int K, int group) {
-    (void)K;
-    const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
+constexpr size_t kPfSplitOffset = 256;              // byte offset of the K-split partial outputs in the workspace
+
+// Estimated time of the tensor-core path with the work of every tile split `nsplit` ways along K:
+// rounds of one work item per SM, each K / nsplit long, plus (split only) the launch of the summing
+// kernel and its traffic.
+static double prefill_seconds(int M, int N, int K, int group, int nsplit) {
+    const long long items = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN) * nsplit;
     const long long sms = sm_count();
-    const long long rounds = (tiles + sms - 1) / sms;
-    const double per_round = 950000.0 * prefill_round_seconds_per_k(group) / 7.0e-9;
-    return (double)M * (double)N > (double)rounds * per_round;
+    const long long rounds = (items + sms - 1) / sms;
+    double t = (double)rounds * (K / nsplit) * prefill_round_seconds_per_k(group);
+    if (nsplit > 1) t += 2.0e-6 + (double)(nsplit + 1) * M * N * 4.0 / 3.0e12;
+    return t;
+}
+
+// K splits for a shape the kernel supports: 1, 2, 4 or 8.  A problem with few output tiles leaves
+// most SMs idle (one CTA per 128 x 128 tile walking all of K); splitting K puts more of them to work
+// at the price of fp32 partial outputs in the workspace and a second, small kernel that adds them in
+// split order.  Every split is a whole number of 256-k blocks and of scale groups, at least two blocks.
+// W2A8_PF_KSPLIT = 1, 2, 4, 8 forces a count (if it divides the shape).
+int prefill_ksplit(int M, int N, int K, int group) {
+    auto valid = [&](int sp) {
+        if (sp == 1) return true;
+        const int ks = K / sp;
+        return K % sp == 0 && ks % kPfBK == 0 && ks % group == 0 && ks >= 2 * kPfBK;
+    };
+    const int forced = env_int("W2A8_PF_KSPLIT", 0);
+    if (forced == 1 || forced == 2 || forced == 4 || forced == 8) return valid(forced) ? forced : 1;
+    int best = 1;
+    double best_t = prefill_seconds(M, N, K, group, 1);
+    for (int sp = 2; sp <= 8; sp *= 2) {
+        if (!valid(sp)) continue;
+        const double t = prefill_seconds(M, N, K, group, sp);
+        if (t < best_t * 0.95) { best_t = t; best = sp; }      // a split has to pay by 5 % or more
+    }
+    return best;
+}
+
+// Bytes the kernel needs in the workspace (behind the status word) for a shape: the K-split partial outputs.
+size_t prefill_workspace_bytes(int M, int N, int K, int group) {
+    const int sp = prefill_ksplit(M, N, K, group);
+    return sp > 1 ? kPfSplitOffset + (size_t)sp * M * N * sizeof(float) : 0;
+}
+
+// Whether the tensor-core kernel is expected to beat the streaming kernel on a shape it supports.
+// At group 64 without a K split the two cost models cross at M * N of about 0.95 million per round of
+// tiles (measured: 14336x4096 at M = 128: 94 us against 66 us streaming; at M = 256: 97 against 127;
+// 4096x4096 at M = 64: 31 against 11); the same margin (the tensor-core estimate has to be 8 % below
+// the streaming one) is kept with a split.  `can_split` = false: the caller's kernel has no K split.
+bool prefill_preferred(int M, int N, int K, int group, bool can_split) {
+    const int sp = can_split ? prefill_ksplit(M, N, K, group) : 1;
+    const double t_tc = prefill_seconds(M, N, K, group, sp);
+    const double t_stream = kStreamSecondsPerMac * (double)M * (double)N * (double)K;
+    return t_tc * (950000.0 / 875000.0) < t_stream;
 }
 
 // How many of the N channels the tensor-core kernel should take when the rest may go to the
@@ -539,6 +614,7 @@ bool prefill_preferred(int M, int N, int K, int group) {
 // streaming kernel can remove that round.  Same cost model as prefill_preferred, plus 2 us for
 // the extra launch.  Returns a multiple of 128 in (0, N].
 int prefill_channel_split(int M, int N, int K, int group) {
+    if (prefill_ksplit(M, N, K, group) > 1) return N;   // few tiles: K is split instead
     const int ct = N / kPfBM, tiles_m = (M + kPfBN - 1) / kPfBN;
     const long long sms = sm_count();
     const double round_s = prefill_round_seconds_per_k(group) * K;
@@ -577,11 +653,16 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
     p.M = M; p.N = N; p.K = K; p.G = K / group; p.group = group;
     p.words_per_row = K / 16;
     p.slices_per_group = group / 64;
+    // K split: only for the whole matrix (the caller gives no channel remainder to the streaming
+    // kernel then) and never for the parity export
+    const int nsplit = (partials || ldy != N) ? 1 : prefill_ksplit(M, N, K, group);
+    p.ks_shift = nsplit == 8 ? 3 : nsplit == 4 ? 2 : nsplit == 2 ? 1 : 0;
+    p.split_out = nsplit > 1 ? reinterpret_cast<float *>(reinterpret_cast<char *>(status) + kPfSplitOffset) : nullptr;
     const size_t smem = (size_t)kPfStages * kPfStageBytes + 1024;
-    const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN);
+    const long long tiles = (long long)(N / kPfBM) * ((M + kPfBN - 1) / kPfBN) * nsplit;
     const int sms = sm_count();
     dim3 grid((unsigned)(tiles < sms ? tiles : sms));   // persistent CTAs, one per SM
-    static PerDeviceFlags configured[15];
+    static PerDeviceFlags configured[21];
     auto launch = [&](auto kernel, int slot, int threads) -> bool {
         if (allow_dynamic_smem(kernel, configured[slot], (int)smem) != cudaSuccess) return false;
         kernel<<<grid, threads, smem, st>>>(map, p);
@@ -589,23 +670,36 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
     };
     // The MMA-issuing code is specialised on the 64-k slices per scale group: 1, 2, or whole stages
     // (0); the warp layout on the number of unpack warps (the parity export keeps the 12-warp one).
-    const int uw = prefill_unpack_warps(group);
+    // A K split runs on the group's default layout only.
+    const int uw = nsplit > 1 ? (group >= 128 ? 4 : 2) : prefill_unpack_warps(group);
     auto launch_dps = [&](auto partials_c, auto h16_c, auto uw_c, int slot0) -> bool {
         constexpr bool P = decltype(partials_c)::value, H = decltype(h16_c)::value;
         constexpr int U = decltype(uw_c)::value;
-        if (group == 64) return launch(w2a8_prefill_kernel<P, H, 1, U>, slot0, pf_threads(U));
-        if (group == 128) return launch(w2a8_prefill_kernel<P, H, 2, U>, slot0 + 1, pf_threads(U));
-        return launch(w2a8_prefill_kernel<P, H, 0, U>, slot0 + 2, pf_threads(U));
+        if (group == 64) return launch(w2a8_prefill_kernel<P, H, 1, U, false>, slot0, pf_threads(U));
+        if (group == 128) return launch(w2a8_prefill_kernel<P, H, 2, U, false>, slot0 + 1, pf_threads(U));
+        return launch(w2a8_prefill_kernel<P, H, 0, U, false>, slot0 + 2, pf_threads(U));
+    };
+    auto launch_split = [&](auto h16_c, int slot0) -> bool {
+        constexpr bool H = decltype(h16_c)::value;
+        if (group == 64) return launch(w2a8_prefill_kernel<false, H, 1, 2, true>, slot0, pf_threads(2));
+        if (group == 128) return launch(w2a8_prefill_kernel<false, H, 2, 4, true>, slot0 + 1, pf_threads(4));
+        return launch(w2a8_prefill_kernel<false, H, 0, 4, true>, slot0 + 2, pf_threads(4));
     };
     using U2 = std::integral_constant<int, 2>;
     using U4 = std::integral_constant<int, 4>;
     const bool launched =
-        partials ? launch_dps(std::true_type{}, std::false_type{}, U2{}, 3)
-        : h16    ? (uw == 4 ? launch_dps(std::false_type{}, std::true_type{}, U4{}, 12)
-                            : launch_dps(std::false_type{}, std::true_type{}, U2{}, 6))
-                 : (uw == 4 ? launch_dps(std::false_type{}, std::false_type{}, U4{}, 9)
-                            : launch_dps(std::false_type{}, std::false_type{}, U2{}, 0));
+        partials     ? launch_dps(std::true_type{}, std::false_type{}, U2{}, 3)
+        : nsplit > 1 ? (h16 ? launch_split(std::true_type{}, 18) : launch_split(std::false_type{}, 15))
+        : h16        ? (uw == 4 ? launch_dps(std::false_type{}, std::true_type{}, U4{}, 12)
+                                : launch_dps(std::false_type{}, std::true_type{}, U2{}, 6))
+                     : (uw == 4 ? launch_dps(std::false_type{}, std::false_type{}, U4{}, 9)
+                                : launch_dps(std::false_type{}, std::false_type{}, U2{}, 0));
     if (!launched) return W2A8_ERR_CUDA;
+    if (nsplit > 1) {
+        const size_t quads = (size_t)M * (N / 4);
+        const unsigned blocks = (unsigned)((quads + 255) / 256 < (size_t)(8 * sms) ? (quads + 255) / 256 : (size_t)(8 * sms));
+        pf_splitk_reduce_kernel<<<blocks, 256, 0, st>>>(p.split_out, y, M, N, nsplit, ldy, p.y16);
+    }
     return cudaGetLastError() == cudaSuccess ? W2A8_OK : W2A8_ERR_CUDA;
 }
 

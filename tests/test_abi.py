@@ -169,7 +169,7 @@ def test_dispatch_queries_need_no_gpu(lib, monkeypatch):
     """Which kernel serves a shape, and how the channels are split between the two kernels, is
     host logic: pinned here on the shapes of the benchmark configurations."""
     from paper_2508_06753_b200 import binding as b
-    for name in ("W2A8_PREFILL", "W2A8_PF_SPLIT"):
+    for name in ("W2A8_PREFILL", "W2A8_PF_SPLIT", "W2A8_PF_KSPLIT", "W2A8_TC_KIND"):
         monkeypatch.delenv(name, raising=False)
     # few tokens: streaming kernel
     for M in (1, 4, 16, 32, 63):
@@ -181,9 +181,16 @@ def test_dispatch_queries_need_no_gpu(lib, monkeypatch):
     assert b.w2a8_tensor_core_channels(2048, 14336, 4096, 64) == 111 * 128      # 1776 tiles = 12 x 148
     assert b.w2a8_tensor_core_channels(8192, 14336, 4096, 64) == 14336          # the rest would cost more than a round
     assert b.w2a8_tensor_core_channels(2048, 4096, 14336, 64) == 4096
-    # too few output tiles for 148 SMs: streaming kernel even with many tokens
-    assert b.w2a8_kernel_for(128, 4096, 14336, 64) == "streaming"
+    # too few output tiles for 148 SMs: K is split so that every SM has work ...
+    assert b.w2a8_kernel_for(128, 4096, 14336, 64) == "tensor_core"
+    assert b.w2a8_tensor_core_ksplit(128, 4096, 14336, 64) == 4
+    assert b.w2a8_tensor_core_channels(128, 4096, 14336, 64) == 4096
+    assert b.w2a8_tensor_core_ksplit(256, 4096, 4096, 64) == 2
+    assert b.w2a8_tensor_core_ksplit(2048, 14336, 4096, 64) == 1
+    assert b.w2a8_workspace_bytes(128, 4096, 14336, 64) >= 256 + 4 * 128 * 4096 * 4
+    # ... or the streaming kernel takes it where that does not pay
     assert b.w2a8_kernel_for(64, 4096, 4096, 64) == "streaming"
+    assert b.w2a8_tensor_core_ksplit(64, 4096, 4096, 64) == 0
     # shapes the tensor-core kernel does not tile
     assert b.w2a8_kernel_for(512, 1040, 4096, 64) == "streaming"
     assert b.w2a8_kernel_for(512, 4096, 4160, 64) == "streaming"

@@ -77,6 +77,84 @@ def test_prefill_against_reference(gpu, oracle, monkeypatch, M, N, K, group, kin
     assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), float((err / np.abs(y_ref).max(axis=1)).max())
 
 
+SPLIT_CASES = [
+    # M, N, K, group, forced K splits
+    (128, 256, 2048, 64, 2),
+    (128, 256, 2048, 64, 4),        # two 256-k blocks per split: the smallest allowed
+    (200, 128, 4096, 128, 8),       # ragged token tile
+    (130, 256, 2048, 256, 4),       # a split is two groups of one block each
+    (300, 384, 3072, 512, 2),       # groups of two blocks, three per split; ragged tokens
+    (64, 4096, 1024, 64, 2),        # 64 work items
+]
+
+
+@pytest.mark.parametrize("h16", [False, True])
+@pytest.mark.parametrize("M,N,K,group,split", SPLIT_CASES)
+def test_k_split(gpu, oracle, monkeypatch, M, N, K, group, split, h16):
+    """K split of the int8 tensor-core kernel: partial outputs per split in the workspace, added in
+    split order by the second kernel.  Same result on a repeat (fixed order), within the tolerance of
+    the reference, and within a few units in the last place of the unsplit kernel's result."""
+    torch, b = gpu
+    monkeypatch.setenv("W2A8_PF_KSPLIT", str(split))
+    assert b.w2a8_kernel_for(M, N, K, group) == "tensor_core"
+    assert b.w2a8_tensor_core_ksplit(M, N, K, group) == split
+    codes, s_w = synth.make_linear(3 * M + N + K + split, K, N, group)
+    bits = synth.activations_bf16(M + K + split, M, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, group))
+    a_ref, s_ref = oracle.quantize(bits)
+    if h16:
+        s_h = s_w.astype(np.float16)
+        run = lambda w: b.w2a8_gemm_h16(a, s_a, packed, _dev(torch, s_h), group, w)
+        y_ref = oracle.gemm(a_ref, s_ref, codes, s_h.astype(np.float32), group)
+    else:
+        run = lambda w: b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), group, w)
+        y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, group)
+    y = run(ws)
+    y2 = run(ws)
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    assert torch.equal(y, y2)
+    rowmax = np.abs(y_ref).max(axis=1)
+    err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max(axis=1)
+    assert (err <= TOL * rowmax).all(), float((err / rowmax).max())
+    if h16:     # bf16 result: the same fp32 sums, rounded once by the summing kernel
+        y16 = b.w2a8_gemm_h16(a, s_a, packed, _dev(torch, s_h), group, ws, out_dtype=torch.bfloat16)
+        assert torch.equal(y16, y.to(torch.bfloat16))
+    monkeypatch.setenv("W2A8_PF_KSPLIT", "1")
+    assert b.w2a8_tensor_core_ksplit(M, N, K, group) == 1
+    y1 = run(b.new_workspace(b.w2a8_workspace_bytes(M, N, K, group)))
+    torch.cuda.synchronize()
+    diff = (y.double() - y1.double()).abs().max(dim=1).values.cpu().numpy()
+    assert (diff <= 4e-6 * rowmax).all(), float((diff / rowmax).max())      # only the order of fp32 additions differs
+
+
+def test_k_split_default_rule(gpu, oracle, monkeypatch):
+    """Default dispatch on a few-tile shape of the benchmark layer (`down` at 128 tokens: 32 output
+    tiles on 148 SMs): tensor-core kernel with K split four ways; sampled rows against the reference."""
+    torch, b = gpu
+    monkeypatch.delenv("W2A8_PREFILL", raising=False)
+    monkeypatch.delenv("W2A8_PF_KSPLIT", raising=False)
+    M, N, K, g = 128, 4096, 14336, 64
+    assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
+    assert b.w2a8_tensor_core_ksplit(M, N, K, g) == 4
+    assert b.w2a8_tensor_core_channels(M, N, K, g) == N
+    codes, s_w = synth.make_linear(4242, K, N, g)
+    bits = synth.activations_bf16(4243, M, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws).cpu().numpy()
+    assert b.w2a8_workspace_status(ws) == 0
+    rows = [0, 1, 63, 64, 127]
+    a_ref, s_ref = oracle.quantize(bits[rows])
+    assert np.array_equal(a.cpu().numpy()[rows], a_ref)
+    y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+    err = np.abs(y[rows].astype(np.float64) - y_ref).max(axis=1)
+    assert (err <= TOL * np.abs(y_ref).max(axis=1)).all()
+
+
 def test_prefill_matches_streaming_path(gpu, monkeypatch):
     """The tensor-core path and the streaming (decode) path agree on the same problem."""
     torch, b = gpu
@@ -158,7 +236,8 @@ def test_dispatch_rule(gpu, oracle, monkeypatch):
     monkeypatch.delenv("W2A8_PREFILL", raising=False)
     assert b.w2a8_kernel_for(2048, 14336, 4096, 64) == "tensor_core"
     assert b.w2a8_kernel_for(512, 4096, 14336, 64) == "tensor_core"
-    assert b.w2a8_kernel_for(128, 4096, 14336, 64) == "streaming"       # 32 tiles on 148 SMs
+    assert b.w2a8_kernel_for(128, 4096, 14336, 64) == "tensor_core"     # 32 tiles on 148 SMs: K split four ways
+    assert b.w2a8_kernel_for(64, 14336, 4096, 64) == "streaming"
     assert b.w2a8_kernel_for(64, 4096, 4096, 64) == "streaming"
     assert b.w2a8_kernel_for(256, 4096, 4096, 64) == "tensor_core"
     assert b.w2a8_kernel_for(63, 14336, 4096, 64) == "streaming"        # below the token threshold
