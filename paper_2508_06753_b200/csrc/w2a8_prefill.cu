@@ -35,6 +35,12 @@
 #include "w2a8_tc.cuh"
 
 namespace w2a8 {
+// Of every eight drained values, how many are turned into floats by the integer-add route (the rest
+// by the conversion instruction): the two routes load different pipes -- the conversion instruction
+// issues at a quarter of the rate of an integer add, the add route takes one more issue slot per two
+// values -- and a mix beats either alone (4096 -> 14336, 2048 tokens, group 64: all conversions
+// 693 TOPS, all adds 702, half and half 760, two of eight by adds 772).
+constexpr int kPfMagicOfEight = 2;
 
 // Two warp layouts (template parameter UW = unpack warps):
 //   UW = 2: 12 warps -- 2 MMA issuers, 2 unpack warps (lane 0 of the first also issues the TMA
@@ -443,7 +449,10 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                         }
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) pf_cvt_fma2<DPS == 1 || DPS == 2>(acc[j], acc[j + 1], v0[j], v0[j + 1], sc);
+                        for (int j = 0; j < 32; j += 2) {
+                            if ((j & 7) < kPfMagicOfEight) pf_cvt_fma2<DPS == 1 || DPS == 2>(acc[j], acc[j + 1], v0[j], v0[j + 1], sc);
+                            else                  pf_cvt_fma2<false>(acc[j], acc[j + 1], v0[j], v0[j + 1], sc);
+                        }
                     }
                     pf_tmem_ld_wait();                     // second half is in v1
                     {
@@ -470,7 +479,8 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; j += 2)
-                            pf_cvt_fma2<DPS == 1 || DPS == 2>(acc[32 + j], acc[32 + j + 1], v1[j], v1[j + 1], sc);
+                            if ((j & 7) < kPfMagicOfEight) pf_cvt_fma2<DPS == 1 || DPS == 2>(acc[32 + j], acc[32 + j + 1], v1[j], v1[j + 1], sc);
+                            else                  pf_cvt_fma2<false>(acc[32 + j], acc[32 + j + 1], v1[j], v1[j + 1], sc);
                     }
                 }
             }
