@@ -114,7 +114,6 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
     auto item_stage0 = [&](int item) { return (item & (nsplit - 1)) * nstages; };          // first 256-k block
     // stage buffers, 1024-byte aligned (swizzle atom = 8 rows x 128 B)
     const uint32_t smem_base = (pf_smem_u32(pf_smem_raw) + 1023u) & ~1023u;
-    unsigned char *smem_gen = pf_smem_raw + (smem_base - pf_smem_u32(pf_smem_raw));
 
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
@@ -337,7 +336,7 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 pf_tma_load_2d(dst, &act_map, k, m0, bar);
                 pf_tma_load_2d(dst + kPfHalfBytes, &act_map, k + 128, m0, bar);
             }
-            unsigned char *a_stage = smem_gen + s * kPfStageBytes;
+            const uint32_t a_stage = smem_base + s * kPfStageBytes;      // shared-space address
 #pragma unroll
             for (int i = 0; i < kUnits; ++i) {
                 const int u = ut + 64 * i;
@@ -345,11 +344,9 @@ w2a8_prefill_kernel(const __grid_constant__ CUtensorMap act_map, const PrefillPa
                 const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
 #pragma unroll
                 for (int sl = 0; sl < 4; ++sl) {    // slice sl: k = 64 sl + 16 t .. + 15 of this block
-                    uint4 v;
-                    v.x = lane_codes(ws[sl], 0); v.y = lane_codes(ws[sl], 1);
-                    v.z = lane_codes(ws[sl], 2); v.w = lane_codes(ws[sl], 3);
                     const int chunk = (4 * (sl & 1) + t) ^ (r & 7);
-                    *reinterpret_cast<uint4 *>(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16) = v;
+                    pf_st_shared_v4(a_stage + (sl >> 1) * kPfHalfBytes + r * 128 + chunk * 16,
+                                    lane_codes(ws[sl], 0), lane_codes(ws[sl], 1), lane_codes(ws[sl], 2), lane_codes(ws[sl], 3));
                 }
             }
             pf_fence_proxy_async();     // make the generic-proxy stores visible to the tensor core
