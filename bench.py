@@ -1035,6 +1035,7 @@ def prefill_probe(device, peaks, Ms=(512, 2048, 8192), reps=5):
         ms = e0.elapsed_time(e1) / reps
         tops = 2.0 * M * N * K / (ms * 1e-3) / 1e12
         by_group.append({"shape": f"{K}x{N}", "M": M, "group": g, "ms_gemm": ms, "tops": tops,
+                         "tile_tokens": b.w2a8_tensor_core_tile_tokens(M, N, K, g),
                          "frac_of_measured_int8_sustained": tops / int8_peak_sustained,
                          "status": b.w2a8_workspace_status(ws)})
         del packed, s_w_d, ws

@@ -242,6 +242,20 @@ int w2a8_tensor_core_channels(int M, int N, int K, int group);
 int w2a8_tensor_core_ksplit(int M, int N, int K, int group);
 
 /*
+ * Token rows per output tile of the tensor-core kernel that serves this shape:
+ * 0 when the streaming kernel takes the problem, else 128, or 256 for the
+ * kernel with 128-channel x 256-token tiles.  That one needs one scale per
+ * channel (group == K): a tile's accumulators then stay in tensor memory until
+ * its epilogue, every unpacked weight stage feeds twice the MACs (Sec. II-D:
+ * larger output tiles per work-group; Sec. II-C: the up-convert in shared
+ * memory), and the result is bit-equal to the 128-token kernel's.  It is taken
+ * when the cost model expects it to be faster (many tokens, enough tiles);
+ * W2A8_PF_WIDE = 0 never, 2 whenever the shape allows.  Host only.
+ * W2A8_ERR_SHAPE for a shape that is not accepted.
+ */
+int w2a8_tensor_core_tile_tokens(int M, int N, int K, int group);
+
+/*
  * w2a8_gemm_partials -- parity/debug export of the exact int32 per-group sums
  * P[m][n][gi] computed by the same inner-product code as w2a8_gemm.
  *   partials [M][N][K/group] int32, fully overwritten.

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libw2a8.so")
 EXPORTS = [
     "w2a8_version", "w2a8_status_string", "w2_packed_bytes", "w2_pack", "a8_quantize",
     "w2a8_workspace_bytes", "w2a8_workspace_init", "w2a8_workspace_status", "w2a8_gemm", "w2a8_gemm_partials",
-    "w2a8_kernel_for", "w2a8_tensor_core_channels", "w2a8_tensor_core_ksplit", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
+    "w2a8_kernel_for", "w2a8_tensor_core_channels", "w2a8_tensor_core_ksplit", "w2a8_tensor_core_tile_tokens", "w2a8_gemm_h16", "w2a16_gemm", "w2a8_linear", "w2a8_linear_host_workspace_bytes", "w2a8_linear_host", "w2a8_gemm_static",
     "w2a8_gemm_grouped", "w2a8_linear_grouped", "w2a8_grouped_workspace_bytes", "w2a8_grouped_plan",
     "w2a8_read_probe", "w2a8_tensor_core_kind",
     "w2a8_linear_grouped_host", "w2a8_linear_grouped_host_workspace_bytes",
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.w2a8_kernel_for.argtypes = [i, i, i, i]
         L.w2a8_tensor_core_channels.argtypes = [i, i, i, i]
         L.w2a8_tensor_core_ksplit.argtypes = [i, i, i, i]
+        L.w2a8_tensor_core_tile_tokens.argtypes = [i, i, i, i]
         L.w2a16_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_gemm_partials.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.w2a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
@@ -201,6 +202,13 @@ def w2a8_tensor_core_ksplit(M: int, N: int, K: int, group: int) -> int:
     """K splits of the tensor-core kernel for this shape (0: streaming kernel; host only)."""
     r = int(lib().w2a8_tensor_core_ksplit(M, N, K, group))
     _check(r if r < 0 else 0, "w2a8_tensor_core_ksplit")
+    return r
+
+
+def w2a8_tensor_core_tile_tokens(M: int, N: int, K: int, group: int) -> int:
+    """Token rows per tile of the tensor-core kernel for this shape (0: streaming kernel; host only)."""
+    r = int(lib().w2a8_tensor_core_tile_tokens(M, N, K, group))
+    _check(r if r < 0 else 0, "w2a8_tensor_core_tile_tokens")
     return r
 
 

@@ -27,6 +27,7 @@ bool prefill_supported(int M, int N, int K, int group);
 bool prefill_preferred(int M, int N, int K, int group, bool can_split);
 size_t prefill_workspace_bytes(int M, int N, int K, int group);
 int prefill_ksplit(int M, int N, int K, int group);
+bool prefill_uses_wide(int M, int N, int K, int group);
 int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
                    void *y, int32_t *partials, int M, int N, int K, int group, int *status,
                    cudaStream_t st, bool h16, bool y16, int ldy);
@@ -424,6 +425,14 @@ int w2a8_tensor_core_ksplit(int M, int N, int K, int group) {
     if (!takes_tensor_core_kernel(M, N, K, group)) return 0;
     if (tensor_core_kind_is_16(M, N, K, group)) return 1;
     return prefill_ksplit(M, N, K, group);
+}
+
+int w2a8_tensor_core_tile_tokens(int M, int N, int K, int group) {
+    ShapeInfo si;
+    if (!shape_ok(M, N, K, group, &si)) return W2A8_ERR_SHAPE;
+    if (!takes_tensor_core_kernel(M, N, K, group)) return 0;
+    if (tensor_core_kind_is_16(M, N, K, group)) return 128;
+    return prefill_uses_wide(M, N, K, group) ? 256 : 128;
 }
 
 }  // extern "C"

@@ -558,6 +558,11 @@ static double prefill_round_seconds_per_k(int group) {
     return group <= 64 ? 7.0e-9 : group <= 128 ? 4.8e-9 : group <= 256 ? 3.6e-9 : 3.0e-9;
 }
 constexpr double kStreamSecondsPerMac = 8.0e-15;    // streaming kernel, per token x weight
+// a round of 128 x 256 tiles of the one-scale-per-channel kernel (2114 TOPS at 4096 -> 14336, 2048 tokens: 6 rounds)
+constexpr double kWideRoundSecondsPerK = 4.63e-9;
+
+static double split_plan(int M, int N, int K, int tile_tokens, double round_seconds_per_k, int *channels);
+bool prefill_uses_wide(int M, int N, int K, int group);
 
 constexpr size_t kPfSplitOffset = 256;              // byte offset of the K-split partial outputs in the workspace
 
@@ -609,22 +614,28 @@ size_t prefill_workspace_bytes(int M, int N, int K, int group) {
 // the streaming one) is kept with a split.  `can_split` = false: the caller's kernel has no K split.
 bool prefill_preferred(int M, int N, int K, int group, bool can_split) {
     const int sp = can_split ? prefill_ksplit(M, N, K, group) : 1;
-    const double t_tc = prefill_seconds(M, N, K, group, sp);
+    double t_tc = prefill_seconds(M, N, K, group, sp);
+    if (can_split && prefill_uses_wide(M, N, K, group)) {
+        int c;
+        const double t_wide = split_plan(M, N, K, 256, kWideRoundSecondsPerK, &c);
+        if (t_wide < t_tc) t_tc = t_wide;
+    }
     const double t_stream = kStreamSecondsPerMac * (double)M * (double)N * (double)K;
     return t_tc * (950000.0 / 875000.0) < t_stream;
 }
 
-// How many of the N channels the tensor-core kernel should take when the rest may go to the
-// streaming kernel.  Tiles are handed out in rounds of one tile per SM (148 on B200); a last round with a handful of tiles
-// costs as much as a full one (4096x14336 at M = 512: 448 tiles = 3 rounds + 4 tiles).  Tiles are
-// ordered channel tile first, so giving the last few channel tiles (at most eight) to the
-// streaming kernel can remove that round.  Same cost model as prefill_preferred, plus 2 us for
-// the extra launch.  Returns a multiple of 128 in (0, N].
-int prefill_channel_split(int M, int N, int K, int group) {
-    if (prefill_ksplit(M, N, K, group) > 1) return N;   // few tiles: K is split instead
-    const int ct = N / kPfBM, tiles_m = (M + kPfBN - 1) / kPfBN;
+bool prefill_wide_supported(int M, int N, int K, int group);
+int launch_prefill_wide(const int8_t *a, const float *a_scale, const uint32_t *packed, const void *w_scale,
+                        void *y, int M, int N, int K, int *status, cudaStream_t st, bool h16, bool y16, int ldy);
+
+// Best way to give the first channel tiles to a tensor-core kernel with tiles of `tile_tokens` tokens and
+// the last few (at most eight) to the streaming kernel: tiles are handed out in rounds of one tile per SM
+// (148 on B200), and a last round with a handful of tiles costs as much as a full one (4096x14336 at
+// M = 512: 448 tiles = 3 rounds + 4 tiles).  Returns the estimated seconds; *channels = a multiple of 128.
+static double split_plan(int M, int N, int K, int tile_tokens, double round_seconds_per_k, int *channels) {
+    const int ct = N / kPfBM, tiles_m = (M + tile_tokens - 1) / tile_tokens;
     const long long sms = sm_count();
-    const double round_s = prefill_round_seconds_per_k(group) * K;
+    const double round_s = round_seconds_per_k * K;
     double best = 1e30;
     int best_ct = ct;
     for (int c = ct; c >= 1 && c >= ct - 8; --c) {
@@ -633,7 +644,29 @@ int prefill_channel_split(int M, int N, int K, int group) {
         if (c < ct) t += 2.0e-6 + kStreamSecondsPerMac * (double)M * (double)(ct - c) * kPfBM * (double)K;
         if (t < best * 0.97) { best = t; best_ct = c; }      // a split has to pay by 3 % or more
     }
-    return best_ct * kPfBM;
+    *channels = best_ct * kPfBM;
+    return best;
+}
+
+// One scale per channel and many tokens: whether the 256-token-tile kernel takes the shape (its round of
+// tiles costs more per k, but there are half as many tiles).  W2A8_PF_WIDE = 0 never, 2 whenever supported.
+bool prefill_uses_wide(int M, int N, int K, int group) {
+    if (!prefill_wide_supported(M, N, K, group)) return false;
+    if (env_int("W2A8_PF_WIDE", 1) == 2) return true;
+    if (prefill_ksplit(M, N, K, group) > 1) return false;
+    int c128, c256;
+    return split_plan(M, N, K, 256, kWideRoundSecondsPerK, &c256) <
+           split_plan(M, N, K, kPfBN, prefill_round_seconds_per_k(group), &c128);
+}
+
+// How many of the N channels the tensor-core kernel should take when the rest may go to the
+// streaming kernel (see split_plan).  Returns a multiple of 128 in (0, N].
+int prefill_channel_split(int M, int N, int K, int group) {
+    if (prefill_ksplit(M, N, K, group) > 1 && !prefill_uses_wide(M, N, K, group)) return N;   // few tiles: K is split instead
+    int channels;
+    if (prefill_uses_wide(M, N, K, group)) split_plan(M, N, K, 256, kWideRoundSecondsPerK, &channels);
+    else                                   split_plan(M, N, K, kPfBN, prefill_round_seconds_per_k(group), &channels);
+    return channels;
 }
 
 // Enqueue the prefill kernel.  `partials` != nullptr selects the parity export.
@@ -641,6 +674,10 @@ int launch_prefill(const int8_t *a, const float *a_scale, const uint32_t *packed
                    void *y, int32_t *partials, int M, int N, int K, int group, int *status,
                    cudaStream_t st, bool h16, bool y16, int ldy) {
     if (h16 && partials) return W2A8_ERR_SHAPE;
+    // one scale per channel and enough tokens: the 256-token-tile kernel
+    if (!partials && ldy >= N && prefill_uses_wide(M, ldy, K, group) &&
+        (N == ldy || N == prefill_channel_split(M, ldy, K, group)))
+        return launch_prefill_wide(a, a_scale, packed, w_scale, y, M, N, K, status, st, h16, y16, ldy);
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return W2A8_ERR_CUDA;
     CUtensorMap map;

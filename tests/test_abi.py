@@ -169,7 +169,7 @@ def test_dispatch_queries_need_no_gpu(lib, monkeypatch):
     """Which kernel serves a shape, and how the channels are split between the two kernels, is
     host logic: pinned here on the shapes of the benchmark configurations."""
     from paper_2508_06753_b200 import binding as b
-    for name in ("W2A8_PREFILL", "W2A8_PF_SPLIT", "W2A8_PF_KSPLIT", "W2A8_TC_KIND"):
+    for name in ("W2A8_PREFILL", "W2A8_PF_SPLIT", "W2A8_PF_KSPLIT", "W2A8_TC_KIND", "W2A8_PF_WIDE"):
         monkeypatch.delenv(name, raising=False)
     # few tokens: streaming kernel
     for M in (1, 4, 16, 32, 63):
@@ -188,6 +188,11 @@ def test_dispatch_queries_need_no_gpu(lib, monkeypatch):
     assert b.w2a8_tensor_core_ksplit(256, 4096, 4096, 64) == 2
     assert b.w2a8_tensor_core_ksplit(2048, 14336, 4096, 64) == 1
     assert b.w2a8_workspace_bytes(128, 4096, 14336, 64) >= 256 + 4 * 128 * 4096 * 4
+    # one scale per channel and many tokens: 256-token tiles
+    assert b.w2a8_tensor_core_tile_tokens(2048, 14336, 4096, 4096) == 256
+    assert b.w2a8_tensor_core_channels(2048, 14336, 4096, 4096) == 111 * 128     # 888 wide tiles = 6 x 148
+    assert b.w2a8_tensor_core_tile_tokens(2048, 14336, 4096, 64) == 128
+    assert b.w2a8_tensor_core_tile_tokens(4, 14336, 4096, 4096) == 0
     # ... or the streaming kernel takes it where that does not pay
     assert b.w2a8_kernel_for(64, 4096, 4096, 64) == "streaming"
     assert b.w2a8_tensor_core_ksplit(64, 4096, 4096, 64) == 0

@@ -155,6 +155,57 @@ def test_k_split_default_rule(gpu, oracle, monkeypatch):
     assert (err <= TOL * np.abs(y_ref).max(axis=1)).all()
 
 
+WIDE_CASES = [
+    # M, N, K: one scale per channel, 256-token tiles
+    (257, 128, 1280),       # second token tile holds one token
+    (130, 128, 512),        # ragged single tile, two 256-k blocks
+    (512, 256, 2048),
+    (1000, 384, 768),       # ragged last tile, odd number of blocks
+    (300, 19200, 256),      # 300 tiles on 148 CTAs: both accumulator buffers re-used, one block per tile
+]
+
+
+@pytest.mark.parametrize("h16", [False, True])
+@pytest.mark.parametrize("M,N,K", WIDE_CASES)
+def test_wide_tiles_one_scale_per_channel(gpu, oracle, monkeypatch, M, N, K, h16):
+    """The 256-token-tile kernel (group = K): against the reference, and bit for bit against the
+    128-token kernel (same sums, same order of the float operations)."""
+    torch, b = gpu
+    g = K
+    codes, s_w = synth.make_linear(5 * M + N + K, K, N, g)
+    bits = synth.activations_bf16(M + 3 * K, M, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    a_ref, s_ref = oracle.quantize(bits)
+    if h16:
+        s_h = s_w.astype(np.float16)
+        run = lambda **kw: b.w2a8_gemm_h16(a, s_a, packed, _dev(torch, s_h), g, ws, **kw)
+        y_ref = oracle.gemm(a_ref, s_ref, codes, s_h.astype(np.float32), g)
+    else:
+        run = lambda **kw: b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
+        y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+    monkeypatch.setenv("W2A8_PF_WIDE", "2")
+    assert b.w2a8_tensor_core_tile_tokens(M, N, K, g) == 256
+    y = run()
+    y2 = run()
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    assert torch.equal(y, y2)
+    rowmax = np.abs(y_ref).max(axis=1)
+    err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max(axis=1)
+    assert (err <= TOL * rowmax).all(), float((err / rowmax).max())
+    if h16:
+        y16 = run(out_dtype=torch.bfloat16)
+        assert torch.equal(y16, y.to(torch.bfloat16))
+    monkeypatch.setenv("W2A8_PF_WIDE", "0")
+    monkeypatch.setenv("W2A8_PF_KSPLIT", "1")
+    assert b.w2a8_tensor_core_tile_tokens(M, N, K, g) == 128
+    y128 = run()
+    torch.cuda.synchronize()
+    assert torch.equal(y, y128)
+
+
 def test_prefill_matches_streaming_path(gpu, monkeypatch):
     """The tensor-core path and the streaming (decode) path agree on the same problem."""
     torch, b = gpu
@@ -227,6 +278,39 @@ def test_prefill_full_size_sampled_rows(gpu, oracle, M, K, N, dispatch, monkeypa
     torch.cuda.synchronize()
     assert b.w2a8_workspace_status(ws2) == 0
     assert np.array_equal(P[idx].cpu().numpy(), oracle.partials(a_ref, codes[sel], g))
+
+
+@pytest.mark.parametrize("M", [2048, 1100])
+def test_wide_tiles_full_size_default_rule(gpu, oracle, monkeypatch, M):
+    """One scale per channel on the gate/up shape at the default dispatch: the 256-token-tile kernel on
+    the first 111 channel tiles and the streaming kernel on the last 128 channels (M = 2048), or a ragged
+    token count (M = 1100); sampled token rows of every channel against the reference."""
+    torch, b = gpu
+    for name in ("W2A8_PREFILL", "W2A8_PF_WIDE", "W2A8_PF_KSPLIT"):
+        monkeypatch.delenv(name, raising=False)
+    K, N = 4096, 14336
+    g = K
+    assert b.w2a8_kernel_for(M, N, K, g) == "tensor_core"
+    assert b.w2a8_tensor_core_tile_tokens(M, N, K, g) == 256
+    if M == 2048:
+        assert b.w2a8_tensor_core_channels(M, N, K, g) == 111 * 128
+    codes, s_w = synth.make_linear(5100 + M, K, N, g)
+    bits = synth.activations_bf16(5200 + M, M, K)
+    packed = b.w2_pack(_dev(torch, codes))
+    a, s_a = b.a8_quantize(_dev(torch, bits.view(np.int16)).view(torch.bfloat16))
+    ws = b.new_workspace(b.w2a8_workspace_bytes(M, N, K, g))
+    y = b.w2a8_gemm(a, s_a, packed, _dev(torch, s_w), g, ws)
+    torch.cuda.synchronize()
+    assert b.w2a8_workspace_status(ws) == 0
+    assert bool(torch.isfinite(y).all())
+    rows = sorted(set([0, 127, 128, 255, 256, 1023, 1024, M - 257, M - 256, M - 1] +
+                      [int(r) for r in np.random.default_rng(M).choice(M, size=54, replace=False)]))
+    a_ref, s_ref = oracle.quantize(bits[rows])
+    idx = torch.tensor(rows, device="cuda")
+    assert np.array_equal(a[idx].cpu().numpy(), a_ref)
+    y_ref = oracle.gemm(a_ref, s_ref, codes, s_w, g)
+    err = np.abs(y[idx].cpu().numpy().astype(np.float64) - y_ref).max(axis=1)
+    assert (err <= TOL * np.abs(y_ref).max(axis=1)).all(), float((err / np.abs(y_ref).max(axis=1)).max())
 
 
 def test_dispatch_rule(gpu, oracle, monkeypatch):
