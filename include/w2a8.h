@@ -300,11 +300,13 @@ size_t w2a8_grouped_workspace_bytes(int count, const int *N, int M, int K, int g
  *                   a8_quantize, same bits) into its shared memory.  Possible for
  *                   at most 8 tokens, K % 256 == 0 and rows that fit shared
  *                   memory; where it is not possible this behaves like _OFF.
- *   W2A8_FUSE_AUTO  _ON when the rows a CTA has to scan are small (M * K up to
- *                   8192 values; W2A8_FUSE_MAX_ELEMS in the environment), else _OFF:
+ *   W2A8_FUSE_AUTO  _OFF, unless W2A8_FUSE_MAX_ELEMS in the environment allows
+ *                   fusing up to that many values of M * K per CTA (default 0):
  *                   on B200 the separate quantiser launch hides behind the weight
- *                   prefetch of the launch that follows it, so fusing only saves a
- *                   launch on the host and costs device time from two tokens on
+ *                   prefetch of the launch that follows it, so it is the faster
+ *                   form on the device for every token count (measured: 0.5 us per
+ *                   call at one token, several us from four tokens on); fusing
+ *                   saves one launch on the host
  *   x_bf16     [M][K] bf16 bit patterns, DEVICE
  *   a, a_scale DEVICE buffers that receive what a8_quantize would write; they may
  *              be NULL when the call fuses (then nothing is written), and must

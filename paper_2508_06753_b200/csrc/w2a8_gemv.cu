@@ -38,8 +38,7 @@ namespace w2a8 {
 
 int env_int(const char *name, int dflt);
 
-constexpr int kGvWarps = 16;
-constexpr int kGvThreads = kGvWarps * 32;
+constexpr int kGvWarps = 16;                      // warps per CTA of the full-SM form (the other has 8, two CTAs per SM)
 constexpr int kGvRing = 4;                        // landing slots (cells) per warp (a power of two)
 constexpr int kGvMaxMats = 4;                     // weight matrices per launch
 constexpr int kGvWSlot = 2 * 32 * 16;             // weights of a cell: two channels x 32 lanes x 16 B
@@ -50,6 +49,8 @@ constexpr int kGvPartBytes = 32 * 1024;           // partial sums of one round (
 constexpr int kGvMaxFuseM = 8;                    // most tokens the kernel quantises itself
 constexpr int kGvMaxTokens = 32;                  // most tokens the kernel takes at all
 constexpr int kGvMaxSmem = 220 * 1024;            // dynamic shared memory the kernel may ask for
+constexpr int kGvMaxSmemHalf = 112 * 1024;        // the same for the 8-warp form (two CTAs per SM)
+constexpr int kGvPartBytesHalf = 16 * 1024;       // its partial sums of one round
 constexpr int kGvActPad = 64;                     // staged token rows are K + 64 bytes apart
 
 struct GemvMat {
@@ -79,15 +80,21 @@ struct GemvParams {
 
 // MT: 8-token slabs per virtual tile; SPP: 64-k slices per scale group (capped at 4); ONE: a single
 // token; ASMEM: activations staged in shared memory (copied, or quantised here when p.x is set);
-// BCACHE: one block per K-lane and all tokens in one tile (M <= 8 * MT): activation fragments live
-// in registers.
-template <int MT, int SPP, bool ONE, bool ASMEM, bool BCACHE>
-__global__ void __launch_bounds__(kGvThreads, 1)
+// BCACHE: NB blocks per K-lane and all tokens in one tile (M <= 8 * MT): activation fragments live
+// in registers.  W: warps per CTA.  16: one CTA per SM, NB = 1.  8: two CTAs per SM (the same warps
+// and registers per SM), NB = 2 -- a launch's CTAs then leave and arrive in units of half an SM, so
+// the head of the next launch (under programmatic dependent launch: its first ring-full of weights)
+// overlaps the tail of this one instead of waiting for a whole SM.
+template <int MT, int SPP, bool ONE, bool ASMEM, bool BCACHE, int W>
+__global__ void __launch_bounds__(W * 32, W == 8 ? 2 : 1)
 w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
+    constexpr int kThreads = W * 32;
+    constexpr int kRingBytes = W * kGvWarpBytes;
+    constexpr int NB = (BCACHE && W == 8) ? 2 : 1;      // blocks per K-lane with register-resident activations
     constexpr int SPB = 4 / SPP;                  // scales per block and channel
     constexpr int kRed = ONE ? 16 : MT * 128;     // sums a K-lane parks per tile
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ uint32_t wmax[kGvMaxFuseM][kGvWarps];
+    __shared__ uint32_t wmax[kGvMaxFuseM][W];
     __shared__ float s_scale[kGvMaxTokens];     // token scales: written here, read by the epilogue
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, t = lane & 3;
@@ -95,15 +102,15 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
     const int tl = warp % TG, ks = warp / TG;
     // this K-lane's run of blocks in every tile
     const int b0 = (ks * p.blocks) >> p.ks_shift;
-    const int n_my = BCACHE ? 1 : (((ks + 1) * p.blocks) >> p.ks_shift) - b0;
+    const int n_my = BCACHE ? NB : (((ks + 1) * p.blocks) >> p.ks_shift) - b0;
 
     unsigned char *wslots = smem + warp * kGvWarpBytes + lane * 16;
     unsigned char *sslots = smem + warp * kGvWarpBytes + kGvRing * kGvWSlot;
     const uint32_t wslots_u32 = smem_u32(wslots);
     const uint32_t sslot_u32 = smem_u32(sslots) + (lane & 15) * 16;
     const int part_floats = p.round_tiles * KS * kRed;
-    float *part_all = reinterpret_cast<float *>(smem + kGvRingBytes);
-    unsigned char *act = smem + kGvRingBytes + 2 * part_floats * 4;
+    float *part_all = reinterpret_cast<float *>(smem + kRingBytes);
+    unsigned char *act = smem + kRingBytes + 2 * part_floats * 4;
 
     // this CTA's virtual tiles: v_lo + li, li < nt_cta; this warp takes li = tl, tl + TG, ...
     const int v_lo = (int)blockIdx.x * p.per_cta + min((int)blockIdx.x, p.extra);
@@ -159,7 +166,7 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
                 for (int i = 0; i < SPB; ++i) cp_async4(sdst + 4 * i, qw.s + q_c * SPB + i);
             }
         }
-        if (BCACHE || ++q_c == n_my) {
+        if (++q_c == n_my) {
             q_c = 0;
             q_li += TG;
             if (q_li < nt_cta) {
@@ -195,7 +202,7 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
             uint32_t am[kGvMaxFuseM];
 #pragma unroll
             for (int m = 0; m < kGvMaxFuseM; ++m) am[m] = 0u;
-            for (int i = threadIdx.x; i < nvec; i += kGvThreads) {
+            for (int i = threadIdx.x; i < nvec; i += kThreads) {
 #pragma unroll
                 for (int m = 0; m < kGvMaxFuseM; ++m)
                     if (m < p.M)
@@ -212,9 +219,9 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
             }
             __syncthreads();
             for (int m = 0; m < p.M; ++m) {
-                uint32_t v = wmax[m][lane & (kGvWarps - 1)];
+                uint32_t v = wmax[m][lane & (W - 1)];
 #pragma unroll
-                for (int o = kGvWarps / 2; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+                for (int o = W / 2; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
                 float inv;
                 const float s = quant_scale(v, &inv);
                 if (threadIdx.x == 0) {
@@ -223,7 +230,7 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
                 }
                 const int8_t *xr = reinterpret_cast<const int8_t *>(p.x + (size_t)m * p.K);
                 int round = 0;
-                for (int i = threadIdx.x; i < nvec; i += kGvThreads, ++round) {
+                for (int i = threadIdx.x; i < nvec; i += kThreads, ++round) {
                     const uint4 xv = ld_act16(xr + 16 * i);
                     uint2 o;
                     o.x = quant4(xv.x, xv.y, inv);
@@ -237,7 +244,7 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
         } else {
             const int nvec = p.K >> 4;                    // 16-byte vectors per int8 row
             for (int m = 0; m < p.M; ++m)
-                for (int i = threadIdx.x; i < nvec; i += kGvThreads)
+                for (int i = threadIdx.x; i < nvec; i += kThreads)
                     *reinterpret_cast<uint4 *>(act + (size_t)m * p.act_stride + 16 * i) =
                         ld_act16(p.a + (size_t)m * p.K + 16 * i);
         }
@@ -251,15 +258,17 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
         if constexpr (ASMEM) return act_ptr(act_u32 + row * p.act_stride + kb * kBlockK + t * 16);
         else                 return p.a + (size_t)row * p.K + kb * kBlockK + t * 16;
     };
-    uint4 B[MT][4];
+    uint4 B[NB][MT][4];
     if constexpr (BCACHE) {
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-            const int8_t *src = act_at(min(8 * mt + gq, p.M - 1), b0);
+        for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-            for (int s = 0; s < 4; ++s)
-                B[mt][s] = ASMEM ? ld_act16_smem(src + s * kSliceK) : ld_act16(src + s * kSliceK);
-        }
+            for (int mt = 0; mt < MT; ++mt) {
+                const int8_t *src = act_at(min(8 * mt + gq, p.M - 1), b0 + nb);
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    B[nb][mt][s] = ASMEM ? ld_act16_smem(src + s * kSliceK) : ld_act16(src + s * kSliceK);
+            }
     }
 
     // ---- compute side ---------------------------------------------------------------------
@@ -281,27 +290,32 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
             }
         };
         if constexpr (BCACHE) {
-            // one cell per tile; four tiles per trip so that the slot offsets are immediates
-            // (rounds are multiples of 4 * TG tiles, so every round starts at slot 0)
-            for (int li = tl; li < nt; li += kGvRing * TG) {
+            // NB cells per tile; a ring-full of tiles per trip so that the slot offsets are immediates
+            // (rounds are multiples of that many tiles per warp, so every round starts at slot 0)
+            constexpr int kTrip = kGvRing / NB;
+            for (int li = tl; li < nt; li += kTrip * TG) {
 #pragma unroll
-                for (int u = 0; u < kGvRing; ++u) {
+                for (int u = 0; u < kTrip; ++u) {
                     if (li + u * TG < nt) {                       // warp-uniform
-                        cp_async_wait_group<kGvRing - 1>();
-                        __syncwarp();                             // the scales were copied by other lanes
-                        const uint4 wa = *reinterpret_cast<const uint4 *>(wslots + u * kGvWSlot);
-                        const uint4 wb = *reinterpret_cast<const uint4 *>(wslots + u * kGvWSlot + 32 * 16);
-                        const unsigned char *sc0 = sslots + u * kGvSSlot + gq * 16;
                         float acc[MT][4];
 #pragma unroll
                         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                             for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
-                        compute_cell_breg<MT, SPP, ONE>(wa, wb, sc0, sc0 + 8 * 16, B, acc);
+#pragma unroll
+                        for (int nb = 0; nb < NB; ++nb) {
+                            const int sl = u * NB + nb;           // a constant after unrolling
+                            cp_async_wait_group<kGvRing - 1>();
+                            __syncwarp();                         // the scales were copied by other lanes
+                            const uint4 wa = *reinterpret_cast<const uint4 *>(wslots + sl * kGvWSlot);
+                            const uint4 wb = *reinterpret_cast<const uint4 *>(wslots + sl * kGvWSlot + 32 * 16);
+                            const unsigned char *sc0 = sslots + sl * kGvSSlot + gq * 16;
+                            compute_cell_breg<MT, SPP, ONE>(wa, wb, sc0, sc0 + 8 * 16, B[nb], acc);
+                            __syncwarp();                         // every lane has read the slot
+                            if (q_li < nt_cta) request(sl);
+                            cp_async_commit();
+                        }
                         park(li + u * TG, acc);
-                        __syncwarp();                             // every lane has read the slot
-                        if (q_li < nt_cta) request(u);
-                        cp_async_commit();
                     }
                 }
             }
@@ -343,7 +357,7 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
 
         // ---- the round's outputs: K-lanes of a tile in lane order, scale, store ----------------
         const float *rpart = part_all + buf * part_floats;
-        for (int e = threadIdx.x; e < nt * kRed; e += kGvThreads) {
+        for (int e = threadIdx.x; e < nt * kRed; e += kThreads) {
             const int li = e / kRed, r = e % kRed;
             Where ow;
             locate(v_lo + rbase + li, ow);
@@ -360,12 +374,12 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
             // all K-lane sums of the output are fetched first (independent loads), then added in
             // lane order: the order, and with it the bits of y, does not depend on anything else
             const float *src = rpart + li * KS * kRed + r;
-            float part[kGvWarps];
+            float part[W];
 #pragma unroll
-            for (int k2 = 0; k2 < kGvWarps; ++k2) part[k2] = k2 < KS ? src[k2 * kRed] : 0.f;
+            for (int k2 = 0; k2 < W; ++k2) part[k2] = k2 < KS ? src[k2 * kRed] : 0.f;
             float v = 0.f;
 #pragma unroll
-            for (int k2 = 0; k2 < kGvWarps; ++k2) v += part[k2];
+            for (int k2 = 0; k2 < W; ++k2) v += part[k2];
             ow.y[(size_t)mm * ow.ldy + nn] = v * (s_scale[mm] * (1.0f / kCodeGain));
         }
     }
@@ -374,8 +388,23 @@ w2a8_gemv_kernel(const __grid_constant__ GemvParams p) {
 // ---- host side ---------------------------------------------------------------------------
 struct GemvPlan {
     int mt, slabs, vtiles, ks_shift, tg, round_tiles, grid, asmem, bcache, act_stride, s_vec;
+    int warps;                  // warps per CTA: 16 (one CTA per SM) or 8 (two)
     size_t smem;
 };
+
+// Warps per CTA for a problem: the 8-warp form (two CTAs per SM) for up to eight tokens when its
+// shared memory fits twice into an SM with the activations staged (so that the fused and the
+// unfused call of a shape run the same form).  A function of M and K alone, like the K-lanes: the
+// bits of y do not depend on how the matrices of a layer are grouped into launches.
+// W2A8_GEMV_WARPS = 8 / 16 overrides (8 only where it fits).
+static int gemv_warps(int M, int K) {
+    const bool fits = M <= 8 && (size_t)8 * kGvWarpBytes + 2 * (size_t)kGvPartBytesHalf + (size_t)M * (K + kGvActPad) <=
+                                    (size_t)kGvMaxSmemHalf;
+    const int forced = env_int("W2A8_GEMV_WARPS", 0);
+    if (forced == 16) return 16;
+    if (forced == 8) return fits ? 8 : 16;
+    return fits ? 8 : 16;
+}
 
 // Whether this kernel serves the shape at all: whole 256-k blocks only (a ragged last block is
 // left to the one-shot streaming kernel), at most kGvMaxTokens tokens.  W2A8_GEMV=0 switches the
@@ -428,41 +457,51 @@ bool gemv_preferred(int M, int K, int group, int tiles, int count) {
 // The kernel can quantise the activations itself for this many tokens and this K.
 bool gemv_can_fuse(int M, int K, int group) {
     if (!gemv_supported(M, K, group) || M > kGvMaxFuseM) return false;
+    if (gemv_warps(M, K) == 8) return true;      // by construction of gemv_warps
     return (size_t)M * (K + kGvActPad) <= (size_t)(kGvMaxSmem - kGvRingBytes - 2 * kGvPartBytes);
 }
 
 // The paper exposes the abs-max scales "inside the GEMM or in a kernel of their own" as a knob
 // (Sec. II-D) and finds the fused form ahead for GEMV-sized problems only.  Here every CTA repeats
-// the abs-max, so the rule is by the values a CTA has to scan, M * K.  Measured on B200 (us per
-// call, fused / quantiser launch + persistent kernel): one token, K = 4096: 5.2 / 5.2 (q|k|v), 4.7 /
-// 4.7 (o), 11.0 / 10.9 (gate|up); one token, K = 14336: 9.1 / 8.3; four tokens, K = 4096: 7.6 / 5.3;
-// eight: 11.0 / 5.8.  Under programmatic dependent launch the quantiser launch hides behind the
-// weight prefetch of the kernel that follows it, so fusing gains nothing on the device even for
-// one token and loses from two tokens on; what it saves is one launch on the host.
+// the abs-max, and under programmatic dependent launch a separate quantiser launch hides behind the
+// weight prefetch of the kernel that follows it.  Measured on B200 (us per call, fused / quantiser
+// launch + persistent kernel): one token, K = 4096: 5.3 / 4.75 (q|k|v), 4.7 / 4.2 (o), 10.7 / 10.1
+// (gate|up); one token, K = 14336: 9.3 / 7.7; four tokens, K = 4096: 8.8 / 5.2; eight: 13.9 / 5.7.  So
+// the separate launch is ahead everywhere on the device (the layer pass at one token: 25.9 against
+// 28.3 us); what fusing saves is one launch on the host.  The automatic rule therefore fuses only up
+// to W2A8_FUSE_MAX_ELEMS values of M * K per CTA (default 0: never; W2A8_FUSE_ON asks for it).
 bool gemv_fuse_preferred(int M, int K, int group) {
     if (!gemv_can_fuse(M, K, group)) return false;
-    return (long long)M * K <= (long long)env_int("W2A8_FUSE_MAX_ELEMS", 8192);
+    return (long long)M * K <= (long long)env_int("W2A8_FUSE_MAX_ELEMS", 0);
 }
 
 static GemvPlan gemv_plan(int M, int K, int tiles, const ShapeInfo &si, bool fused) {
     GemvPlan pl;
     pl.mt = M <= 8 ? 1 : 2;
     pl.slabs = (M + 8 * pl.mt - 1) / (8 * pl.mt);
-    // K-lanes per tile: 16 when the row has at least 16 blocks, else 8, else 4 (with 2, 3 tiles
-    // side by side).  A function of K alone.
-    const int ks = si.blocks >= 16 ? 16 : si.blocks >= 8 ? 8 : 4;
-    pl.ks_shift = ks == 16 ? 4 : ks == 8 ? 3 : 2;
-    pl.tg = kGvWarps / ks;
-    pl.bcache = pl.slabs == 1 && si.blocks == ks && env_int("W2A8_GEMV_BCACHE", 1) != 0;
+    pl.warps = gemv_warps(M, K);
+    const int ctas_per_sm = 16 / pl.warps;
+    // K-lanes per tile with 16 warps: 16 when the row has at least 16 blocks, else 8, else 4 (with 2, 4
+    // tiles side by side); half as many with 8 warps.  A function of M and K alone.
+    const int ks16 = si.blocks >= 16 ? 16 : si.blocks >= 8 ? 8 : 4;
+    const int ks = ks16 / ctas_per_sm;
+    pl.ks_shift = ks == 16 ? 4 : ks == 8 ? 3 : ks == 4 ? 2 : 1;
+    pl.tg = pl.warps / ks;
+    // register-resident activations: a K-lane holds one block (16 warps) or two (8 warps)
+    pl.bcache = pl.slabs == 1 && si.blocks == ks16 && env_int("W2A8_GEMV_BCACHE", 1) != 0;
+    const int nb = pl.bcache ? ctas_per_sm : 1;
     pl.vtiles = tiles * pl.slabs;
-    const int sms = sm_count();
+    const int sms = sm_count() * ctas_per_sm;
     pl.grid = pl.vtiles < sms ? pl.vtiles : sms;
+    const int ring_bytes = pl.warps * kGvWarpBytes;
+    const int part_budget = pl.warps == 8 ? kGvPartBytesHalf : kGvPartBytes;
+    const size_t max_smem = pl.warps == 8 ? kGvMaxSmemHalf : kGvMaxSmem;
     // tiles per round: what one partial buffer holds, no more than a CTA has, in units that keep
     // the ring aligned (see the BCACHE loop)
     const int red_floats = (M == 1) ? 16 : pl.mt * 128;
-    const int unit = pl.bcache ? kGvRing * pl.tg : pl.tg;
+    const int unit = pl.bcache ? (kGvRing / nb) * pl.tg : pl.tg;
     const int per_cta = (pl.vtiles + pl.grid - 1) / pl.grid;
-    int fit = kGvPartBytes / (ks * red_floats * 4) / unit * unit;
+    int fit = part_budget / (ks * red_floats * 4) / unit * unit;
     if (fit < unit) fit = unit;
     const int need = (per_cta + unit - 1) / unit * unit;
     pl.round_tiles = need < fit ? need : fit;
@@ -474,18 +513,27 @@ static GemvPlan gemv_plan(int M, int K, int tiles, const ShapeInfo &si, bool fus
     // (their B-fragment loads from L1 touch eight lines each), or on request
     const int forced = env_int("W2A8_GEMV_ASMEM", -1);
     pl.asmem = fused ? 1 : (forced >= 0 ? (forced != 0) : (pl.mt == 2)) &&
-                           kGvRingBytes + part_bytes + act_bytes <= (size_t)kGvMaxSmem;
-    pl.smem = (size_t)kGvRingBytes + part_bytes + (pl.asmem ? act_bytes : 0);
+                           ring_bytes + part_bytes + act_bytes <= max_smem;
+    pl.smem = (size_t)ring_bytes + part_bytes + (pl.asmem ? act_bytes : 0);
     return pl;
+}
+
+template <int MT, int SPP, bool ONE, bool ASMEM, bool BCACHE, int W>
+static cudaError_t launch_gemv_w(const GemvParams &p, const GemvPlan &pl, cudaStream_t st) {
+    static PerDeviceFlags configured;   // per kernel instantiation
+    if (cudaError_t e = allow_dynamic_smem(w2a8_gemv_kernel<MT, SPP, ONE, ASMEM, BCACHE, W>, configured,
+                                           W == 8 ? kGvMaxSmemHalf : kGvMaxSmem))
+        return e;
+    return launch_kernel(w2a8_gemv_kernel<MT, SPP, ONE, ASMEM, BCACHE, W>, dim3(pl.grid), dim3(W * 32), pl.smem, st,
+                         pdl_enabled(), p);
 }
 
 template <int MT, int SPP, bool ONE, bool ASMEM, bool BCACHE>
 static cudaError_t launch_gemv_inst(const GemvParams &p, const GemvPlan &pl, cudaStream_t st) {
-    static PerDeviceFlags configured;   // per kernel instantiation
-    if (cudaError_t e = allow_dynamic_smem(w2a8_gemv_kernel<MT, SPP, ONE, ASMEM, BCACHE>, configured, kGvMaxSmem))
-        return e;
-    return launch_kernel(w2a8_gemv_kernel<MT, SPP, ONE, ASMEM, BCACHE>, dim3(pl.grid), dim3(kGvThreads), pl.smem, st,
-                         pdl_enabled(), p);
+    if constexpr (MT == 1) {
+        if (pl.warps == 8) return launch_gemv_w<MT, SPP, ONE, ASMEM, BCACHE, 8>(p, pl, st);
+    }
+    return launch_gemv_w<MT, SPP, ONE, ASMEM, BCACHE, 16>(p, pl, st);
 }
 
 template <int MT, int SPP, bool ONE>

@@ -139,7 +139,12 @@ def test_grouped_plan_needs_no_gpu(lib, monkeypatch):
                  "W2A8_CLUSTER", "W2A8_MIN_WARPS", "W2A8_RELAX"):
         monkeypatch.delenv(name, raising=False)
     qkv, gateup = [4096, 1024, 1024], [14336, 14336]
+    assert b.w2a8_grouped_plan(qkv, 1, 4096, 64) == {"one_launch": True, "fused": False}       # the separate quantiser is ahead on the device
+    assert b.w2a8_grouped_plan(qkv, 1, 4096, 64, b.FUSE_ON) == {"one_launch": True, "fused": True}
+    monkeypatch.setenv("W2A8_FUSE_MAX_ELEMS", "8192")
     assert b.w2a8_grouped_plan(qkv, 1, 4096, 64) == {"one_launch": True, "fused": True}
+    assert b.w2a8_grouped_plan(qkv, 4, 4096, 64) == {"one_launch": True, "fused": False}
+    monkeypatch.delenv("W2A8_FUSE_MAX_ELEMS")
     assert b.w2a8_grouped_plan(qkv, 4, 4096, 64) == {"one_launch": True, "fused": False}
     assert b.w2a8_grouped_plan(qkv, 16, 4096, 64) == {"one_launch": True, "fused": False}
     assert b.w2a8_grouped_plan(gateup, 4, 4096, 64) == {"one_launch": True, "fused": False}
