@@ -39,8 +39,8 @@ NOMINAL_HBM_GBS = 8000.0
 # launch are 18,411,524.
 NCU_TRAFFIC_BYTES_GATE_M1 = 18_378_752
 # the same for one grouped launch of the persistent kernel on gate|up, 4096x(14336+14336), M=1:
-# 36,818,948 algorithmic bytes, 36,736,256 read from DRAM (the activations come from L2), 0 written
-NCU_TRAFFIC_BYTES_GATEUP_M1 = 36_736_256
+# 36,818,948 algorithmic bytes, 36,734,720 read from DRAM (the activations come from L2), 256 written
+NCU_TRAFFIC_BYTES_GATEUP_M1 = 36_734_976
 
 
 # --------------------------------------------------------------------- accounting
@@ -920,7 +920,7 @@ def run_ours(args):
     roofline = {"bound": "hbm", "achieved": dom["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": dom["gbs"] / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES_GATEUP_M1,
                 "peak_source": peaks["source"],
-                "kernel": "w2a8_gemv_kernel<MT=1,SPP=1,ONE,BCACHE> (persistent) on gate|up 4096x(14336+14336) as one "
+                "kernel": "w2a8_gemv_kernel<MT=1,SPP=1,ONE,BCACHE,W=8> (persistent, two 8-warp CTAs per SM) on gate|up 4096x(14336+14336) as one "
                           "grouped launch, M=1: the launch with the largest share of the step (the other large "
                           "launches, and the one-shot kernel on gate alone, are in roofline_by_m)",
                 "bytes_per_launch": dom["bytes_per_launch"], "us_per_launch": dom["us_per_launch"],
