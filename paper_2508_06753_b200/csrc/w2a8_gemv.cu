@@ -438,7 +438,9 @@ bool gemv_supported(int M, int K, int group) {
 // of matrices that are latency-bound one by one, on problems of more than one such wave, and
 // where a K-lane is a single block so that the activation fragments stay in registers (K <= 4096,
 // at most 16 tokens) unless the problem is a single matrix near the one-wave size.  (The table was
-// taken before the register-resident form existed for 9 .. 16 tokens.)
+// taken before the register-resident form existed for 9 .. 16 tokens and before the 8-warp form: with
+// that one the persistent side reads 4.75 / 4.2 / 10.1 / 7.7 at one token and 5.2 / 4.5 / 11.4 / 9.8 at
+// four for q|k|v / o / gate|up / down, which leaves the choices as they are.)
 // W2A8_GEMV=2: whenever it serves the shape; W2A8_GEMV=0: never.
 bool gemv_preferred(int M, int K, int group, int tiles, int count) {
     if (!gemv_supported(M, K, group)) return false;
