@@ -220,3 +220,44 @@ def test_dispatch_queries_need_no_gpu(lib, monkeypatch):
     assert with_split >= b.w2a8_workspace_bytes(512, 14336, 4096, 64) > 0
     with pytest.raises(b.W2A8Error):
         b.w2a8_kernel_for(4, 100, 4096, 64)
+
+
+def test_dispatch_plan_invariants(lib, monkeypatch):
+    """Host-side planning on random accepted shapes: what the report functions say is consistent
+    (no device needed): channel splits are whole 128-channel tiles, K splits are whole 256-k blocks
+    and whole scale groups of at least two blocks, the workspace covers the partial outputs, 256-token
+    tiles only with one scale per channel."""
+    import random
+    from paper_2508_06753_b200 import binding as b
+    for name in ("W2A8_PREFILL", "W2A8_PF_SPLIT", "W2A8_PF_KSPLIT", "W2A8_TC_KIND", "W2A8_PF_WIDE", "W2A8_GEMV"):
+        monkeypatch.delenv(name, raising=False)
+    rng = random.Random(5)
+    seen_tc = seen_split = seen_wide = 0
+    for _ in range(400):
+        M = rng.choice([1, 8, 33, 64, 96, 128, 200, 256, 512, 1000, 2048, 4096])
+        N = 16 * rng.choice([1, 8, 64, 256, 512, 896, 1024, 1792])
+        K = 64 * rng.choice([1, 4, 8, 16, 32, 64, 128, 224])
+        g = rng.choice([64, 128, 256, K])
+        if K % g or (g not in (64, 128) and g % 256 and g != K):
+            continue
+        kernel = b.w2a8_kernel_for(M, N, K, g)
+        ch, sp, tok = (b.w2a8_tensor_core_channels(M, N, K, g), b.w2a8_tensor_core_ksplit(M, N, K, g),
+                       b.w2a8_tensor_core_tile_tokens(M, N, K, g))
+        ws = b.w2a8_workspace_bytes(M, N, K, g)
+        assert ws >= 4 and ws % 16 == 0
+        if kernel == "streaming":
+            assert (ch, sp, tok) == (0, 0, 0)
+            continue
+        seen_tc += 1
+        assert M >= 64 and N % 128 == 0 and K % 256 == 0
+        assert 0 < ch <= N and ch % 128 == 0 and N - ch <= 8 * 128
+        assert sp in (1, 2, 4, 8) and tok in (128, 256)
+        if sp > 1:
+            seen_split += 1
+            assert ch == N and tok == 128
+            assert (K // sp) % 256 == 0 and (K // sp) % g == 0 and K // sp >= 512
+            assert ws >= 256 + sp * M * N * 4
+        if tok == 256:
+            seen_wide += 1
+            assert g == K and M >= 129 and sp == 1
+    assert seen_tc > 20 and seen_split > 0 and seen_wide > 0
